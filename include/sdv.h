@@ -1,0 +1,200 @@
+/*
+ * sdv — speculative-decoding verify path on one NVIDIA B200 (sm_100a).
+ *
+ * One sdv_ctx holds one sequence: the model weights (re-laid out for streaming), a bf16 KV
+ * cache with a committed length L, the token history (request context followed by generated
+ * tokens) and a small device-resident state block.  The calls follow the online workflow of
+ * the paper (Sec. 4.1): chunked prefill of the request context, then repeatedly draft ->
+ * verify -> accept/commit.
+ *
+ * Conventions
+ *   - Every function returns an int status: SDV_OK (0) or a negative SDV_E* code.  Nothing
+ *     throws, aborts or prints.  sdv_strerror() names a code; sdv_last_cuda_error() gives the
+ *     CUDA runtime code behind the last SDV_ECUDA.
+ *   - "host" pointers are ordinary CPU memory; "dev" pointers are CUDA device memory on the
+ *     current device.  The caller owns every buffer it passes in, including the workspace,
+ *     which must outlive the context and be 256-byte aligned.
+ *   - All GPU work is ordered on the stream given to sdv_create (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream).  Calls that hand values back to the host
+ *     synchronise that stream; calls given NULL output pointers do not.
+ *   - A context is not thread-safe.  There is no CPU fallback: without a usable CUDA device
+ *     every call that would launch work returns SDV_ECUDA.
+ */
+#ifndef SDV_H_
+#define SDV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    SDV_OK = 0,
+    SDV_EINVAL = -1,    /* bad argument or unsupported shape */
+    SDV_ENOMEM = -2,    /* workspace too small */
+    SDV_ECAPACITY = -3, /* KV cache / history would exceed max_seq */
+    SDV_ESTATE = -4,    /* call order: e.g. verify before prefill finished, commit without verify */
+    SDV_ECUDA = -5,     /* CUDA runtime error, see sdv_last_cuda_error() */
+    SDV_ETIMEOUT = -6   /* a bounded device-side wait ran out; the context must be re-created */
+};
+
+#define SDV_K_MAX 16 /* longest draft per verify step (M = k+1 <= 17 rows) */
+
+typedef struct sdv_ctx sdv_ctx;
+
+/* Model shape and drafter settings.  Supported: head_dim 64 or 128; d_model and d_ffn multiples
+ * of 64; vocab a multiple of 16; n_q_heads a multiple of n_kv_heads with at most 8 query heads
+ * per KV head and (n_q_heads / n_kv_heads) * (k_max + 1) <= 128; 1 <= k_max <= SDV_K_MAX;
+ * 1 <= ngram_min <= ngram_n <= 8. */
+typedef struct {
+    int n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    int max_seq;        /* KV rows / history entries the context can hold */
+    int k_max;          /* largest draft length that will be verified */
+    int tied_lm_head;   /* LM head shares the embedding matrix */
+    int qkv_bias;       /* q, k, v projections carry a bias */
+    int ngram_n;        /* longest history suffix the drafter tries to match */
+    int ngram_min;      /* shortest suffix match that still yields a draft */
+    int search_history; /* 0: drafter searches the request context only; 1: context + generated tokens */
+    float rope_theta, rms_eps;
+} sdv_config;
+
+/* Weights as the caller holds them: bf16 bit patterns, row-major [out_features][in_features]
+ * (matrices) and fp32 vectors.  Pointers may be host or device memory.  Biases are read only
+ * when qkv_bias is set; lm_head is read only when tied_lm_head is 0. */
+typedef struct {
+    const uint16_t *wq, *wk, *wv; /* [n_q*hd][d], [n_kv*hd][d], [n_kv*hd][d] */
+    const uint16_t *wo;           /* [d][n_q*hd] */
+    const uint16_t *wg, *wu;      /* [f][d] */
+    const uint16_t *wd;           /* [d][f] */
+    const float *norm1, *norm2;   /* [d] RMSNorm scales before attention / before the FFN */
+    const float *bq, *bk, *bv;    /* [n_q*hd], [n_kv*hd], [n_kv*hd] or NULL */
+} sdv_layer_weights;
+
+typedef struct {
+    const uint16_t *emb;             /* [vocab][d] */
+    const uint16_t *lm_head;         /* [vocab][d] or NULL when tied */
+    const float *final_norm;         /* [d] */
+    const sdv_layer_weights *layers; /* [n_layers] */
+} sdv_weights;
+
+/* Bytes of device workspace sdv_create needs for this configuration (0 if it is invalid). */
+size_t sdv_workspace_bytes(const sdv_config *cfg);
+
+/* Creates a context inside caller-provided device memory (dev_workspace, bytes).  The context
+ * keeps the pointer; it allocates only a small host structure and a pinned host staging page.
+ * Errors: SDV_EINVAL (shape), SDV_ENOMEM (bytes too small), SDV_ECUDA. */
+int sdv_create(const sdv_config *cfg, void *dev_workspace, size_t bytes, void *cuda_stream, sdv_ctx **out);
+
+/* Copies the weights into the workspace, re-laid out in the order the kernels stream them.
+ * Synchronises the stream.  May be called again to replace the weights. */
+int sdv_load_weights(sdv_ctx *ctx, const sdv_weights *w);
+
+/* Chunked prefill (paper Sec. 4.1 "the prompt is split into fixed-size chunks", Sec. 4.2 graph
+ * equivalence): appends n context tokens (host int32, each in [0, vocab)) to the history, runs
+ * the decoder over them at positions L..L+n-1 and advances L by n.  Chunks of any length n >= 1
+ * give the same cache as one long call.  With is_last != 0 the logits of the last token are
+ * reduced to the first generated token T (greedy), which becomes the pending token and is
+ * appended to the history; drafting and verification may start afterwards.  Synchronises.
+ * Errors: SDV_ESTATE after the last chunk, SDV_ECAPACITY, SDV_EINVAL. */
+int sdv_prefill_chunk(sdv_ctx *ctx, const int32_t *host_tokens, int n, int is_last);
+
+/* Retrieval drafter (paper Sec. 3.2 / Sec. 5.5: drafts come from the request context by
+ * matching the current suffix and copying what followed).  Finds the position p of the search
+ * array whose preceding tokens share the longest suffix (at most ngram_n, at least ngram_min
+ * tokens) with the history, preferring the latest among equally long matches, and copies up to
+ * k tokens after p into the device draft buffer.  host_draft (k ints) and draft_len may be NULL;
+ * if either is given the stream is synchronised.  draft_len may be less than k, or 0. */
+int sdv_draft(sdv_ctx *ctx, int k, int32_t *host_draft, int *draft_len);
+
+/* Verify step (paper Sec. 3.2 "verifies them in parallel", Sec. 4.4: x = [T, x_1..x_n],
+ * y = [y_1..y_{n+1}]): runs the decoder once over the pending token T and the drafts at
+ * positions L..L+n, writing their KV rows speculatively, takes the greedy token y_{j+1} of
+ * every row (lowest id wins ties) and the accept length a = number of leading x_i == y_i.
+ * host_draft != NULL: verify these draft_len tokens (0 <= draft_len <= k_max).
+ * host_draft == NULL: verify the draft left by the last sdv_draft (draft_len is ignored; k+1
+ *   rows are computed, rows past the drafter's own draft length are padding and never accepted).
+ * host_y (draft_len+1 ints; k_max+1 is always enough) and accept_len may be NULL; if either is
+ * given the stream is synchronised.  Nothing is committed: L, T and the history are unchanged.
+ * Errors: SDV_ESTATE before prefill has finished, SDV_ECAPACITY, SDV_EINVAL, SDV_ETIMEOUT. */
+int sdv_verify(sdv_ctx *ctx, const int32_t *host_draft, int draft_len, int32_t *host_y, int *accept_len);
+
+/* Commit / rollback (paper Sec. 3.2: tokens after the first mismatch are discarded; Sec. 4.4:
+ * the accepted prefix is x_1..x_{e-1}, y_e): emits x_1..x_a, y_{a+1} of the last verify, cut to
+ * max_emit tokens when max_emit > 0; appends them to the history; L += number emitted; the last
+ * emitted token becomes the pending token.  KV rows beyond the new L are simply left behind.
+ * host_emitted (k_max+1 ints), n_emitted and kv_len may be NULL.  Always synchronises.
+ * Errors: SDV_ESTATE when no verify result is outstanding. */
+int sdv_commit(sdv_ctx *ctx, int max_emit, int32_t *host_emitted, int *n_emitted, int *kv_len);
+
+/* Sets L to new_kv_len (1 <= new_kv_len <= current L): the history is cut to new_kv_len + 1
+ * tokens and its last token becomes the pending token again. */
+int sdv_rollback(sdv_ctx *ctx, int new_kv_len);
+
+/* Current committed KV length L, or a negative error code. */
+int sdv_kv_len(const sdv_ctx *ctx);
+
+/* Parity mode: when on, every verify (and the last prefill chunk) also stores the fp32 logits of
+ * all rows so that sdv_get_logits can return them.  Off by default (it adds rows x vocab x 4
+ * bytes of writes per step). */
+int sdv_set_parity_mode(sdv_ctx *ctx, int on);
+int sdv_get_logits(sdv_ctx *ctx, float *host_logits, int rows); /* [rows][vocab] of the last verify */
+
+/* Frees the host-side structure; never touches the workspace. */
+int sdv_destroy(sdv_ctx *ctx);
+
+const char *sdv_strerror(int code);
+int sdv_last_cuda_error(const sdv_ctx *ctx);
+
+/* Verify-step accounting: bytes a step over `rows` rows at KV length kv_len has to move once
+ * (all linear weights; KV rows read + written), as defined by the shapes alone. */
+int sdv_step_bytes(const sdv_ctx *ctx, int rows, int kv_len, double *weight_bytes, double *kv_bytes);
+
+/* ---- entry points for tests and measurement ------------------------------------------------
+ * They run the same device code as the calls above on caller-supplied state. */
+
+/* Replaces the token history by hist[0..hist_len) of which the first n_ctx tokens are the request
+ * context, without running the model (drafter tests).  L becomes hist_len - 1. */
+int sdv_debug_set_history(sdv_ctx *ctx, const int32_t *host_hist, int hist_len, int n_ctx);
+
+/* Runs the accept scan on host-given predictions y (draft_len+1 ints) against host-given drafts,
+ * leaving the result where sdv_commit expects it. */
+int sdv_debug_accept(sdv_ctx *ctx, const int32_t *host_draft, int draft_len, const int32_t *host_y,
+                     int *accept_len);
+
+/* Like sdv_commit, but with a caller-chosen accept length (<= draft_len of the last verify) and
+ * next token: teacher forcing for step-by-step comparisons. */
+int sdv_debug_force_commit(sdv_ctx *ctx, int accept_len, int32_t next_token);
+
+/* Copies rows [pos0, pos0+n) of one layer's key (which = 0) or value (which = 1) cache to the
+ * host as fp32 [n_kv_heads][n][head_dim]. */
+int sdv_debug_read_kv(sdv_ctx *ctx, int layer, int which, int pos0, int n, float *host_out);
+
+/* Copies the residual stream of the last forward pass, fp32 [rows][d_model]. */
+int sdv_debug_read_hidden(sdv_ctx *ctx, int rows, float *host_out);
+
+/* Y[M][N] = X[M][K] * W[N][K]^T with the verify path's weight-streaming GEMM (bf16 operands, fp32
+ * accumulate).  host_x fp32 [M][K] (rounded to bf16 on the way in), host_w bf16 bits [N][K],
+ * host_y fp32 [M][N]; M <= 32, N % 16 == 0, K % 64 == 0, K <= max(d_model, d_ffn, n_q*hd) and
+ * N*K*2 bytes no larger than max(64 MiB, one layer's gate+up matrices).  dev_ms (optional)
+ * receives the kernel's device time in milliseconds. */
+int sdv_debug_gemm(sdv_ctx *ctx, const float *host_x, const uint16_t *host_w, float *host_y, int M, int N, int K,
+                   float *dev_ms);
+
+/* Launches a one-thread kernel that waits, with a limit of a few milliseconds, on a flag nothing
+ * ever sets; returns SDV_ETIMEOUT when the bounded wait reported its expiry as designed (the
+ * context stays usable), SDV_OK if the wait wrongly succeeded. */
+int sdv_debug_timeout_probe(sdv_ctx *ctx);
+
+/* Number of kernels launched by this context since creation. */
+long long sdv_launch_count(const sdv_ctx *ctx);
+
+/* Device time in milliseconds of the last forward kernel launched by sdv_verify (CUDA events on
+ * the context's stream; synchronises on the closing event). */
+int sdv_last_verify_ms(sdv_ctx *ctx, float *ms);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDV_H_ */

@@ -1,0 +1,776 @@
+// C-ABI of the verify-path library (see include/sdv.h): context set-up, the static work
+// partition, weight re-layout, and the launch sequences of prefill / draft / verify / commit.
+#include "../../include/sdv.h"
+
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "forward.cuh"
+#include "layout.cuh"
+#include "small_kernels.cuh"
+
+using namespace sdv;
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Regions {
+    size_t state, bar, never, hist, rope, norm_w, bias, wlayers, wlm, emb, kcache, vcache, h, qkv_acc, sumsq, act,
+        part_o, part_ml, cand_val, cand_idx, logits, raw_out, staging, wraw, xstage, total;
+    size_t layer_stride, staging_bytes, act_k;
+};
+
+constexpr int kMaxGrid = 256;  // per-block candidate arrays are sized for this many blocks
+
+bool config_ok(const sdv_config* c) {
+    if (!c) return false;
+    if (c->n_layers < 1 || c->d_model < 64 || c->d_model % 64 || c->d_ffn < 64 || c->d_ffn % 64) return false;
+    if (c->vocab < 16 || c->vocab % 16) return false;
+    if (c->head_dim != 64 && c->head_dim != 128) return false;
+    if (c->n_kv_heads < 1 || c->n_q_heads < 1 || c->n_q_heads % c->n_kv_heads) return false;
+    const int g = c->n_q_heads / c->n_kv_heads;
+    if (g > 8) return false;
+    if (c->k_max < 1 || c->k_max > SDV_K_MAX) return false;
+    if (g * (c->k_max + 1) > 128) return false;  // query tile of the attention step
+    if (c->max_seq < c->k_max + 2) return false;
+    if (c->ngram_n < 1 || c->ngram_n > 8 || c->ngram_min < 1 || c->ngram_min > c->ngram_n) return false;
+    if (!(c->rope_theta > 0.f) || !(c->rms_eps > 0.f)) return false;
+    return true;
+}
+
+Regions carve(const sdv_config* c) {
+    Regions r;
+    memset(&r, 0, sizeof(r));
+    const size_t d = c->d_model, f = c->d_ffn, V = c->vocab, hd = c->head_dim;
+    const size_t nq = (size_t)c->n_q_heads * hd, nkv = (size_t)c->n_kv_heads * hd, nqkv = nq + 2 * nkv;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t o = off;
+        off = align_up(off + bytes, 256);
+        return o;
+    };
+    r.state = take(ST_WORDS * 4);
+    r.bar = take(256);
+    r.never = take(256);
+    r.hist = take(((size_t)c->max_seq + 64) * 4);
+    r.rope = take((size_t)c->max_seq * (hd / 2) * sizeof(float2));
+    r.norm_w = take(((size_t)c->n_layers * 2 + 1) * d * 4);
+    r.bias = take((size_t)c->n_layers * nqkv * 4);
+    r.layer_stride = (nqkv * d + d * nq + 2 * f * d + d * f) * 2;
+    r.wlayers = take(r.layer_stride * c->n_layers);
+    r.wlm = take(V * d * 2);
+    r.emb = take(V * d * 2);
+    const size_t kvb = (size_t)c->n_layers * c->n_kv_heads * c->max_seq * hd * 2;
+    r.kcache = take(kvb);
+    r.vcache = take(kvb);
+    r.h = take((size_t)kMaxRows * d * 4);
+    r.qkv_acc = take((size_t)kMaxRows * nqkv * 4);
+    r.sumsq = take(2 * kMaxRows * 4);
+    size_t act_k = f;  // the stand-alone GEMM stages operands of any K up to max(f, d, nq)
+    if (d > act_k) act_k = d;
+    if (nq > act_k) act_k = nq;
+    r.act_k = act_k;
+    r.act = take(act_k / 64 * kMaxRows * 128);
+    r.part_o = take((size_t)c->n_q_heads * (kMaxSplits + 1) * kMaxRows * hd * 4);
+    r.part_ml = take((size_t)c->n_q_heads * (kMaxSplits + 1) * kMaxRows * 2 * 4);
+    r.cand_val = take((size_t)kMaxGrid * kMaxRows * 4);
+    r.cand_idx = take((size_t)kMaxGrid * kMaxRows * 4);
+    r.logits = take((size_t)kMaxRows * V * 4);
+    size_t st = 2 * f * d * 2;  // gate | up of one layer, the largest per-layer group
+    if (nqkv * d * 2 > st) st = nqkv * d * 2;
+    if (d * nq * 2 > st) st = d * nq * 2;
+    if (st < ((size_t)64 << 20)) st = (size_t)64 << 20;
+    r.staging_bytes = st;
+    r.staging = take(st);
+    r.wraw = take(st);
+    r.raw_out = take((size_t)kMaxRows * (st / 128) * 4);  // N <= staging / (2 bytes * 64 columns)
+    r.xstage = take((size_t)kMaxRows * act_k * 4);
+    r.total = off;
+    return r;
+}
+
+// Chooses how an operation's tile grid is cut among the blocks: minimise the largest per-block
+// share, then the number of sequential pipeline stages, then the number of column partitions.
+void choose_partition(OpDesc& o, int G, bool full_k) {
+    long long best_cost = -1;
+    int best_stages = 0, bp_row = 1, bp_k = 1;
+    for (int pr = 1; pr <= o.T && pr <= G; ++pr) {
+        const int pk_max = full_k ? 1 : (G / pr < o.C ? G / pr : o.C);
+        for (int pk = 1; pk <= pk_max; ++pk) {
+            const int tiles = (o.T + pr - 1) / pr, chunks = (o.C + pk - 1) / pk;
+            const int passes = (tiles + kConsumerWarps - 1) / kConsumerWarps;
+            const long long cost = (long long)tiles * chunks;
+            const int stages = passes * chunks;
+            if (best_cost < 0 || cost < best_cost || (cost == best_cost && stages < best_stages) ||
+                (cost == best_cost && stages == best_stages && pk < bp_k)) {
+                best_cost = cost;
+                best_stages = stages;
+                bp_row = pr;
+                bp_k = pk;
+            }
+        }
+    }
+    o.P_row = bp_row;
+    o.P_k = bp_k;
+}
+
+}  // namespace
+
+struct sdv_ctx {
+    sdv_config cfg;
+    uint8_t* ws;
+    size_t ws_bytes;
+    Regions r;
+    cudaStream_t stream;
+    int G;
+    FwdParams P;  // template; per-launch fields are filled at launch
+    int* pinned;  // host staging for the state block
+    cudaEvent_t ev0, ev1;
+    // host mirror of the device state
+    int kv_len, hist_len, n_ctx;
+    bool prefill_done, weights_loaded, verified, draft_pending;
+    int draft_k;    // k of the pending sdv_draft
+    int last_rows;  // rows of the last verify
+    int bar_base;
+    int parity;
+    int last_cuda;
+    long long launches;
+    bool have_verify_time;
+    bool poisoned;
+};
+
+namespace {
+
+int cuda_fail(sdv_ctx* ctx, cudaError_t e) {
+    if (ctx) ctx->last_cuda = (int)e;
+    return SDV_ECUDA;
+}
+#define CK(call)                                          \
+    do {                                                  \
+        cudaError_t e_ = (call);                          \
+        if (e_ != cudaSuccess) return cuda_fail(ctx, e_); \
+    } while (0)
+
+template <int NT>
+cudaError_t launch_forward_nt(sdv_ctx* ctx, const FwdParams& P) {
+    using SL = SmemLayout<NT>;
+    cudaError_t e = cudaFuncSetAttribute(sdv_forward_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::TOTAL);
+    if (e != cudaSuccess) return e;
+    void* args[] = {(void*)&P};
+    // phases meet at grid barriers, so more than one phase needs all blocks co-resident
+    if (P.ph_end - P.ph_begin > 1)
+        return cudaLaunchCooperativeKernel((const void*)sdv_forward_kernel<NT>, dim3(P.G), dim3(kThreads), args, SL::TOTAL,
+                                           ctx->stream);
+    return cudaLaunchKernel((const void*)sdv_forward_kernel<NT>, dim3(P.G), dim3(kThreads), args, SL::TOTAL, ctx->stream);
+}
+
+// Runs phases [ph_begin, ph_end) over `rows` token rows at position L.
+int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph_end, bool timed) {
+    FwdParams P = ctx->P;
+    P.L = L;
+    P.M = rows;
+    P.mode = mode;
+    P.ph_begin = ph_begin;
+    P.ph_end = ph_end;
+    P.bar_base = ctx->bar_base;
+    P.store_logits = ctx->parity;
+    const int nbar = ph_end - ph_begin - 1;
+    ctx->bar_base += nbar * ctx->G;
+    const int NT = (rows + 7) / 8;
+    if (timed) CK(cudaEventRecord(ctx->ev0, ctx->stream));
+    cudaError_t e;
+    switch (NT) {
+        case 1: e = launch_forward_nt<1>(ctx, P); break;
+        case 2: e = launch_forward_nt<2>(ctx, P); break;
+        case 3: e = launch_forward_nt<3>(ctx, P); break;
+        case 4: e = launch_forward_nt<4>(ctx, P); break;
+        default: return SDV_EINVAL;
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches++;
+    if (timed) {
+        CK(cudaEventRecord(ctx->ev1, ctx->stream));
+        ctx->have_verify_time = true;
+    }
+    return SDV_OK;
+}
+
+int read_state(sdv_ctx* ctx) {
+    CK(cudaMemcpyAsync(ctx->pinned, ctx->ws + ctx->r.state, ST_WORDS * 4, cudaMemcpyDeviceToHost, ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
+    if (ctx->pinned[ST_ERR] == 1) {
+        ctx->poisoned = true;
+        return SDV_ETIMEOUT;
+    }
+    return SDV_OK;
+}
+
+int pack_op(sdv_ctx* ctx, const OpDesc& o, uint8_t* dst_base, const uint16_t* s0, int rows0, const uint16_t* s1,
+            int rows1, const uint16_t* s2, int K, int mode, int t_begin, int t_end, int row_base) {
+    const long long total = (long long)(t_end - t_begin) * o.C * 128;
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    pack_weights_kernel<<<blocks, 256, 0, ctx->stream>>>(o, dst_base, s0, rows0, s1, rows1, s2, K, mode, t_begin, t_end,
+                                                       row_base);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    return SDV_OK;
+}
+
+void fill_draft_arg(DraftArg& a, const int32_t* tok, int n) {
+    memset(&a, 0, sizeof(a));
+    a.n = n;
+    for (int i = 0; i < n; ++i) a.tok[i] = tok[i];
+}
+
+int commit_common(sdv_ctx* ctx, int max_emit, int force_accept, int force_token, int32_t* host_emitted, int* n_emitted,
+                  int* kv_len) {
+    int* hist = (int*)(ctx->ws + ctx->r.hist);
+    commit_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, hist, max_emit, force_accept, force_token);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    int rc = read_state(ctx);
+    if (rc) return rc;
+    const int n = ctx->pinned[ST_N_EMITTED];
+    ctx->kv_len = ctx->pinned[ST_KV_LEN];
+    ctx->hist_len = ctx->pinned[ST_HIST_LEN];
+    ctx->verified = false;
+    ctx->draft_pending = false;
+    if (n_emitted) *n_emitted = n;
+    if (kv_len) *kv_len = ctx->kv_len;
+    if (host_emitted)
+        for (int i = 0; i < n; ++i) host_emitted[i] = ctx->pinned[ST_EMITTED + i];
+    return SDV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sdv_strerror(int code) {
+    switch (code) {
+        case SDV_OK: return "ok";
+        case SDV_EINVAL: return "invalid argument or unsupported shape";
+        case SDV_ENOMEM: return "workspace too small";
+        case SDV_ECAPACITY: return "KV cache or history capacity exceeded";
+        case SDV_ESTATE: return "call not valid in the current state";
+        case SDV_ECUDA: return "CUDA runtime error";
+        case SDV_ETIMEOUT: return "a bounded device-side wait ran out";
+        default: return "unknown error";
+    }
+}
+
+size_t sdv_workspace_bytes(const sdv_config* cfg) {
+    if (!config_ok(cfg)) return 0;
+    return carve(cfg).total;
+}
+
+int sdv_last_cuda_error(const sdv_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+long long sdv_launch_count(const sdv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+int sdv_kv_len(const sdv_ctx* ctx) { return ctx ? ctx->kv_len : SDV_EINVAL; }
+
+int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* cuda_stream, sdv_ctx** out) {
+    if (!out) return SDV_EINVAL;
+    *out = nullptr;
+    if (!config_ok(cfg) || !dev_workspace || ((uintptr_t)dev_workspace & 255)) return SDV_EINVAL;
+    if (bytes < sdv_workspace_bytes(cfg)) return SDV_ENOMEM;
+    sdv_ctx* ctx = new (std::nothrow) sdv_ctx();
+    if (!ctx) return SDV_ENOMEM;
+    memset(ctx, 0, sizeof(*ctx));
+    ctx->cfg = *cfg;
+    ctx->ws = (uint8_t*)dev_workspace;
+    ctx->ws_bytes = bytes;
+    ctx->stream = (cudaStream_t)cuda_stream;
+    int sms = 0, dev = 0, coop = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    if (e != cudaSuccess || sms <= 0 || !coop) {
+        delete ctx;
+        return SDV_ECUDA;
+    }
+    if (sms > kMaxGrid) sms = kMaxGrid;
+    ctx->G = sms;  // one persistent block per SM
+    ctx->r = carve(cfg);
+    e = cudaHostAlloc((void**)&ctx->pinned, 4096, cudaHostAllocDefault);
+    if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev0);
+    if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev1);
+    if (e != cudaSuccess) {
+        delete ctx;
+        return SDV_ECUDA;
+    }
+
+    const int d = cfg->d_model, f = cfg->d_ffn, hd = cfg->head_dim;
+    const int nq = cfg->n_q_heads * hd, nkv = cfg->n_kv_heads * hd, nqkv = nq + 2 * nkv;
+    FwdParams& P = ctx->P;
+    P.n_layers = cfg->n_layers; P.d = d; P.n_q = cfg->n_q_heads; P.n_kv = cfg->n_kv_heads; P.hd = hd; P.f = f;
+    P.V = cfg->vocab; P.max_seq = cfg->max_seq; P.g = cfg->n_q_heads / cfg->n_kv_heads; P.n_qkv = nqkv;
+    P.eps = cfg->rms_eps;
+    P.scale_log2e = (float)((1.0 / sqrt((double)hd)) * 1.4426950408889634);
+    P.G = ctx->G;
+    // operations of one layer, in streaming order, and the LM head
+    struct { int idx, N, K; bool full_k; } ops[5] = {
+        {OP_QKV, nqkv, d, false}, {OP_O, d, nq, false}, {OP_GU, 2 * f, d, true}, {OP_DOWN, d, f, false},
+        {OP_LM, cfg->vocab, d, true}};
+    unsigned long long woff = 0;
+    int rot = 0;
+    for (int i = 0; i < 5; ++i) {
+        OpDesc& o = P.op[ops[i].idx];
+        o.T = ops[i].N / 16;
+        o.C = ops[i].K / 64;
+        choose_partition(o, ctx->G, ops[i].full_k);
+        o.rot = rot % ctx->G;
+        rot += o.P_row * o.P_k;
+        o.w_off = (ops[i].idx == OP_LM) ? 0 : woff;
+        if (ops[i].idx != OP_LM) woff += (unsigned long long)ops[i].N * ops[i].K * 2;
+    }
+    P.layer_stride = ctx->r.layer_stride;
+    uint8_t* ws = ctx->ws;
+    P.wlayers = ws + ctx->r.wlayers;
+    P.wlm = ws + ctx->r.wlm;
+    P.wraw = ws + ctx->r.wraw;
+    P.emb = (const __nv_bfloat16*)(ws + ctx->r.emb);
+    P.norm_w = (const float*)(ws + ctx->r.norm_w);
+    P.bias = cfg->qkv_bias ? (const float*)(ws + ctx->r.bias) : nullptr;
+    P.rope = (const float2*)(ws + ctx->r.rope);
+    P.kcache = (__nv_bfloat16*)(ws + ctx->r.kcache);
+    P.vcache = (__nv_bfloat16*)(ws + ctx->r.vcache);
+    P.h = (float*)(ws + ctx->r.h);
+    P.qkv_acc = (float*)(ws + ctx->r.qkv_acc);
+    P.sumsq = (float*)(ws + ctx->r.sumsq);
+    P.act = ws + ctx->r.act;
+    P.part_o = (float*)(ws + ctx->r.part_o);
+    P.part_ml = (float*)(ws + ctx->r.part_ml);
+    P.cand_val = (float*)(ws + ctx->r.cand_val);
+    P.cand_idx = (int*)(ws + ctx->r.cand_idx);
+    P.logits = (float*)(ws + ctx->r.logits);
+    P.raw_out = (float*)(ws + ctx->r.raw_out);
+    P.raw_N = 0;
+    P.state = (int*)(ws + ctx->r.state);
+    P.hist = (const int*)(ws + ctx->r.hist);
+    P.bar = (int*)(ws + ctx->r.bar);
+    P.wait_limit_ns = 2000000000ull;
+
+    // rotary table in double, rounded once to fp32
+    {
+        const size_t n = (size_t)cfg->max_seq * (hd / 2);
+        std::vector<float2> tab(n);
+        for (int i = 0; i < hd / 2; ++i) {
+            const double inv = pow((double)cfg->rope_theta, -2.0 * (double)i / (double)hd);
+            for (int p = 0; p < cfg->max_seq; ++p) {
+                const double a = (double)p * inv;
+                tab[(size_t)p * (hd / 2) + i] = make_float2((float)cos(a), (float)sin(a));
+            }
+        }
+        e = cudaMemcpyAsync(ws + ctx->r.rope, tab.data(), n * sizeof(float2), cudaMemcpyHostToDevice, ctx->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+    }
+    if (e == cudaSuccess) e = cudaMemsetAsync(ws + ctx->r.state, 0, ST_WORDS * 4, ctx->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ws + ctx->r.bar, 0, 256, ctx->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ws + ctx->r.never, 0, 256, ctx->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ws + ctx->r.hist, 0, ((size_t)cfg->max_seq + 64) * 4, ctx->stream);
+    // activations: h .. part_ml are contiguous regions
+    if (e == cudaSuccess) e = cudaMemsetAsync(ws + ctx->r.h, 0, ctx->r.cand_val - ctx->r.h, ctx->stream);
+    if (e == cudaSuccess) {
+        fill_f32_kernel<<<8, 256, 0, ctx->stream>>>(P.cand_val, -INFINITY, (long long)kMaxGrid * kMaxRows);
+        fill_i32_kernel<<<8, 256, 0, ctx->stream>>>(P.cand_idx, 0x7fffffff, (long long)kMaxGrid * kMaxRows);
+        ctx->launches += 2;
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+    if (e != cudaSuccess) {
+        cudaFreeHost(ctx->pinned);
+        delete ctx;
+        return SDV_ECUDA;
+    }
+    *out = ctx;
+    return SDV_OK;
+}
+
+int sdv_destroy(sdv_ctx* ctx) {
+    if (!ctx) return SDV_EINVAL;
+    cudaStreamSynchronize(ctx->stream);
+    if (ctx->pinned) cudaFreeHost(ctx->pinned);
+    cudaEventDestroy(ctx->ev0);
+    cudaEventDestroy(ctx->ev1);
+    delete ctx;
+    return SDV_OK;
+}
+
+int sdv_load_weights(sdv_ctx* ctx, const sdv_weights* w) {
+    if (!ctx || !w || !w->emb || !w->final_norm || !w->layers) return SDV_EINVAL;
+    const sdv_config& c = ctx->cfg;
+    if (!c.tied_lm_head && !w->lm_head) return SDV_EINVAL;
+    const size_t d = c.d_model, f = c.d_ffn, hd = c.head_dim, V = c.vocab;
+    const size_t nq = c.n_q_heads * hd, nkv = c.n_kv_heads * hd, nqkv = nq + 2 * nkv;
+    uint8_t* ws = ctx->ws;
+    uint16_t* stg = (uint16_t*)(ws + ctx->r.staging);
+    float* norm_w = (float*)(ws + ctx->r.norm_w);
+    float* bias = (float*)(ws + ctx->r.bias);
+    cudaStream_t s = ctx->stream;
+    for (int l = 0; l < c.n_layers; ++l) {
+        const sdv_layer_weights& L = w->layers[l];
+        if (!L.wq || !L.wk || !L.wv || !L.wo || !L.wg || !L.wu || !L.wd || !L.norm1 || !L.norm2) return SDV_EINVAL;
+        if (c.qkv_bias && (!L.bq || !L.bk || !L.bv)) return SDV_EINVAL;
+        uint8_t* lbase = ws + ctx->r.wlayers + (size_t)l * ctx->r.layer_stride;
+        int rc;
+        // q | k | v stacked
+        CK(cudaMemcpyAsync(stg, L.wq, nq * d * 2, cudaMemcpyDefault, s));
+        CK(cudaMemcpyAsync(stg + nq * d, L.wk, nkv * d * 2, cudaMemcpyDefault, s));
+        CK(cudaMemcpyAsync(stg + (nq + nkv) * d, L.wv, nkv * d * 2, cudaMemcpyDefault, s));
+        rc = pack_op(ctx, ctx->P.op[OP_QKV], lbase + ctx->P.op[OP_QKV].w_off, stg, (int)nq, stg + nq * d, (int)nkv,
+                     stg + (nq + nkv) * d, (int)d, 0, 0, ctx->P.op[OP_QKV].T, 0);
+        if (rc) return rc;
+        CK(cudaStreamSynchronize(s));
+        // o
+        CK(cudaMemcpyAsync(stg, L.wo, d * nq * 2, cudaMemcpyDefault, s));
+        rc = pack_op(ctx, ctx->P.op[OP_O], lbase + ctx->P.op[OP_O].w_off, stg, (int)d, nullptr, 0, nullptr, (int)nq, 0, 0,
+                     ctx->P.op[OP_O].T, 0);
+        if (rc) return rc;
+        CK(cudaStreamSynchronize(s));
+        // gate | up, interleaved 8 + 8 rows per tile
+        CK(cudaMemcpyAsync(stg, L.wg, f * d * 2, cudaMemcpyDefault, s));
+        CK(cudaMemcpyAsync(stg + f * d, L.wu, f * d * 2, cudaMemcpyDefault, s));
+        rc = pack_op(ctx, ctx->P.op[OP_GU], lbase + ctx->P.op[OP_GU].w_off, stg, (int)f, stg + f * d, (int)f, nullptr,
+                     (int)d, 1, 0, ctx->P.op[OP_GU].T, 0);
+        if (rc) return rc;
+        CK(cudaStreamSynchronize(s));
+        // down
+        CK(cudaMemcpyAsync(stg, L.wd, d * f * 2, cudaMemcpyDefault, s));
+        rc = pack_op(ctx, ctx->P.op[OP_DOWN], lbase + ctx->P.op[OP_DOWN].w_off, stg, (int)d, nullptr, 0, nullptr, (int)f,
+                     0, 0, ctx->P.op[OP_DOWN].T, 0);
+        if (rc) return rc;
+        CK(cudaStreamSynchronize(s));
+        CK(cudaMemcpyAsync(norm_w + ((size_t)l * 2 + 0) * d, L.norm1, d * 4, cudaMemcpyDefault, s));
+        CK(cudaMemcpyAsync(norm_w + ((size_t)l * 2 + 1) * d, L.norm2, d * 4, cudaMemcpyDefault, s));
+        if (c.qkv_bias) {
+            CK(cudaMemcpyAsync(bias + (size_t)l * nqkv, L.bq, nq * 4, cudaMemcpyDefault, s));
+            CK(cudaMemcpyAsync(bias + (size_t)l * nqkv + nq, L.bk, nkv * 4, cudaMemcpyDefault, s));
+            CK(cudaMemcpyAsync(bias + (size_t)l * nqkv + nq + nkv, L.bv, nkv * 4, cudaMemcpyDefault, s));
+        }
+    }
+    CK(cudaMemcpyAsync(norm_w + (size_t)c.n_layers * 2 * d, w->final_norm, d * 4, cudaMemcpyDefault, s));
+    CK(cudaMemcpyAsync(ws + ctx->r.emb, w->emb, V * d * 2, cudaMemcpyDefault, s));
+    // LM head: packed from row blocks that fit the staging area
+    {
+        const uint16_t* src = c.tied_lm_head ? w->emb : w->lm_head;
+        const OpDesc& o = ctx->P.op[OP_LM];
+        const size_t tiles_per = ctx->r.staging_bytes / (16 * d * 2);
+        if (tiles_per < 1) return SDV_ENOMEM;
+        for (size_t t0 = 0; t0 < (size_t)o.T; t0 += tiles_per) {
+            const size_t t1 = (t0 + tiles_per < (size_t)o.T) ? t0 + tiles_per : (size_t)o.T;
+            const size_t rows = (t1 - t0) * 16;
+            CK(cudaMemcpyAsync(stg, src + t0 * 16 * d, rows * d * 2, cudaMemcpyDefault, s));
+            int rc = pack_op(ctx, o, ws + ctx->r.wlm, stg, (int)rows, nullptr, 0, nullptr, (int)d, 0, (int)t0, (int)t1,
+                             (int)(t0 * 16));
+            if (rc) return rc;
+            CK(cudaStreamSynchronize(s));
+        }
+    }
+    CK(cudaStreamSynchronize(s));
+    ctx->weights_loaded = true;
+    return SDV_OK;
+}
+
+int sdv_set_parity_mode(sdv_ctx* ctx, int on) {
+    if (!ctx) return SDV_EINVAL;
+    ctx->parity = on ? 1 : 0;
+    return SDV_OK;
+}
+
+int sdv_prefill_chunk(sdv_ctx* ctx, const int32_t* host_tokens, int n, int is_last) {
+    if (!ctx || !host_tokens || n < 1) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->weights_loaded || ctx->prefill_done) return SDV_ESTATE;
+    const sdv_config& c = ctx->cfg;
+    if (ctx->kv_len + n + 1 + c.k_max + 1 > c.max_seq) return SDV_ECAPACITY;
+    for (int i = 0; i < n; ++i)
+        if (host_tokens[i] < 0 || host_tokens[i] >= c.vocab) return SDV_EINVAL;
+    int* hist = (int*)(ctx->ws + ctx->r.hist);
+    CK(cudaMemcpyAsync(hist + ctx->hist_len, host_tokens, (size_t)n * 4, cudaMemcpyDefault, ctx->stream));
+    // rows per launch: the attention step's query tile holds (q heads per kv head) x rows <= 128
+    const int g = c.n_q_heads / c.n_kv_heads;
+    int tile = 128 / g;
+    if (tile > 24) tile = 24;
+    tile = tile / 8 * 8;
+    if (tile < 8) tile = 8;
+    const int n_ph = 1 + 5 * c.n_layers;
+    int done = 0;
+    while (done < n) {
+        const int rows = (n - done < tile) ? n - done : tile;
+        const bool last_tile = is_last && (done + rows == n);
+        int rc = launch_forward(ctx, rows, ctx->kv_len, 1, 0, last_tile ? n_ph + 1 : n_ph, false);
+        if (rc) return rc;
+        ctx->kv_len += rows;
+        ctx->hist_len += rows;
+        done += rows;
+        if (done == n) {
+            // the context now covers everything prefilled so far
+            ctx->n_ctx = ctx->hist_len;
+            set_state_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, ctx->kv_len, ctx->hist_len, ctx->n_ctx, 0, hist);
+            ctx->launches++;
+            CK(cudaGetLastError());
+            if (last_tile) {
+                // greedy token of the last context row: appended to the history as the pending token T
+                prefill_final_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, hist, ctx->P.cand_val, ctx->P.cand_idx,
+                                                              ctx->G, rows - 1);
+                ctx->launches++;
+                CK(cudaGetLastError());
+                ctx->hist_len += 1;
+                ctx->prefill_done = true;
+            }
+        }
+    }
+    return read_state(ctx);
+}
+
+int sdv_draft(sdv_ctx* ctx, int k, int32_t* host_draft, int* draft_len) {
+    if (!ctx || k < 1 || k > ctx->cfg.k_max) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->prefill_done) return SDV_ESTATE;
+    int* hist = (int*)(ctx->ws + ctx->r.hist);
+    ngram_draft_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->P.state, hist, ctx->cfg.ngram_n, ctx->cfg.ngram_min, k,
+                                                    ctx->cfg.search_history);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    ctx->draft_pending = true;
+    ctx->draft_k = k;
+    ctx->verified = false;
+    if (host_draft || draft_len) {
+        int rc = read_state(ctx);
+        if (rc) return rc;
+        const int dl = ctx->pinned[ST_DRAFT_LEN];
+        if (draft_len) *draft_len = dl;
+        if (host_draft)
+            for (int i = 0; i < dl; ++i) host_draft[i] = ctx->pinned[ST_DRAFT + i];
+    }
+    return SDV_OK;
+}
+
+int sdv_verify(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, int32_t* host_y, int* accept_len) {
+    if (!ctx) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->prefill_done || !ctx->weights_loaded) return SDV_ESTATE;
+    const sdv_config& c = ctx->cfg;
+    int rows;
+    if (host_draft) {
+        if (draft_len < 0 || draft_len > c.k_max) return SDV_EINVAL;
+        for (int i = 0; i < draft_len; ++i)
+            if (host_draft[i] < 0 || host_draft[i] >= c.vocab) return SDV_EINVAL;
+        rows = draft_len + 1;
+    } else {
+        rows = ctx->draft_pending ? ctx->draft_k + 1 : 1;
+    }
+    if (ctx->kv_len + rows > c.max_seq) return SDV_ECAPACITY;
+    if (host_draft) {
+        DraftArg a;
+        fill_draft_arg(a, host_draft, draft_len);
+        set_draft_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, a);
+        ctx->launches++;
+        CK(cudaGetLastError());
+    }
+    int rc = launch_forward(ctx, rows, ctx->kv_len, 0, 0, 2 + 5 * c.n_layers, true);
+    if (rc) return rc;
+    accept_kernel<<<1, 32 * rows, 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    ctx->verified = true;
+    ctx->last_rows = rows;
+    if (host_y || accept_len) {
+        rc = read_state(ctx);
+        if (rc) return rc;
+        const int dl = ctx->pinned[ST_DRAFT_LEN];
+        if (accept_len) *accept_len = ctx->pinned[ST_ACCEPT_LEN];
+        if (host_y)
+            for (int i = 0; i <= dl; ++i) host_y[i] = ctx->pinned[ST_Y + i];
+    }
+    return SDV_OK;
+}
+
+int sdv_commit(sdv_ctx* ctx, int max_emit, int32_t* host_emitted, int* n_emitted, int* kv_len) {
+    if (!ctx) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->verified) return SDV_ESTATE;
+    return commit_common(ctx, max_emit, -1, 0, host_emitted, n_emitted, kv_len);
+}
+
+int sdv_debug_force_commit(sdv_ctx* ctx, int accept_len, int32_t next_token) {
+    if (!ctx) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->verified) return SDV_ESTATE;
+    if (accept_len < 0 || accept_len + 1 > ctx->last_rows || next_token < 0 || next_token >= ctx->cfg.vocab)
+        return SDV_EINVAL;
+    return commit_common(ctx, 0, accept_len, next_token, nullptr, nullptr, nullptr);
+}
+
+int sdv_rollback(sdv_ctx* ctx, int new_kv_len) {
+    if (!ctx) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->prefill_done) return SDV_ESTATE;
+    if (new_kv_len < 1 || new_kv_len > ctx->kv_len) return SDV_EINVAL;
+    int* hist = (int*)(ctx->ws + ctx->r.hist);
+    ctx->kv_len = new_kv_len;
+    ctx->hist_len = new_kv_len + 1;
+    set_state_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, ctx->kv_len, ctx->hist_len, ctx->n_ctx, 1, hist);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    ctx->verified = false;
+    ctx->draft_pending = false;
+    CK(cudaStreamSynchronize(ctx->stream));
+    return SDV_OK;
+}
+
+int sdv_get_logits(sdv_ctx* ctx, float* host_logits, int rows) {
+    if (!ctx || !host_logits || rows < 1 || rows > kMaxRows) return SDV_EINVAL;
+    if (!ctx->parity) return SDV_ESTATE;
+    CK(cudaMemcpyAsync(host_logits, ctx->ws + ctx->r.logits, (size_t)rows * ctx->cfg.vocab * 4, cudaMemcpyDeviceToHost,
+                       ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
+    return SDV_OK;
+}
+
+int sdv_step_bytes(const sdv_ctx* ctx, int rows, int kv_len, double* weight_bytes, double* kv_bytes) {
+    if (!ctx || rows < 1) return SDV_EINVAL;
+    const sdv_config& c = ctx->cfg;
+    const double hd = c.head_dim, nq = c.n_q_heads * hd, nkv = c.n_kv_heads * hd, d = c.d_model, f = c.d_ffn;
+    const double per_layer = (nq + 2 * nkv) * d + d * nq + 3 * d * f;
+    if (weight_bytes) *weight_bytes = 2.0 * (c.n_layers * per_layer + (double)c.vocab * d);
+    if (kv_bytes) *kv_bytes = (double)c.n_layers * 2.0 * nkv * 2.0 * ((double)kv_len + rows);
+    return SDV_OK;
+}
+
+int sdv_last_verify_ms(sdv_ctx* ctx, float* ms) {
+    if (!ctx || !ms) return SDV_EINVAL;
+    if (!ctx->have_verify_time) return SDV_ESTATE;
+    CK(cudaEventSynchronize(ctx->ev1));
+    CK(cudaEventElapsedTime(ms, ctx->ev0, ctx->ev1));
+    return SDV_OK;
+}
+
+// ------------------------------------------------------------------------------------------ debug
+int sdv_debug_set_history(sdv_ctx* ctx, const int32_t* host_hist, int hist_len, int n_ctx) {
+    if (!ctx || !host_hist || hist_len < 1 || n_ctx < 0 || n_ctx > hist_len) return SDV_EINVAL;
+    if (hist_len > ctx->cfg.max_seq) return SDV_ECAPACITY;
+    int* hist = (int*)(ctx->ws + ctx->r.hist);
+    CK(cudaMemcpyAsync(hist, host_hist, (size_t)hist_len * 4, cudaMemcpyDefault, ctx->stream));
+    ctx->hist_len = hist_len;
+    ctx->kv_len = hist_len - 1;
+    ctx->n_ctx = n_ctx;
+    set_state_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, ctx->kv_len, ctx->hist_len, ctx->n_ctx, 1, hist);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    ctx->prefill_done = true;
+    ctx->verified = false;
+    ctx->draft_pending = false;
+    CK(cudaStreamSynchronize(ctx->stream));
+    return SDV_OK;
+}
+
+int sdv_debug_accept(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, const int32_t* host_y, int* accept_len) {
+    if (!ctx || !host_y || draft_len < 0 || draft_len > ctx->cfg.k_max || (draft_len && !host_draft)) return SDV_EINVAL;
+    DraftArg a, y;
+    fill_draft_arg(a, host_draft, draft_len);
+    fill_draft_arg(y, host_y, draft_len + 1);
+    set_draft_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, a);
+    set_y_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, y);
+    accept_kernel<<<1, 32 * (draft_len + 1), 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 1);
+    ctx->launches += 3;
+    CK(cudaGetLastError());
+    ctx->verified = true;
+    ctx->last_rows = draft_len + 1;
+    int rc = read_state(ctx);
+    if (rc) return rc;
+    if (accept_len) *accept_len = ctx->pinned[ST_ACCEPT_LEN];
+    return SDV_OK;
+}
+
+int sdv_debug_read_kv(sdv_ctx* ctx, int layer, int which, int pos0, int n, float* host_out) {
+    if (!ctx || !host_out || layer < 0 || layer >= ctx->cfg.n_layers || pos0 < 0 || n < 1 ||
+        pos0 + n > ctx->cfg.max_seq)
+        return SDV_EINVAL;
+    const sdv_config& c = ctx->cfg;
+    const size_t hd = c.head_dim;
+    std::vector<uint16_t> tmp((size_t)n * hd);
+    const uint8_t* base = ctx->ws + (which ? ctx->r.vcache : ctx->r.kcache);
+    for (int a = 0; a < c.n_kv_heads; ++a) {
+        const size_t off = (((size_t)layer * c.n_kv_heads + a) * c.max_seq + pos0) * hd * 2;
+        CK(cudaMemcpyAsync(tmp.data(), base + off, tmp.size() * 2, cudaMemcpyDeviceToHost, ctx->stream));
+        CK(cudaStreamSynchronize(ctx->stream));
+        for (size_t i = 0; i < tmp.size(); ++i) {
+            const uint32_t u = (uint32_t)tmp[i] << 16;
+            memcpy(&host_out[(size_t)a * n * hd + i], &u, 4);
+        }
+    }
+    return SDV_OK;
+}
+
+int sdv_debug_read_hidden(sdv_ctx* ctx, int rows, float* host_out) {
+    if (!ctx || !host_out || rows < 1 || rows > kMaxRows) return SDV_EINVAL;
+    CK(cudaMemcpyAsync(host_out, ctx->ws + ctx->r.h, (size_t)rows * ctx->cfg.d_model * 4, cudaMemcpyDeviceToHost,
+                       ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
+    return SDV_OK;
+}
+
+int sdv_debug_gemm(sdv_ctx* ctx, const float* host_x, const uint16_t* host_w, float* host_y, int M, int N, int K,
+                   float* dev_ms) {
+    if (!ctx || !host_x || !host_w || !host_y) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (M < 1 || M > kMaxRows || N < 16 || N % 16 || K < 64 || K % 64) return SDV_EINVAL;
+    if ((size_t)K > ctx->r.act_k || (size_t)N * K * 2 > ctx->r.staging_bytes || (size_t)N > ctx->r.staging_bytes / 128)
+        return SDV_EINVAL;
+    const sdv_config& c = ctx->cfg;
+    uint8_t* ws = ctx->ws;
+    cudaStream_t s = ctx->stream;
+    OpDesc o;
+    memset(&o, 0, sizeof(o));
+    o.T = N / 16;
+    o.C = K / 64;
+    choose_partition(o, ctx->G, false);
+    const int NT = (M + 7) / 8;
+    CK(cudaMemcpyAsync(ws + ctx->r.staging, host_w, (size_t)N * K * 2, cudaMemcpyDefault, s));
+    int rc = pack_op(ctx, o, ws + ctx->r.wraw, (const uint16_t*)(ws + ctx->r.staging), N, nullptr, 0, nullptr, K, 0, 0,
+                     o.T, 0);
+    if (rc) return rc;
+    CK(cudaMemcpyAsync(ws + ctx->r.xstage, host_x, (size_t)M * K * 4, cudaMemcpyDefault, s));
+    stage_operand_kernel<<<64, 256, 0, s>>>((const float*)(ws + ctx->r.xstage), ws + ctx->r.act, M, K, 8 * NT);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    CK(cudaMemsetAsync(ws + ctx->r.raw_out, 0, (size_t)kMaxRows * N * 4, s));
+    const OpDesc saved = ctx->P.op[OP_RAW];
+    const int saved_N = ctx->P.raw_N;
+    ctx->P.op[OP_RAW] = o;
+    ctx->P.raw_N = N;
+    const int ph = 2 + 5 * c.n_layers;
+    rc = launch_forward(ctx, M, 0, 1, ph, ph + 1, true);
+    ctx->P.op[OP_RAW] = saved;
+    ctx->P.raw_N = saved_N;
+    if (rc) return rc;
+    CK(cudaMemcpyAsync(host_y, ws + ctx->r.raw_out, (size_t)M * N * 4, cudaMemcpyDeviceToHost, s));
+    rc = read_state(ctx);
+    if (rc) return rc;
+    if (dev_ms) CK(cudaEventElapsedTime(dev_ms, ctx->ev0, ctx->ev1));
+    return SDV_OK;
+}
+
+int sdv_debug_timeout_probe(sdv_ctx* ctx) {
+    if (!ctx) return SDV_EINVAL;
+    timeout_probe_kernel<<<1, 1, 0, ctx->stream>>>(ctx->P.state, (const int*)(ctx->ws + ctx->r.never), 5000000ull);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    CK(cudaMemcpyAsync(ctx->pinned, ctx->ws + ctx->r.state, ST_WORDS * 4, cudaMemcpyDeviceToHost, ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
+    const int err = ctx->pinned[ST_ERR];
+    CK(cudaMemsetAsync(ctx->P.state + ST_ERR, 0, 4, ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
+    return err == 2 ? SDV_ETIMEOUT : SDV_OK;
+}
+
+}  // extern "C"

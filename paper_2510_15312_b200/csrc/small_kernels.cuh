@@ -1,0 +1,243 @@
+// The integer kernels of the path (n-gram drafter, accept scan, commit) and set-up helpers
+// (weight re-layout, operand staging for the stand-alone GEMM, fills).
+#pragma once
+#include <math_constants.h>
+
+#include "layout.cuh"
+#include "ptx.cuh"
+
+namespace sdv {
+
+// ------------------------------------------------------------------------------------------
+// Weight re-layout: row-major bf16 [rows][K] -> streaming tile order (see layout.cuh).
+// mode 0: the operation's rows are src0 | src1 | src2 stacked (the sources hold the rows from
+// row_base on); mode 1: every 16-row tile holds 8 rows of src0 (gate) followed by the 8 matching
+// rows of src1 (up).  Only tiles [t_begin, t_end) are written.
+__global__ void pack_weights_kernel(OpDesc o, uint8_t* dst_base, const uint16_t* src0, int rows0,
+                                    const uint16_t* src1, int rows1, const uint16_t* src2, int K, int mode,
+                                    int t_begin, int t_end, int row_base) {
+    const long long total = (long long)(t_end - t_begin) * o.C * 128;
+    for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < total;
+         u += (long long)gridDim.x * blockDim.x) {
+        const int q = (int)(u & 7), r = (int)((u >> 3) & 15);
+        const long long tc = u >> 7;
+        const int c = (int)(tc % o.C), t = t_begin + (int)(tc / o.C);
+        const uint16_t* src;
+        if (mode == 1) {
+            src = (r < 8) ? src0 + (size_t)(8 * t + r) * K : src1 + (size_t)(8 * t + r - 8) * K;
+        } else {
+            const int row = 16 * t + r - row_base;
+            if (row < rows0) src = src0 + (size_t)row * K;
+            else if (row < rows0 + rows1) src = src1 + (size_t)(row - rows0) * K;
+            else src = src2 + (size_t)(row - rows0 - rows1) * K;
+        }
+        const uint4 v = *reinterpret_cast<const uint4*>(src + c * 64 + q * 8);
+        *reinterpret_cast<uint4*>(dst_base + tile_offset(o, t, c) + swz_unit(r, q)) = v;
+    }
+}
+
+// fp32 [M][K] -> the bf16 chunked operand layout [K/64][rows][64] (swizzled), rows >= M zero.
+__global__ void stage_operand_kernel(const float* x, uint8_t* act, int M, int K, int rows) {
+    const int total = (K / 64) * rows * 8;
+    for (int u = blockIdx.x * blockDim.x + threadIdx.x; u < total; u += gridDim.x * blockDim.x) {
+        const int q = u & 7, tok = (u >> 3) % rows, c = (u >> 3) / rows;
+        uint4 out = make_uint4(0, 0, 0, 0);
+        if (tok < M) {
+            const float* p = x + (size_t)tok * K + c * 64 + q * 8;
+            out = make_uint4(pack_bf16(p[0], p[1]), pack_bf16(p[2], p[3]), pack_bf16(p[4], p[5]), pack_bf16(p[6], p[7]));
+        }
+        *reinterpret_cast<uint4*>(act + (size_t)c * rows * 128 + swz_unit(tok, q)) = out;
+    }
+}
+
+__global__ void fill_f32_kernel(float* p, float v, long long n) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        p[i] = v;
+}
+__global__ void fill_i32_kernel(int* p, int v, long long n) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        p[i] = v;
+}
+
+// ------------------------------------------------------------------------------------------
+// Retrieval drafter.  One block; thread p tests search position p: the length m(p) of the common
+// suffix of search[0..p] and the history (capped at n), then a block-wide maximum of (m(p), p)
+// picks the longest and, among those, the latest match; up to k following tokens are the draft.
+// The search array is the history's own prefix: the request context (first n_ctx tokens), or,
+// with search_history, everything but the last token (the suffix must not match itself).
+__global__ void ngram_draft_kernel(int* state, const int* hist, int n, int n_min, int k, int search_history) {
+    __shared__ unsigned long long best_s[32];
+    const int hist_len = state[ST_HIST_LEN];
+    const int n_search = search_history ? hist_len : state[ST_N_CTX];
+    const int exclude_from = search_history ? hist_len - 1 : n_search;
+    unsigned long long best = 0;
+    for (int p = threadIdx.x; p + 1 < n_search && p < exclude_from; p += blockDim.x) {
+        int cap = n;
+        if (p + 1 < cap) cap = p + 1;
+        if (hist_len < cap) cap = hist_len;
+        int mlen = 0;
+        while (mlen < cap && hist[p - mlen] == hist[hist_len - 1 - mlen]) ++mlen;
+        if (mlen >= n_min && mlen > 0) {
+            const unsigned long long key = ((unsigned long long)mlen << 32) | (unsigned)p;
+            if (key > best) best = key;
+        }
+    }
+    for (int off = 16; off; off >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, off);
+        if (o > best) best = o;
+    }
+    if ((threadIdx.x & 31) == 0) best_s[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        best = (threadIdx.x < (blockDim.x >> 5)) ? best_s[threadIdx.x] : 0ull;
+        for (int off = 16; off; off >>= 1) {
+            const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, off);
+            if (o > best) best = o;
+        }
+        int dl = 0, pos = -1, mlen = 0;
+        if (best != 0) {
+            pos = (int)(best & 0xffffffffu);
+            mlen = (int)(best >> 32);
+            dl = n_search - 1 - pos;
+            if (dl > k) dl = k;
+            if ((int)threadIdx.x < dl) state[ST_DRAFT + threadIdx.x] = hist[pos + 1 + threadIdx.x];
+        }
+        if (threadIdx.x == 0) {
+            state[ST_DRAFT_LEN] = dl;
+            state[ST_MATCH_POS] = pos;
+            state[ST_MATCH_LEN] = mlen;
+        }
+    }
+}
+
+struct DraftArg {
+    int n;
+    int tok[kMaxDraftWords];
+};
+
+// Caller-supplied drafts (by value: no host buffer has to outlive the call).
+__global__ void set_draft_kernel(int* state, DraftArg a) {
+    if ((int)threadIdx.x < a.n) state[ST_DRAFT + threadIdx.x] = a.tok[threadIdx.x];
+    if (threadIdx.x == 0) state[ST_DRAFT_LEN] = a.n;
+}
+// Caller-supplied predictions for the stand-alone accept scan.
+__global__ void set_y_kernel(int* state, DraftArg a) {
+    if ((int)threadIdx.x < a.n) state[ST_Y + threadIdx.x] = a.tok[threadIdx.x];
+}
+
+// ------------------------------------------------------------------------------------------
+// Greedy tokens and accept scan.  Row j's token is the best of the per-block candidates
+// (largest logit, lowest id among equals); a = number of leading drafts equal to the model's
+// prediction; emitted = x_1..x_a, y_{a+1}.  One block of 32 * rows threads: warp j reduces row j.
+__global__ void accept_kernel(int* state, const float* cand_val, const int* cand_idx, int G, int from_host_y) {
+    __shared__ int y_s[kMaxRows + 1];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int dl = state[ST_DRAFT_LEN];
+    if (warp <= dl) {
+        int bi;
+        if (from_host_y) {
+            bi = state[ST_Y + warp];
+        } else {
+            float bv = -CUDART_INF_F;
+            bi = 0x7fffffff;
+            for (int c = lane; c < G; c += 32) {
+                const float v = cand_val[(size_t)c * kMaxRows + warp];
+                const int i = cand_idx[(size_t)c * kMaxRows + warp];
+                if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+            }
+            for (int off = 16; off; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+            }
+            if (bi == 0x7fffffff) bi = 0;
+        }
+        if (lane == 0) { y_s[warp] = bi; state[ST_Y + warp] = bi; }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int a = 0;
+        while (a < dl && state[ST_DRAFT + a] == y_s[a]) ++a;
+        for (int i = 0; i < a; ++i) state[ST_EMITTED + i] = state[ST_DRAFT + i];
+        state[ST_EMITTED + a] = y_s[a];
+        state[ST_ACCEPT_LEN] = a;
+        state[ST_N_EMITTED] = a + 1;
+        state[ST_VERIFIED] = 1;
+    }
+}
+
+// Commit: append the emitted tokens (cut to max_emit when > 0) to the history, advance the KV
+// length by their number, make the last one the pending token.  KV rows past the new length
+// are left as they are and overwritten by later steps.
+__global__ void commit_kernel(int* state, int* hist, int max_emit, int force_accept, int force_token) {
+    if (threadIdx.x != 0) return;
+    int n = state[ST_N_EMITTED];
+    if (force_accept >= 0) {
+        n = force_accept + 1;
+        for (int i = 0; i < force_accept; ++i) state[ST_EMITTED + i] = state[ST_DRAFT + i];
+        state[ST_EMITTED + force_accept] = force_token;
+        state[ST_ACCEPT_LEN] = force_accept;
+    }
+    if (max_emit > 0 && n > max_emit) n = max_emit;
+    const int hl = state[ST_HIST_LEN];
+    for (int i = 0; i < n; ++i) hist[hl + i] = state[ST_EMITTED + i];
+    state[ST_N_EMITTED] = n;
+    state[ST_HIST_LEN] = hl + n;
+    state[ST_KV_LEN] += n;
+    state[ST_PENDING] = state[ST_EMITTED + n - 1];
+    state[ST_DRAFT_LEN] = 0;
+    state[ST_VERIFIED] = 0;
+}
+
+// After the last prefill tile: the greedy token of its last row becomes the pending token.
+__global__ void prefill_final_kernel(int* state, int* hist, const float* cand_val, const int* cand_idx, int G,
+                                     int row) {
+    const int lane = threadIdx.x;
+    float bv = -CUDART_INF_F;
+    int bi = 0x7fffffff;
+    for (int c = lane; c < G; c += 32) {
+        const float v = cand_val[(size_t)c * kMaxRows + row];
+        const int i = cand_idx[(size_t)c * kMaxRows + row];
+        if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+    }
+    for (int off = 16; off; off >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+    }
+    if (lane == 0) {
+        if (bi == 0x7fffffff) bi = 0;
+        const int hl = state[ST_HIST_LEN];
+        hist[hl] = bi;
+        state[ST_HIST_LEN] = hl + 1;
+        state[ST_PENDING] = bi;
+        state[ST_DRAFT_LEN] = 0;
+        state[ST_Y] = bi;
+    }
+}
+
+__global__ void set_state_kernel(int* state, int kv_len, int hist_len, int n_ctx, int pending_from_hist,
+                                 const int* hist) {
+    if (threadIdx.x != 0) return;
+    state[ST_KV_LEN] = kv_len;
+    state[ST_HIST_LEN] = hist_len;
+    state[ST_N_CTX] = n_ctx;
+    if (pending_from_hist && hist_len > 0) state[ST_PENDING] = hist[hist_len - 1];
+    state[ST_DRAFT_LEN] = 0;
+    state[ST_VERIFIED] = 0;
+}
+
+// A bounded wait on a word nothing ever sets: exercises the give-up path of the device waits.
+__global__ void timeout_probe_kernel(int* state, const int* never_set, unsigned long long limit_ns) {
+    const uint64_t t0 = global_timer_ns();
+    bool expired = false;
+    while (ld_acquire_gpu(never_set) != 0x5eed) {
+        if (global_timer_ns() - t0 > limit_ns) {
+            expired = true;
+            break;
+        }
+    }
+    if (expired) atomicExch(state + ST_ERR, 2);
+}
+
+}  // namespace sdv
