@@ -1,0 +1,260 @@
+"""ctypes binding of libsdv.so.  Method names follow the C entry points (include/sdv.h)."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+from .build import LIB_PATH, build
+
+OK, EINVAL, ENOMEM, ECAPACITY, ESTATE, ECUDA, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
+K_MAX = 16
+
+EXPORTS = [
+    "sdv_workspace_bytes", "sdv_create", "sdv_load_weights", "sdv_prefill_chunk", "sdv_draft", "sdv_verify",
+    "sdv_commit", "sdv_rollback", "sdv_kv_len", "sdv_set_parity_mode", "sdv_get_logits", "sdv_destroy",
+    "sdv_strerror", "sdv_last_cuda_error", "sdv_step_bytes", "sdv_debug_set_history", "sdv_debug_accept",
+    "sdv_debug_force_commit", "sdv_debug_read_kv", "sdv_debug_read_hidden", "sdv_debug_gemm",
+    "sdv_debug_timeout_probe", "sdv_launch_count", "sdv_last_verify_ms",
+]
+
+
+class SdvConfig(C.Structure):
+    _fields_ = [(n, C.c_int) for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn",
+                                       "vocab", "max_seq", "k_max", "tied_lm_head", "qkv_bias", "ngram_n",
+                                       "ngram_min", "search_history")] + \
+               [("rope_theta", C.c_float), ("rms_eps", C.c_float)]
+
+
+class _LayerWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("wq", "wk", "wv", "wo", "wg", "wu", "wd", "norm1", "norm2",
+                                          "bq", "bk", "bv")]
+
+
+class _Weights(C.Structure):
+    _fields_ = [("emb", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
+                ("layers", C.POINTER(_LayerWeights))]
+
+
+class SdvError(RuntimeError):
+    def __init__(self, code: int, where: str, cuda: int = 0):
+        self.code = code
+        msg = lib().sdv_strerror(code).decode() if _lib is not None else str(code)
+        super().__init__(f"{where}: {msg} ({code})" + (f", CUDA error {cuda}" if cuda else ""))
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None):
+    """Loads (building it first if the sources are newer) the CUDA library.  Fails loudly."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = path or build()
+    L = C.CDLL(path)
+    vp, ip, i32p = C.c_void_p, C.POINTER(C.c_int), C.c_void_p
+    L.sdv_workspace_bytes.argtypes = [C.POINTER(SdvConfig)]
+    L.sdv_workspace_bytes.restype = C.c_size_t
+    L.sdv_create.argtypes = [C.POINTER(SdvConfig), vp, C.c_size_t, vp, C.POINTER(vp)]
+    L.sdv_load_weights.argtypes = [vp, C.POINTER(_Weights)]
+    L.sdv_prefill_chunk.argtypes = [vp, i32p, C.c_int, C.c_int]
+    L.sdv_draft.argtypes = [vp, C.c_int, i32p, ip]
+    L.sdv_verify.argtypes = [vp, i32p, C.c_int, i32p, ip]
+    L.sdv_commit.argtypes = [vp, C.c_int, i32p, ip, ip]
+    L.sdv_rollback.argtypes = [vp, C.c_int]
+    L.sdv_kv_len.argtypes = [vp]
+    L.sdv_set_parity_mode.argtypes = [vp, C.c_int]
+    L.sdv_get_logits.argtypes = [vp, vp, C.c_int]
+    L.sdv_destroy.argtypes = [vp]
+    L.sdv_strerror.argtypes = [C.c_int]
+    L.sdv_strerror.restype = C.c_char_p
+    L.sdv_last_cuda_error.argtypes = [vp]
+    L.sdv_step_bytes.argtypes = [vp, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    L.sdv_debug_set_history.argtypes = [vp, i32p, C.c_int, C.c_int]
+    L.sdv_debug_accept.argtypes = [vp, i32p, C.c_int, i32p, ip]
+    L.sdv_debug_force_commit.argtypes = [vp, C.c_int, C.c_int]
+    L.sdv_debug_read_kv.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, vp]
+    L.sdv_debug_read_hidden.argtypes = [vp, C.c_int, vp]
+    L.sdv_debug_gemm.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_float)]
+    L.sdv_debug_timeout_probe.argtypes = [vp]
+    L.sdv_launch_count.argtypes = [vp]
+    L.sdv_launch_count.restype = C.c_longlong
+    L.sdv_last_verify_ms.argtypes = [vp, C.POINTER(C.c_float)]
+    for name in EXPORTS:
+        if name not in ("sdv_workspace_bytes", "sdv_strerror", "sdv_launch_count"):
+            getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def lib():
+    return load_library()
+
+
+def config_from(cfg, k_max: Optional[int] = None, max_seq: Optional[int] = None,
+                search_history: bool = False) -> SdvConfig:
+    """Builds the C configuration from an object with the ModelConfig field names."""
+    return SdvConfig(cfg.n_layers, cfg.d_model, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.d_ffn, cfg.vocab,
+                     int(max_seq or cfg.max_seq), int(k_max or cfg.k), int(cfg.tied_lm_head), int(cfg.qkv_bias),
+                     cfg.ngram_n, cfg.ngram_min, int(search_history), cfg.rope_theta, cfg.rms_eps)
+
+
+def _ptr(a):
+    if a is None:
+        return None
+    if isinstance(a, np.ndarray):
+        return a.ctypes.data
+    return a.data_ptr()  # torch tensor
+
+
+class Sdv:
+    """One sequence on the current CUDA device.  Owns the torch workspace tensor."""
+
+    def __init__(self, cconfig: SdvConfig, stream=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise SdvError(ECUDA, "Sdv: no CUDA device (there is no CPU fallback)")
+        L = lib()
+        self.cfg = cconfig
+        nbytes = L.sdv_workspace_bytes(C.byref(cconfig))
+        if nbytes == 0:
+            raise SdvError(EINVAL, "sdv_workspace_bytes")
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        self._stream = stream
+        sp = None if stream is None else stream.cuda_stream
+        h = C.c_void_p()
+        self._h = None
+        self._check(L.sdv_create(C.byref(cconfig), base, nbytes, sp, C.byref(h)), "sdv_create", ctx=None)
+        self._h = h
+        self.workspace_bytes = nbytes
+
+    # -- helpers
+    def _check(self, rc: int, where: str, ctx="self"):
+        if rc != OK:
+            cuda = lib().sdv_last_cuda_error(self._h) if (ctx and self._h) else 0
+            raise SdvError(rc, where, cuda)
+
+    def close(self):
+        if self._h is not None:
+            lib().sdv_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the calls
+    def load_weights(self, weights):
+        """weights: an object with the ModelWeights field names (numpy arrays or CUDA tensors)."""
+        n = len(weights.layers)
+        arr = (_LayerWeights * n)()
+        for i, lw in enumerate(weights.layers):
+            for name in ("wq", "wk", "wv", "wo", "wg", "wu", "wd", "norm1", "norm2", "bq", "bk", "bv"):
+                setattr(arr[i], name, _ptr(getattr(lw, name)))
+        w = _Weights(_ptr(weights.emb), _ptr(weights.lm_head), _ptr(weights.final_norm), arr)
+        self._check(lib().sdv_load_weights(self._h, C.byref(w)), "sdv_load_weights")
+
+    def prefill_chunk(self, tokens, is_last: bool):
+        t = np.ascontiguousarray(tokens, dtype=np.int32)
+        self._check(lib().sdv_prefill_chunk(self._h, t.ctypes.data, len(t), int(is_last)), "sdv_prefill_chunk")
+
+    def draft(self, k: int, fetch: bool = True) -> Optional[List[int]]:
+        if not fetch:
+            self._check(lib().sdv_draft(self._h, k, None, None), "sdv_draft")
+            return None
+        out = np.zeros(K_MAX, dtype=np.int32)
+        dl = C.c_int(0)
+        self._check(lib().sdv_draft(self._h, k, out.ctypes.data, C.byref(dl)), "sdv_draft")
+        return out[:dl.value].tolist()
+
+    def verify(self, draft: Optional[Sequence[int]] = None, fetch: bool = True) -> Optional[Tuple[List[int], int]]:
+        """draft=None verifies the device draft left by draft(); returns (y, accept_len) when fetch."""
+        d = None if draft is None else np.ascontiguousarray(draft, dtype=np.int32)
+        dp = None if d is None else (d.ctypes.data if len(d) else np.zeros(1, np.int32).ctypes.data)
+        dl = 0 if d is None else len(d)
+        if not fetch:
+            self._check(lib().sdv_verify(self._h, dp, dl, None, None), "sdv_verify")
+            return None
+        y = np.zeros(K_MAX + 1, dtype=np.int32)
+        a = C.c_int(0)
+        self._check(lib().sdv_verify(self._h, dp, dl, y.ctypes.data, C.byref(a)), "sdv_verify")
+        return y, a.value
+
+    def commit(self, max_emit: int = 0) -> Tuple[List[int], int]:
+        out = np.zeros(K_MAX + 1, dtype=np.int32)
+        n, kv = C.c_int(0), C.c_int(0)
+        self._check(lib().sdv_commit(self._h, max_emit, out.ctypes.data, C.byref(n), C.byref(kv)), "sdv_commit")
+        return out[:n.value].tolist(), kv.value
+
+    def rollback(self, new_kv_len: int):
+        self._check(lib().sdv_rollback(self._h, new_kv_len), "sdv_rollback")
+
+    def kv_len(self) -> int:
+        return lib().sdv_kv_len(self._h)
+
+    def set_parity_mode(self, on: bool):
+        self._check(lib().sdv_set_parity_mode(self._h, int(on)), "sdv_set_parity_mode")
+
+    def get_logits(self, rows: int) -> np.ndarray:
+        out = np.empty((rows, self.cfg.vocab), dtype=np.float32)
+        self._check(lib().sdv_get_logits(self._h, out.ctypes.data, rows), "sdv_get_logits")
+        return out
+
+    def step_bytes(self, rows: int, kv_len: int) -> Tuple[float, float]:
+        w, k = C.c_double(0), C.c_double(0)
+        self._check(lib().sdv_step_bytes(self._h, rows, kv_len, C.byref(w), C.byref(k)), "sdv_step_bytes")
+        return w.value, k.value
+
+    def launch_count(self) -> int:
+        return int(lib().sdv_launch_count(self._h))
+
+    def last_verify_ms(self) -> float:
+        ms = C.c_float(0)
+        self._check(lib().sdv_last_verify_ms(self._h, C.byref(ms)), "sdv_last_verify_ms")
+        return ms.value
+
+    # -- test / measurement entry points
+    def debug_set_history(self, hist, n_ctx: int):
+        h = np.ascontiguousarray(hist, dtype=np.int32)
+        self._check(lib().sdv_debug_set_history(self._h, h.ctypes.data, len(h), n_ctx), "sdv_debug_set_history")
+
+    def debug_accept(self, draft, y) -> int:
+        d = np.ascontiguousarray(draft, dtype=np.int32)
+        yy = np.ascontiguousarray(y, dtype=np.int32)
+        a = C.c_int(0)
+        dp = d.ctypes.data if len(d) else None
+        self._check(lib().sdv_debug_accept(self._h, dp, len(d), yy.ctypes.data, C.byref(a)), "sdv_debug_accept")
+        return a.value
+
+    def debug_force_commit(self, accept_len: int, next_token: int):
+        self._check(lib().sdv_debug_force_commit(self._h, accept_len, next_token), "sdv_debug_force_commit")
+
+    def debug_read_kv(self, layer: int, which: int, pos0: int, n: int) -> np.ndarray:
+        out = np.empty((self.cfg.n_kv_heads, n, self.cfg.head_dim), dtype=np.float32)
+        self._check(lib().sdv_debug_read_kv(self._h, layer, which, pos0, n, out.ctypes.data), "sdv_debug_read_kv")
+        return out
+
+    def debug_read_hidden(self, rows: int) -> np.ndarray:
+        out = np.empty((rows, self.cfg.d_model), dtype=np.float32)
+        self._check(lib().sdv_debug_read_hidden(self._h, rows, out.ctypes.data), "sdv_debug_read_hidden")
+        return out
+
+    def debug_gemm(self, x: np.ndarray, w_bits: np.ndarray) -> Tuple[np.ndarray, float]:
+        x = np.ascontiguousarray(x, dtype=np.float32)
+        w_bits = np.ascontiguousarray(w_bits, dtype=np.uint16)
+        M, K = x.shape
+        N = w_bits.shape[0]
+        y = np.empty((M, N), dtype=np.float32)
+        ms = C.c_float(0)
+        self._check(lib().sdv_debug_gemm(self._h, x.ctypes.data, w_bits.ctypes.data, y.ctypes.data, M, N, K,
+                                         C.byref(ms)), "sdv_debug_gemm")
+        return y, ms.value
+
+    def debug_timeout_probe(self) -> int:
+        return lib().sdv_debug_timeout_probe(self._h)

@@ -77,6 +77,7 @@ static_assert(sizeof(Misc) <= kMiscSmemBytes, "misc shared memory");
 // Called by all worker threads.  Returns, identically for all of them, whether some bounded
 // wait in this block has been abandoned (the remaining phases then do no work).
 __device__ __forceinline__ bool grid_barrier(const FwdParams& P, int target, Misc* misc, int wtid) {
+    __threadfence();  // every thread's own stores and reductions are performed before it reports in
     named_bar_sync(1, kWorkerThreads);
     if (wtid == 0) {
         __threadfence();

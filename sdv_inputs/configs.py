@@ -29,6 +29,8 @@ class ModelConfig:
     repeat_spans: int = -1      # exact number of copied spans (>=0) ...
     repeat_frac: float = 0.25   # ... or a fraction of all spans (when repeat_spans < 0)
     zipf_s: float = 1.1
+    resid_scale: float = 0.5    # Wo / Wd scale relative to an embedding row (see make_weights)
+    qk_var: float = 1.0         # variance of the attention scores the random Wq, Wk produce
     seed: int = 0
 
     @property
