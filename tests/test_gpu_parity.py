@@ -1,0 +1,229 @@
+"""GPU-vs-oracle parity of the whole path (prefill, draft, verify, accept, commit) through the
+C-ABI.  Tolerances: drafts, accept lengths and KV lengths bit-exact; logits max |d| <= 0.05 and
+cosine >= 0.999 per row; greedy tokens identical except where the oracle's own top-2 margin is
+below 0.05 (then the other token must be the oracle's runner-up)."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import sdv_oracle as O
+from sdv_inputs import get_config, make_context, make_weights
+from paper_2510_15312_b200.binding import Sdv, config_from
+from helpers import LOGIT_TOL, MARGIN_TOL, compare_step, steps_from_golden, steps_from_oracle
+
+pytestmark = pytest.mark.gpu
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def gpu_prefill(s, ctx, chunk):
+    n = len(ctx)
+    for i in range(0, n, chunk):
+        s.prefill_chunk(ctx[i:i + chunk], is_last=(i + chunk >= n))
+
+
+class Workload:
+    def __init__(self, name, **over):
+        self.cfg = get_config(name).with_(**over) if over else get_config(name)
+        self.w = make_weights(self.cfg)
+        self.ctx = make_context(self.cfg)
+
+
+@pytest.fixture(scope="module", params=["tiny", "mini_gqa", "mini_hd128"])
+def small(request):
+    return Workload(request.param)
+
+
+def true_continuation_drafter(cfg, greedy):
+    step = [0]
+
+    def drafter(hist, k):
+        s = step[0]
+        step[0] += 1
+        i0 = len(hist) - cfg.n_ctx
+        d = [greedy[i0 + i] if i0 + i < cfg.gen else 0 for i in range(k)]
+        e = s % (k + 1) + 1
+        if e <= k:
+            d[e - 1] = (d[e - 1] + 1) % cfg.vocab
+        return d
+    return drafter
+
+
+def check_prefill(s, wl, ref_model, last_logits):
+    cfg = wl.cfg
+    n = cfg.n_ctx
+    T = O.argmax(last_logits)
+    for layer in (0, cfg.n_layers - 1):
+        for which, name in ((0, "k"), (1, "v")):
+            kv = s.debug_read_kv(layer, which, 0, n)
+            ref = ref_model.kv_view(name)[layer][:, :n]
+            scale = np.abs(ref).max()
+            assert np.abs(kv - ref).max() <= 0.02 * scale + 1e-3, (layer, name)
+    return T
+
+
+def test_teacher_forced_steps_with_drafter(small):
+    """Protocol (i) with the n-gram drafter's own drafts, context-only search."""
+    cfg = small.cfg
+    ref = O.OracleModel(small.w)
+    toks, steps = O.spec_decode(ref, small.ctx, cfg.gen, cfg.chunk, cfg.k, cfg.ngram_n, cfg.ngram_min,
+                                keep_logits=True)
+    s = Sdv(config_from(cfg))
+    s.load_weights(small.w)
+    s.set_parity_mode(True)
+    gpu_prefill(s, small.ctx, cfg.chunk)
+    ref2 = O.OracleModel(small.w)
+    last = ref2.prefill(small.ctx, cfg.chunk)
+    check_prefill(s, small, ref2, last)
+    s.debug_set_history(list(small.ctx) + [toks[0]], cfg.n_ctx)
+    stats = {}
+    for st in steps_from_oracle(steps, from_drafter=True):
+        compare_step(s, st, cfg.k, stats)
+    assert s.kv_len() == cfg.n_ctx + cfg.gen - 1
+    print(cfg.name, stats.get("max_err"), stats.get("min_cos"), stats.get("near_tie_flips", 0))
+    s.close()
+
+
+def test_teacher_forced_steps_every_accept_length(small):
+    """Protocol (i) with forced drafts: the true continuation corrupted at a cycling position, so that
+    accept lengths 0..k all occur and rows after the mismatch are exercised."""
+    cfg = small.cfg
+    greedy = O.greedy_decode(O.OracleModel(small.w), small.ctx, cfg.gen, cfg.chunk)
+    ref = O.OracleModel(small.w)
+    toks, steps = O.spec_decode(ref, small.ctx, cfg.gen, cfg.chunk, cfg.k, cfg.ngram_n, cfg.ngram_min,
+                                drafter=true_continuation_drafter(cfg, greedy), keep_logits=True)
+    assert toks == greedy
+    s = Sdv(config_from(cfg))
+    s.load_weights(small.w)
+    s.set_parity_mode(True)
+    gpu_prefill(s, small.ctx, cfg.chunk)
+    s.debug_set_history(list(small.ctx) + [toks[0]], cfg.n_ctx)
+    stats = {}
+    for st in steps_from_oracle(steps, from_drafter=False):
+        compare_step(s, st, cfg.k, stats)
+    assert len(set(stats["accepts"])) >= min(cfg.k + 1, 3)
+    assert s.kv_len() == cfg.n_ctx + cfg.gen - 1
+    s.close()
+
+
+def test_free_running_stream_matches_until_first_near_tie(small):
+    """Protocol (ii): the GPU loop on its own (history search on, so drafts do get accepted)."""
+    cfg = small.cfg
+    ref = O.OracleModel(small.w)
+    last = ref.prefill(small.ctx, cfg.chunk)
+    ref = O.OracleModel(small.w)
+    toks, steps = O.spec_decode(ref, small.ctx, cfg.gen, cfg.chunk, cfg.k, cfg.ngram_n, cfg.ngram_min,
+                                search_history=True)
+    margins = [O.top2_margin(last)]
+    for st in steps:
+        margins.extend(st.margin[:len(st.emitted)])
+    s = Sdv(config_from(cfg, search_history=True))
+    s.load_weights(small.w)
+    gpu_prefill(s, small.ctx, cfg.chunk)
+    out = []      # tokens after the first one (the first is the pending token left by prefill)
+    while len(out) < cfg.gen - 1:
+        s.draft(cfg.k, fetch=False)
+        s.verify(None, fetch=False)
+        emitted, kv = s.commit(max_emit=cfg.gen - 1 - len(out))
+        out.extend(emitted)
+        assert kv == cfg.n_ctx + len(out)
+    first_tie = next((i for i, m in enumerate(margins) if m < MARGIN_TOL), len(margins))
+    matched = 0
+    for a, b in zip(out, toks[1:]):
+        if a != b:
+            break
+        matched += 1
+    required = max(0, min(first_tie, len(toks)) - 1)
+    assert matched >= required, (matched, first_tie)
+    s.close()
+
+
+def test_chunked_prefill_is_chunk_size_invariant(small):
+    """Sec. 4.2 graph equivalence on the GPU path: any chunking gives the same cache and first token
+    (up to bf16 rounding of rows whose fp32 sums were taken in another order)."""
+    cfg = small.cfg
+    ref = None
+    for chunk in (cfg.chunk, 7, cfg.n_ctx):
+        s = Sdv(config_from(cfg))
+        s.load_weights(small.w)
+        gpu_prefill(s, small.ctx, chunk)
+        assert s.kv_len() == cfg.n_ctx
+        k = s.debug_read_kv(cfg.n_layers - 1, 0, 0, cfg.n_ctx)
+        v = s.debug_read_kv(cfg.n_layers - 1, 1, 0, cfg.n_ctx)
+        y, _ = s.verify([])
+        if ref is None:
+            ref = (k, v, y[0])
+        else:
+            assert np.abs(k - ref[0]).max() <= 0.02 * np.abs(ref[0]).max()
+            assert np.abs(v - ref[1]).max() <= 0.02 * np.abs(ref[1]).max()
+        s.close()
+
+
+def test_short_context_verify_is_sensitive_to_the_causal_mask():
+    """With only a handful of cached keys the draft rows dominate each other's attention, so a wrong
+    mask among the new rows could not stay within tolerance."""
+    wl = Workload("mini_hd128", n_ctx=5, gen=40)
+    cfg = wl.cfg
+    greedy = O.greedy_decode(O.OracleModel(wl.w), wl.ctx, cfg.gen, cfg.chunk)
+    ref = O.OracleModel(wl.w)
+    toks, steps = O.spec_decode(ref, wl.ctx, cfg.gen, cfg.chunk, cfg.k, cfg.ngram_n, cfg.ngram_min,
+                                drafter=true_continuation_drafter(cfg, greedy), keep_logits=True)
+    s = Sdv(config_from(cfg))
+    s.load_weights(wl.w)
+    s.set_parity_mode(True)
+    gpu_prefill(s, wl.ctx, cfg.chunk)
+    s.debug_set_history(list(wl.ctx) + [toks[0]], cfg.n_ctx)
+    stats = {}
+    for st in steps_from_oracle(steps, from_drafter=False):
+        compare_step(s, st, cfg.k, stats)
+    s.close()
+
+
+def test_qwen05b_shape_live_oracle():
+    """The 0.5B-shaped workload against the oracle run live, on a shortened generation."""
+    wl = Workload("qwen0.5b", gen=24)
+    cfg = wl.cfg
+    greedy = O.greedy_decode(O.OracleModel(wl.w), wl.ctx, cfg.gen, cfg.chunk)
+    ref = O.OracleModel(wl.w)
+    toks, steps = O.spec_decode(ref, wl.ctx, cfg.gen, cfg.chunk, cfg.k, cfg.ngram_n, cfg.ngram_min,
+                                drafter=true_continuation_drafter(cfg, greedy), keep_logits=True)
+    s = Sdv(config_from(cfg))
+    s.load_weights(wl.w)
+    s.set_parity_mode(True)
+    gpu_prefill(s, wl.ctx, cfg.chunk)
+    s.debug_set_history(list(wl.ctx) + [toks[0]], cfg.n_ctx)
+    stats = {}
+    for st in steps_from_oracle(steps, from_drafter=False):
+        compare_step(s, st, cfg.k, stats)
+    print("qwen0.5b", stats.get("max_err"), stats.get("min_cos"))
+    s.close()
+
+
+@pytest.mark.parametrize("name", ["qwen1.5b", "llama3b", "qwen7b"])
+def test_full_size_workloads_against_stored_oracle_trajectory(name):
+    """Full-size configurations in the launch shape the benchmark times, compared step by step with
+    the oracle trajectory stored by tests/golden/make_golden.py (logits at sampled vocabulary ids
+    and the oracle's own best ids)."""
+    path = os.path.join(GOLD, f"{name}.npz")
+    if not os.path.exists(path):
+        pytest.skip(f"{path} not generated")
+    g = np.load(path)
+    cfg = get_config(name)
+    w = make_weights(cfg, threads=16)
+    ctx = make_context(cfg)
+    s = Sdv(config_from(cfg, k_max=int(g["k"])))
+    s.load_weights(w)
+    s.set_parity_mode(True)
+    gpu_prefill(s, ctx, cfg.chunk)
+    for layer in (0, cfg.n_layers - 1):
+        for which, nm in ((0, "k"), (1, "v")):
+            ref = g[f"{nm}{layer}"]
+            for j, pos in enumerate(g["kv_pos"]):
+                got = s.debug_read_kv(layer, which, int(pos), 1)[:, 0]
+                assert np.abs(got - ref[:, j]).max() <= 0.02 * np.abs(ref).max() + 1e-3
+    s.debug_set_history(list(ctx) + [int(g["first_token"])], cfg.n_ctx)
+    stats = {}
+    for st in steps_from_golden(g):
+        compare_step(s, st, int(g["k"]), stats)
+    print(name, stats.get("max_err"), stats.get("min_cos"), stats.get("near_tie_flips", 0))
+    s.close()
