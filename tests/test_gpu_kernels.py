@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 
 from oracle import sdv_oracle as O
-from sdv_inputs import bf16_bits_to_f32, f32_to_bf16_bits, get_config
+from sdv_inputs import bf16_bits_to_f32, f32_to_bf16_bits, get_config, make_weights
 import paper_2510_15312_b200 as pkg
 from paper_2510_15312_b200.binding import Sdv, config_from
 
@@ -119,6 +119,8 @@ def test_call_order_and_capacity_errors():
     toks = np.zeros(80, np.int32)
     assert L.sdv_prefill_chunk(s._h, toks.ctypes.data, 8, 0) == pkg.ESTATE  # weights not loaded yet
     s.debug_set_history(np.arange(20, dtype=np.int32), 20)
+    assert L.sdv_verify(s._h, None, 0, None, None) == pkg.ESTATE           # still no weights
+    s.load_weights(make_weights(cfg))
     assert L.sdv_draft(s._h, 5, None, None) == pkg.EINVAL                   # k > k_max
     assert L.sdv_verify(s._h, toks.ctypes.data, 5, None, None) == pkg.EINVAL
     bad = np.array([4096], np.int32)
