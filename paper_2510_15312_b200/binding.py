@@ -17,7 +17,7 @@ EXPORTS = [
     "sdv_commit", "sdv_rollback", "sdv_kv_len", "sdv_set_parity_mode", "sdv_get_logits", "sdv_destroy",
     "sdv_strerror", "sdv_last_cuda_error", "sdv_step_bytes", "sdv_debug_set_history", "sdv_debug_accept",
     "sdv_debug_force_commit", "sdv_debug_read_kv", "sdv_debug_read_hidden", "sdv_debug_gemm",
-    "sdv_debug_timeout_probe", "sdv_launch_count", "sdv_last_verify_ms",
+    "sdv_debug_timeout_probe", "sdv_debug_profile", "sdv_launch_count", "sdv_last_verify_ms",
 ]
 
 
@@ -80,6 +80,7 @@ def load_library(path: Optional[str] = None):
     L.sdv_debug_read_hidden.argtypes = [vp, C.c_int, vp]
     L.sdv_debug_gemm.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_float)]
     L.sdv_debug_timeout_probe.argtypes = [vp]
+    L.sdv_debug_profile.argtypes = [vp, C.c_int, vp, C.c_int]
     L.sdv_launch_count.argtypes = [vp]
     L.sdv_launch_count.restype = C.c_longlong
     L.sdv_last_verify_ms.argtypes = [vp, C.POINTER(C.c_float)]
@@ -255,6 +256,21 @@ class Sdv:
         self._check(lib().sdv_debug_gemm(self._h, x.ctypes.data, w_bits.ctypes.data, y.ctypes.data, M, N, K,
                                          C.byref(ms)), "sdv_debug_gemm")
         return y, ms.value
+
+    def debug_profile(self, on: bool, n_phases: int = 0) -> Optional[np.ndarray]:
+        """Switches per-phase timestamps on/off; with n_phases > 0 first returns the last recording
+        as uint64 [n_phases, blocks, 8]."""
+        L = lib()
+        G = L.sdv_debug_profile(self._h, int(on), None, 0)
+        if G < 0:
+            raise SdvError(G, "sdv_debug_profile")
+        if n_phases <= 0:
+            return None
+        out = np.zeros((n_phases, G, 8), dtype=np.uint64)
+        rc = L.sdv_debug_profile(self._h, int(on), out.ctypes.data, n_phases)
+        if rc < 0:
+            raise SdvError(rc, "sdv_debug_profile")
+        return out
 
     def debug_timeout_probe(self) -> int:
         return lib().sdv_debug_timeout_probe(self._h)

@@ -6,11 +6,13 @@
 //                and keeps a ring of 16 KB shared-memory stages full with bulk asynchronous copies.
 //                It never waits for activations or grid barriers, only for free ring slots, so HBM
 //                traffic continues across operation boundaries.
-//   warps 8..10  activation loaders: fill each stage's [rows x 64] bf16 operand from L2, applying
-//                the producing step's deferred work (RMSNorm scale, split-KV combine).
-//   warps 0..7   MMA warps: one 16-row weight tile each per stage (weights are the MMA "A" operand,
-//                token rows the 8-wide "B" operand), epilogues fused per operation.
-// Operations are separated by a bounded grid barrier; attention uses all 11 non-producer warps.
+//   warps 8..10  activation loaders: fill each stage's bf16 operand chunks ([rows x 64] each) from
+//                L2, two chunks in flight per warp, applying the RMSNorm scale where one is due.
+//   warps 0..7   MMA warps in an RW x KW grid: warp (rw, kw) multiplies row tile rw of the stage by
+//                operand chunk kw (weights are the MMA "A" operand, token rows the 8-wide "B"
+//                operand); epilogues are fused per operation.
+// Operations are separated by a bounded grid barrier; attention and the split-KV merge use all 11
+// non-producer warps.
 #pragma once
 #include <math_constants.h>
 
@@ -19,17 +21,18 @@
 
 namespace sdv {
 
-enum PhaseKind { PH_EMBED = 0, PH_QKV, PH_ATTN, PH_O, PH_GU, PH_DOWN, PH_LM, PH_RAW };
+enum PhaseKind { PH_EMBED = 0, PH_QKV, PH_ATTN, PH_COMB, PH_O, PH_GU, PH_DOWN, PH_LM, PH_RAW };
+constexpr int kPhasesPerLayer = 6;
 
-// Phase numbering of a launch: 0 = embedding; 1 + 5*layer + {0..4} = QKV, attention, output
-// projection, gate|up, down; 1 + 5*n_layers = LM head; 2 + 5*n_layers = the stand-alone GEMM.
-__device__ __forceinline__ int decode_phase(int ph, int n_layers, int& layer) {
+// Phase numbering of a launch: 0 = embedding; 1 + 6*layer + {0..5} = QKV, attention, split merge,
+// output projection, gate|up, down; 1 + 6*n_layers = LM head; 2 + 6*n_layers = stand-alone GEMM.
+__host__ __device__ __forceinline__ int decode_phase(int ph, int n_layers, int& layer) {
     layer = 0;
     if (ph == 0) return PH_EMBED;
-    if (ph == 1 + 5 * n_layers) return PH_LM;
-    if (ph == 2 + 5 * n_layers) return PH_RAW;
-    layer = (ph - 1) / 5;
-    return PH_QKV + (ph - 1) % 5;
+    if (ph == 1 + kPhasesPerLayer * n_layers) return PH_LM;
+    if (ph == 2 + kPhasesPerLayer * n_layers) return PH_RAW;
+    layer = (ph - 1) / kPhasesPerLayer;
+    return PH_QKV + (ph - 1) % kPhasesPerLayer;
 }
 __device__ __forceinline__ int phase_op(int kind) {
     switch (kind) {
@@ -51,7 +54,8 @@ __device__ __forceinline__ const uint8_t* op_weights(const FwdParams& P, int kin
 template <int NT>
 struct SmemLayout {
     static constexpr int MP = 8 * NT;
-    static constexpr int A_STAGE = MP * 128;
+    static constexpr int A_CHUNK = MP * 128;
+    static constexpr int A_STAGE = kMaxKW * A_CHUNK;
     static constexpr int NSTAGE =
         (kSmemBudget - 1024 - kAttnSmemBytes - kMiscSmemBytes) / (kStageWeightBytes + A_STAGE);
     static constexpr int W_OFF = 0;
@@ -77,7 +81,6 @@ static_assert(sizeof(Misc) <= kMiscSmemBytes, "misc shared memory");
 // Called by all worker threads.  Returns, identically for all of them, whether some bounded
 // wait in this block has been abandoned (the remaining phases then do no work).
 __device__ __forceinline__ bool grid_barrier(const FwdParams& P, int target, Misc* misc, int wtid) {
-    __threadfence();  // every thread's own stores and reductions are performed before it reports in
     named_bar_sync(1, kWorkerThreads);
     if (wtid == 0) {
         __threadfence();
@@ -103,29 +106,39 @@ __device__ __forceinline__ bool grid_barrier(const FwdParams& P, int target, Mis
 // ------------------------------------------------------------------------------------------
 // Weight streamer (one thread).
 template <int NT>
-__device__ void producer_loop(const FwdParams& P, uint8_t* smem, Misc* misc) {
+__device__ __forceinline__ void producer_loop(const FwdParams& P, uint8_t* smem, Misc* misc) {
     using SL = SmemLayout<NT>;
     const int cta = blockIdx.x;
     const uint64_t policy = l2_policy_evict_first();
     uint32_t it = 0;
+    const uint32_t ahead = (P.ahead >= 1 && P.ahead <= SL::NSTAGE) ? (uint32_t)P.ahead : (uint32_t)SL::NSTAGE;
     bool ok = true;
     for (int ph = P.ph_begin; ph < P.ph_end && ok; ++ph) {
         int layer;
         const int kind = decode_phase(ph, P.n_layers, layer);
         const int op = phase_op(kind);
         if (op < 0) continue;
-        const Part pt = get_part(P.op[op], cta, P.G);
+        const OpDesc& od = P.op[op];
+        const Part pt = get_part(od, cta, P.G);
         if (pt.ntiles == 0) continue;
+        const int KW = kConsumerWarps / od.RW;
         const uint8_t* src = op_weights(P, kind, layer) + pt.off;
-        const int npass = part_passes(pt);
+        const int npass = part_passes(pt, od.RW);
+        const int nst = (pt.nchunks + KW - 1) / KW;
         for (int p = 0; p < npass && ok; ++p) {
-            const uint32_t bytes = (uint32_t)even_count(pt.ntiles, npass, p) * kTileBytes;
-            for (int c = 0; c < pt.nchunks; ++c, ++it) {
-                const uint32_t slot = it % SL::NSTAGE, use = it / SL::NSTAGE;
-                if (use > 0 && !mbar_wait_bounded(&misc->empty[slot], (use - 1) & 1, &misc->abort_flag,
-                                                  P.wait_limit_ns)) {
-                    ok = false;
-                    break;
+            const int pcount = even_count(pt.ntiles, npass, p);
+            for (int st = 0; st < nst; ++st, ++it) {
+                const int kcnt = min(KW, pt.nchunks - st * KW);
+                const uint32_t bytes = (uint32_t)(pcount * kcnt) * kTileBytes;
+                const uint32_t slot = it % SL::NSTAGE;
+                // run at most `ahead` stages in front of the MMA warps: stage it - ahead must be consumed
+                if (it >= ahead) {
+                    const uint32_t j = it - ahead;
+                    if (!mbar_wait_bounded(&misc->empty[j % SL::NSTAGE], (j / SL::NSTAGE) & 1, &misc->abort_flag,
+                                           P.wait_limit_ns)) {
+                        ok = false;
+                        break;
+                    }
                 }
                 mbar_arrive_expect_tx(&misc->full_w[slot], bytes);
                 bulk_g2s(smem + SL::W_OFF + slot * kStageWeightBytes, src, bytes, &misc->full_w[slot], policy);
@@ -147,159 +160,184 @@ __device__ void producer_loop(const FwdParams& P, uint8_t* smem, Misc* misc) {
 }
 
 // ------------------------------------------------------------------------------------------
-// Activation loaders.  Loader warp w fills the operand of every stage with index = w mod 3.
-template <int NT>
-__device__ __forceinline__ void load_norm_chunk(const FwdParams& P, const float* wn, int col0, uint8_t* dst, int lane,
-                                                float (&ss)[2 * NT], bool accumulate) {
-#pragma unroll
-    for (int i = 0; i < 2 * NT; ++i) {
-        const int u = lane + 32 * i, tok = u >> 3, q = u & 7;
-        uint4 out = make_uint4(0, 0, 0, 0);
-        if (tok < P.M) {
-            const float* hp = P.h + (size_t)tok * P.d + col0 + q * 8;
-            const float4 a = ldcg_f4(hp), b = ldcg_f4(hp + 4);
-            const float4 wa = __ldg(reinterpret_cast<const float4*>(wn + col0 + q * 8));
-            const float4 wb = __ldg(reinterpret_cast<const float4*>(wn + col0 + q * 8 + 4));
-            if (accumulate)
-                ss[i] += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w + b.x * b.x + b.y * b.y + b.z * b.z + b.w * b.w;
-            out.x = pack_bf16(a.x * wa.x, a.y * wa.y);
-            out.y = pack_bf16(a.z * wa.z, a.w * wa.w);
-            out.z = pack_bf16(b.x * wb.x, b.y * wb.y);
-            out.w = pack_bf16(b.z * wb.z, b.w * wb.w);
-        }
-        *reinterpret_cast<uint4*>(dst + swz_unit(tok, q)) = out;
-    }
-}
+// Activation loaders.  The operand chunks of a phase are dealt round-robin to the three loader
+// warps; each warp keeps two chunks' loads in flight (registers) and stores a chunk into its
+// stage's slot once the slot is free.
+template <int NT, bool NORM>
+struct ChunkRegs {
+    // NORM: fp32 residual values of 2*NT (token, 8-column) units + the 8 norm weights of the lane's
+    // column group; otherwise 2*NT ready-made 16-byte bf16 units.
+    float4 h[NORM ? 2 * NT : 1][2];
+    float4 w[2];
+    uint4 v[NORM ? 1 : 2 * NT];
+};
 
-template <int NT>
-__device__ __forceinline__ void load_copy_chunk(const uint8_t* src, uint8_t* dst, int lane) {
+template <int NT, bool NORM>
+__device__ __forceinline__ void chunk_issue(const FwdParams& P, ChunkRegs<NT, NORM>& r, const float* wn,
+                                            const uint8_t* src_op, int chunk, int lane) {
+    if (NORM) {
+        const int q = lane & 7;
+        r.w[0] = __ldg(reinterpret_cast<const float4*>(wn + chunk * 64 + q * 8));
+        r.w[1] = __ldg(reinterpret_cast<const float4*>(wn + chunk * 64 + q * 8 + 4));
 #pragma unroll
-    for (int i = 0; i < 2 * NT; ++i) {
-        const int u = lane + 32 * i;
-        *reinterpret_cast<uint4*>(dst + u * 16) = ldcg_u4(src + u * 16);
-    }
-}
-
-__device__ __forceinline__ int attn_splits(int L) {
-    if (L <= 0) return 0;
-    const int s = (L + kSplitTargetKeys - 1) / kSplitTargetKeys;
-    return s < kMaxSplits ? s : kMaxSplits;
-}
-__device__ __forceinline__ int attn_keys_per_split(int L, int S) {
-    const int k = (L + S - 1) / S;
-    return (k + kAttnBlockKeys - 1) / kAttnBlockKeys * kAttnBlockKeys;
-}
-
-// Operand of the output projection: merge the split-KV partial results of one head's columns.
-template <int NT>
-__device__ __forceinline__ void load_combine_chunk(const FwdParams& P, int col0, uint8_t* dst, int lane) {
-    const int hq = col0 / P.hd, co = col0 % P.hd;
-    const int S1 = attn_splits(P.L) + 1;
-#pragma unroll 1
-    for (int i = 0; i < 2 * NT; ++i) {
-        const int u = lane + 32 * i, tok = u >> 3, q = u & 7;
-        uint4 out = make_uint4(0, 0, 0, 0);
-        if (tok < P.M) {
-            const size_t base = ((size_t)hq * (kMaxSplits + 1)) * kMaxRows + tok;
-            float mmax = -CUDART_INF_F;
-            for (int s = 0; s < S1; ++s)
-                mmax = fmaxf(mmax, __ldcg(P.part_ml + (base + (size_t)s * kMaxRows) * 2));
-            float den = 0.f, acc[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-            for (int s = 0; s < S1; ++s) {
-                const size_t row = base + (size_t)s * kMaxRows;
-                const float2 ml = __ldcg(reinterpret_cast<const float2*>(P.part_ml + row * 2));
-                const float wgt = exp2f(ml.x - mmax);  // 0 for a split that saw no key (m = -inf)
-                den += wgt * ml.y;
-                const float* op = P.part_o + row * P.hd + co + q * 8;
-                const float4 a = ldcg_f4(op), b = ldcg_f4(op + 4);
-                acc[0] += wgt * a.x; acc[1] += wgt * a.y; acc[2] += wgt * a.z; acc[3] += wgt * a.w;
-                acc[4] += wgt * b.x; acc[5] += wgt * b.y; acc[6] += wgt * b.z; acc[7] += wgt * b.w;
+        for (int i = 0; i < 2 * NT; ++i) {
+            const int tok = (lane + 32 * i) >> 3;
+            if (tok < P.M) {
+                const float* hp = P.h + (size_t)tok * P.d + chunk * 64 + q * 8;
+                r.h[NORM ? i : 0][0] = ldcg_f4(hp);
+                r.h[NORM ? i : 0][1] = ldcg_f4(hp + 4);
             }
-            const float inv = 1.f / den;
-            out.x = pack_bf16(acc[0] * inv, acc[1] * inv);
-            out.y = pack_bf16(acc[2] * inv, acc[3] * inv);
-            out.z = pack_bf16(acc[4] * inv, acc[5] * inv);
-            out.w = pack_bf16(acc[6] * inv, acc[7] * inv);
         }
-        *reinterpret_cast<uint4*>(dst + swz_unit(tok, q)) = out;
+    } else {
+        const uint8_t* src = src_op + (size_t)chunk * SmemLayout<NT>::A_CHUNK;
+#pragma unroll
+        for (int i = 0; i < 2 * NT; ++i) r.v[NORM ? 0 : i] = ldcg_u4(src + (lane + 32 * i) * 16);
+    }
+}
+
+template <int NT, bool NORM>
+__device__ __forceinline__ void chunk_store(const FwdParams& P, const ChunkRegs<NT, NORM>& r, uint8_t* dst, int lane,
+                                            float (&ss)[2 * NT], bool accumulate) {
+    if (NORM) {
+        const int q = lane & 7;
+#pragma unroll
+        for (int i = 0; i < 2 * NT; ++i) {
+            const int tok = (lane + 32 * i) >> 3;
+            uint4 out = make_uint4(0, 0, 0, 0);
+            if (tok < P.M) {
+                const float4 a = r.h[NORM ? i : 0][0], b = r.h[NORM ? i : 0][1];
+                if (accumulate)
+                    ss[i] += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w + b.x * b.x + b.y * b.y + b.z * b.z +
+                             b.w * b.w;
+                out.x = pack_bf16(a.x * r.w[0].x, a.y * r.w[0].y);
+                out.y = pack_bf16(a.z * r.w[0].z, a.w * r.w[0].w);
+                out.z = pack_bf16(b.x * r.w[1].x, b.y * r.w[1].y);
+                out.w = pack_bf16(b.z * r.w[1].z, b.w * r.w[1].w);
+            }
+            *reinterpret_cast<uint4*>(dst + swz_unit(tok, q)) = out;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 2 * NT; ++i) *reinterpret_cast<uint4*>(dst + (lane + 32 * i) * 16) = r.v[NORM ? 0 : i];
     }
 }
 
 // A bounded wait that ran out marks the warp "dead": it stops touching the pipeline but still
 // walks the control flow, so that every named barrier is reached by all of its threads.
-template <int NT>
-__device__ void loader_phase(const FwdParams& P, int kind, int layer, const Part& pt, uint8_t* smem, Misc* misc,
-                             uint32_t& it, int lw, int lane) {
+template <int NT, bool NORM>
+__device__ __forceinline__ void loader_phase(const FwdParams& P, int kind, int layer, const OpDesc& od, const Part& pt, uint8_t* smem,
+                             Misc* misc, uint32_t& it, uint32_t& ci, int lw, int lane, unsigned long long* prof) {
     using SL = SmemLayout<NT>;
-    const int npass = part_passes(pt);
-    const bool is_norm = (kind == PH_QKV || kind == PH_GU || kind == PH_LM);
+    const int KW = kConsumerWarps / od.RW;
+    const int npass = part_passes(pt, od.RW);
+    const int nst = (pt.nchunks + KW - 1) / KW;
+    const int nchunks = pt.nchunks;
     const float* wn = nullptr;
     if (kind == PH_QKV) wn = P.norm_w + (size_t)(layer * 2 + 0) * P.d;
     if (kind == PH_GU) wn = P.norm_w + (size_t)(layer * 2 + 1) * P.d;
     if (kind == PH_LM) wn = P.norm_w + (size_t)(P.n_layers * 2) * P.d;
+    const uint8_t* src_op = (kind == PH_O) ? P.attn_op : P.act;
     float ss[2 * NT];
 #pragma unroll
     for (int i = 0; i < 2 * NT; ++i) ss[i] = 0.f;
     bool dead = *(volatile int*)&misc->abort_flag != 0;
-    for (int p = 0; p < npass; ++p) {
-        for (int c = 0; c < pt.nchunks; ++c, ++it) {
-            if ((int)(it % kLoaderWarps) != lw) continue;
-            const uint32_t slot = it % SL::NSTAGE, use = it / SL::NSTAGE;
-            if (!dead && use > 0) {
-                const bool got = mbar_wait_bounded(&misc->empty[slot], (use - 1) & 1, &misc->abort_flag, P.wait_limit_ns);
-                if (!__all_sync(0xffffffffu, got)) dead = true;
-            }
-            if (dead) continue;
-            uint8_t* dst = smem + SL::A_OFF + slot * SL::A_STAGE;
-            const int chunk = pt.chunk0 + c;
-            if (is_norm) {
-                load_norm_chunk<NT>(P, wn, chunk * 64, dst, lane, ss, p == 0);
-            } else if (kind == PH_O) {
-                load_combine_chunk<NT>(P, chunk * 64, dst, lane);
-            } else {
-                load_copy_chunk<NT>(P.act + (size_t)chunk * SL::A_STAGE, dst, lane);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&misc->full_a[slot]);
-        }
-        if (p == 0 && is_norm) {
-            // per-row sums of squares of the columns this warp handled
-#pragma unroll
-            for (int i = 0; i < 2 * NT; ++i) {
-                float v = ss[i];
-                v += __shfl_xor_sync(0xffffffffu, v, 1);
-                v += __shfl_xor_sync(0xffffffffu, v, 2);
-                v += __shfl_xor_sync(0xffffffffu, v, 4);
-                const int tok = (lane + 32 * i) >> 3;
-                if ((lane & 7) == 0) {
-                    if (kind == PH_QKV) {
-                        // the attention step normalises q, k, v; only one row partition reports
-                        if (pt.pr == 0 && tok < P.M && !dead) atomicAdd(P.sumsq + (layer & 1) * kMaxRows + tok, v);
-                    } else {
-                        misc->ss_part[lw][tok] = v;
-                    }
-                }
-            }
-            if (kind != PH_QKV) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&misc->rstd_bar);
-            }
-        }
+    const uint32_t it0 = it, ci0 = ci;
+    const int total = npass * nchunks;  // chunk visits of this phase, pass-major
+    // first visit handled by this warp
+    const int x0 = (int)((lw + kLoaderWarps - (ci0 % kLoaderWarps)) % kLoaderWarps);
+
+    // Publish this warp's share of the per-row sums of squares as soon as its first-pass chunks are
+    // done: the MMA warps need them at the end of the first pass, before later passes can drain.
+    bool published = false;
+#define SDV_PUBLISH()                                                                                             \
+    do {                                                                                                          \
+        published = true;                                                                                         \
+        _Pragma("unroll") for (int i = 0; i < 2 * NT; ++i) {                                                      \
+            float v = ss[i];                                                                                      \
+            v += __shfl_xor_sync(0xffffffffu, v, 1);                                                              \
+            v += __shfl_xor_sync(0xffffffffu, v, 2);                                                              \
+            v += __shfl_xor_sync(0xffffffffu, v, 4);                                                              \
+            const int tok = (lane + 32 * i) >> 3;                                                                 \
+            if ((lane & 7) == 0) {                                                                                \
+                if (kind == PH_QKV) {                                                                             \
+                    /* the attention step normalises q, k, v; only one row partition reports */                  \
+                    if (pt.pr == 0 && tok < P.M && !dead) atomicAdd(P.sumsq + (layer & 1) * kMaxRows + tok, v);   \
+                } else {                                                                                          \
+                    misc->ss_part[lw][tok] = v;                                                                   \
+                }                                                                                                 \
+            }                                                                                                     \
+        }                                                                                                         \
+        if (kind != PH_QKV) {                                                                                     \
+            __syncwarp();                                                                                         \
+            if (lane == 0) mbar_arrive(&misc->rstd_bar);                                                          \
+        }                                                                                                         \
+    } while (0)
+
+    if (prof && lw == 0 && lane == 0) prof[6] = global_timer_ns();
+    bool first_done = false;
+    ChunkRegs<NT, NORM> ra, rb;
+    int xa = x0, xb = -1;
+    if (NORM && x0 >= nchunks) SDV_PUBLISH();  // no first-pass chunk falls to this warp
+    if (xa < total && !dead) chunk_issue<NT, NORM>(P, ra, wn, src_op, pt.chunk0 + xa % nchunks, lane);
+    // finish a chunk: wait for its slot, transform + store, signal
+#define SDV_FINISH(REGS, XV)                                                                                      \
+    do {                                                                                                          \
+        const int p_ = (XV) / nchunks, c_ = (XV) % nchunks;                                                       \
+        const uint32_t sidx = it0 + (uint32_t)(p_ * nst + c_ / KW);                                               \
+        const uint32_t slot = sidx % SL::NSTAGE, use = sidx / SL::NSTAGE;                                         \
+        if (!dead && use > 0) {                                                                                   \
+            const bool got =                                                                                      \
+                mbar_wait_bounded(&misc->empty[slot], (use - 1) & 1, &misc->abort_flag, P.wait_limit_ns);         \
+            if (!__all_sync(0xffffffffu, got)) dead = true;                                                       \
+        }                                                                                                         \
+        if (!dead) {                                                                                              \
+            uint8_t* dst = smem + SL::A_OFF + slot * SL::A_STAGE + (c_ % KW) * SL::A_CHUNK;                       \
+            chunk_store<NT, NORM>(P, REGS, dst, lane, ss, p_ == 0);                                               \
+            __syncwarp();                                                                                         \
+            if (lane == 0) {                                                                                      \
+                uint32_t cnt = kMaxKW / KW;                                                                       \
+                if (c_ == nchunks - 1) cnt *= (uint32_t)(KW - (nchunks - 1) % KW); /* ragged last stage */        \
+                mbar_arrive_cnt(&misc->full_a[slot], cnt);                                                        \
+            }                                                                                                     \
+        }                                                                                                         \
+        if (prof && !first_done && lw == 0 && lane == 0) { prof[7] = global_timer_ns(); }                        \
+        first_done = true;                                                                                        \
+        if (NORM && !published && (XV) + kLoaderWarps >= nchunks) SDV_PUBLISH();                                  \
+    } while (0)
+
+    while (xa < total) {
+        xb = xa + kLoaderWarps;
+        if (xb < total && !dead) chunk_issue<NT, NORM>(P, rb, wn, src_op, pt.chunk0 + xb % nchunks, lane);
+        SDV_FINISH(ra, xa);
+        if (xb >= total) break;
+        xa = xb + kLoaderWarps;
+        if (xa < total && !dead) chunk_issue<NT, NORM>(P, ra, wn, src_op, pt.chunk0 + xa % nchunks, lane);
+        SDV_FINISH(rb, xb);
     }
+#undef SDV_FINISH
+
+    if (NORM && !published) SDV_PUBLISH();
+#undef SDV_PUBLISH
+    if (prof && lw == 0 && lane == 0) prof[5] = global_timer_ns();
+    it = it0 + (uint32_t)(npass * nst);
+    ci = ci0 + (uint32_t)total;
 }
 
 // ------------------------------------------------------------------------------------------
 // MMA warps.
 template <int NT>
-__device__ void consumer_phase(const FwdParams& P, int kind, int layer, const Part& pt, uint8_t* smem, Misc* misc,
-                               uint32_t& it, uint32_t& norm_uses, int warp, int lane) {
+__device__ __forceinline__ void consumer_phase(const FwdParams& P, int kind, int layer, const OpDesc& od, const Part& pt, uint8_t* smem,
+                               Misc* misc, uint32_t& it, uint32_t& ci, uint32_t& norm_uses, int warp, int lane,
+                               unsigned long long* prof) {
     using SL = SmemLayout<NT>;
     constexpr int MP = SL::MP;
-    const int npass = part_passes(pt);
+    const int RW = od.RW, KW = kConsumerWarps / RW;
+    const int rw = warp % RW, kw = warp / RW;
+    const int npass = part_passes(pt, RW);
+    const int nst = (pt.nchunks + KW - 1) / KW;
     const int g = lane >> 2, q2 = (lane & 3) * 2;
     const bool need_rstd = (kind == PH_GU || kind == PH_LM);
+    const bool staged = (kind == PH_QKV || kind == PH_O || kind == PH_DOWN || kind == PH_RAW);
     float rstd[NT][2];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) rstd[nt][0] = rstd[nt][1] = 0.f;
@@ -313,16 +351,18 @@ __device__ void consumer_phase(const FwdParams& P, int kind, int layer, const Pa
         bv[nt][0] = bv[nt][1] = -CUDART_INF_F;
         bi[nt][0] = bi[nt][1] = 0x7fffffff;
     }
+    float* red = reinterpret_cast<float*>(smem + SL::ATT_OFF);  // [8 warps][MP][16] partial tiles (staged epilogue)
+    ci += (uint32_t)(npass * pt.nchunks);
 
     for (int p = 0; p < npass; ++p) {
         const int pcount = even_count(pt.ntiles, npass, p);
-        const int tile = pt.tile0 + even_start(pt.ntiles, npass, p) + warp;
-        const bool active = warp < pcount;
+        const int tile_base = pt.tile0 + even_start(pt.ntiles, npass, p);
+        const int tile = tile_base + rw;
         float acc[NT][4];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
 
-        for (int c = 0; c < pt.nchunks; ++c, ++it) {
+        for (int st = 0; st < nst; ++st, ++it) {
             const uint32_t slot = it % SL::NSTAGE, par = (it / SL::NSTAGE) & 1;
             if (!dead) {
                 const bool got = mbar_wait_bounded(&misc->full_w[slot], par, &misc->abort_flag, P.wait_limit_ns) &&
@@ -330,9 +370,12 @@ __device__ void consumer_phase(const FwdParams& P, int kind, int layer, const Pa
                 if (!__all_sync(0xffffffffu, got)) dead = true;
             }
             if (dead) continue;
-            if (active) {
-                const uint32_t wbase = smem_u32(smem + SL::W_OFF + slot * kStageWeightBytes + warp * kTileBytes);
-                const uint32_t abase = smem_u32(smem + SL::A_OFF + slot * SL::A_STAGE);
+            if (prof && p == 0 && st == 0 && warp == 0 && lane == 0) prof[2] = global_timer_ns();
+            const int kcnt = min(KW, pt.nchunks - st * KW);
+            if (rw < pcount && kw < kcnt) {
+                const uint32_t wbase =
+                    smem_u32(smem + SL::W_OFF + slot * kStageWeightBytes + (kw * pcount + rw) * kTileBytes);
+                const uint32_t abase = smem_u32(smem + SL::A_OFF + slot * SL::A_STAGE + kw * SL::A_CHUNK);
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
                     uint32_t a0, a1, a2, a3;
@@ -357,6 +400,7 @@ __device__ void consumer_phase(const FwdParams& P, int kind, int layer, const Pa
             if (lane == 0) mbar_arrive(&misc->empty[slot]);
         }
 
+        if (prof && p == npass - 1 && warp == 0 && lane == 0) prof[3] = global_timer_ns();
         if (need_rstd && !have_rstd && !dead) {
             const bool got = mbar_wait_bounded(&misc->rstd_bar, norm_uses & 1, &misc->abort_flag, P.wait_limit_ns);
             if (!__all_sync(0xffffffffu, got)) dead = true;
@@ -374,29 +418,54 @@ __device__ void consumer_phase(const FwdParams& P, int kind, int layer, const Pa
                 }
             have_rstd = true;
         }
-        if (!active || dead) continue;
 
         // ---------------- epilogues
-        if (kind == PH_QKV || kind == PH_O || kind == PH_DOWN || kind == PH_RAW) {
-            float* out;
-            int stride;
-            if (kind == PH_QKV) { out = P.qkv_acc; stride = P.n_qkv; }
-            else if (kind == PH_RAW) { out = P.raw_out; stride = P.raw_N; }
-            else { out = P.h; stride = P.d; }
-            const int r0 = tile * 16 + g;
+        if (staged) {
+            // partial tiles meet in shared memory: the KW column splits are summed there and each
+            // thread then owns 4 adjacent output rows of one token (one 16-byte global operation)
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const int n = nt * 8 + q2 + e;
-                    if (n < P.M) {
-                        red_add_f32(out + (size_t)n * stride + r0, acc[nt][e]);
-                        red_add_f32(out + (size_t)n * stride + r0 + 8, acc[nt][2 + e]);
+                    red[(warp * MP + n) * 16 + g] = acc[nt][e];
+                    red[(warp * MP + n) * 16 + g + 8] = acc[nt][2 + e];
+                }
+            named_bar_sync(2, kConsumerWarps * 32);
+            if (!dead) {
+                float* out;
+                int stride;
+                if (kind == PH_QKV) { out = P.qkv_acc; stride = P.n_qkv; }
+                else if (kind == PH_RAW) { out = P.raw_out; stride = P.raw_N; }
+                else { out = P.h; stride = P.d; }
+                const int M = P.M, ngroups = pcount * 4 * M;
+                for (int idx = warp * 32 + lane; idx < ngroups; idx += kConsumerWarps * 32) {
+                    const int rwi = idx / (4 * M), rem = idx % (4 * M), n = rem >> 2, r4 = rem & 3;
+                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int kwi = 0; kwi < KW; ++kwi) {
+                        const float4 t =
+                            *reinterpret_cast<const float4*>(red + ((kwi * RW + rwi) * MP + n) * 16 + r4 * 4);
+                        v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+                    }
+                    float* dst = out + (size_t)n * stride + (tile_base + rwi) * 16 + r4 * 4;
+                    if (od.P_k > 1) {
+                        red_add_v4_f32(dst, v);
+                    } else if (kind == PH_QKV || kind == PH_RAW) {
+                        __stcg(reinterpret_cast<float4*>(dst), v);  // sole owner of a zeroed buffer
+                    } else {
+                        const float4 o = ldcg_f4(dst);  // sole owner: residual add in place
+                        __stcg(reinterpret_cast<float4*>(dst), make_float4(o.x + v.x, o.y + v.y, o.z + v.z, o.w + v.w));
                     }
                 }
-        } else if (kind == PH_GU) {
+            }
+            named_bar_sync(2, kConsumerWarps * 32);
+            continue;
+        }
+        if (warp >= pcount || dead) continue;  // RW = 8 here: one tile per warp
+
+        if (kind == PH_GU) {
             const int fi = tile * 8 + g;  // rows 0..7 of the tile are gate rows, 8..15 the matching up rows
-            uint8_t* dst = P.act + (size_t)(fi >> 6) * (MP * 128);
+            uint8_t* dst = P.act + (size_t)(fi >> 6) * SL::A_CHUNK;
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -427,6 +496,7 @@ __device__ void consumer_phase(const FwdParams& P, int kind, int layer, const Pa
                 }
         }
     }
+    if (prof && warp == 0 && lane == 0) prof[4] = global_timer_ns();
     if (need_rstd) ++norm_uses;
 
     if (kind == PH_LM) {
@@ -465,15 +535,26 @@ __device__ void consumer_phase(const FwdParams& P, int kind, int layer, const Pa
 }
 
 // ------------------------------------------------------------------------------------------
-// Attention over one (KV head, key range) unit for all query rows of the head group.
-// Unit s < S covers cache keys [s*kps, min(L, (s+1)*kps)); unit s == S covers the M new rows:
-// it finishes their K/V projection (norm scale, bias, rotary), appends them to the cache and
-// attends to them under the causal mask (row j sees new keys 0..j).
+// Split-KV attention.  The committed cache [0, L) is cut into S key ranges of kps keys (a multiple
+// of 64, as many ranges as there are blocks to take them); unit (kv head, s < S) attends all
+// query rows of the head group to range s; unit (kv head, S) covers the M new rows: it finishes
+// their K/V projection (norm scale, bias, rotary), appends them to the cache and attends to them
+// under the causal mask (row j sees new keys 0..j).  Partial results are merged afterwards.
+__device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps) {
+    if (P.L <= 0) { S = 0; kps = 0; return; }
+    int cap = P.G / P.n_kv - 1;
+    if (cap > kMaxSplits) cap = kMaxSplits;
+    if (cap < 1) cap = 1;
+    kps = ((P.L + cap - 1) / cap + 63) / 64 * 64;
+    S = (P.L + kps - 1) / kps;
+}
+
 template <int HD>
-__device__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int S, int kps, uint8_t* att, int wtid) {
+__device__ __forceinline__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int S, int kps, uint8_t* att, int wtid) {
     constexpr int HD2 = HD / 2;
     constexpr int KSTEPS = HD / 16;
     constexpr int UNITS = HD / 8;  // 16-byte units per K/V row
+    constexpr int UPT = (kAttnBlockKeys * UNITS + kWorkerThreads - 1) / kWorkerThreads;  // units per thread
     const int warp = wtid >> 5, lane = wtid & 31;
     const int M = P.M, L = P.L, R = P.g * M;
     const int MT = (R + 15) >> 4, RP = MT * 16;
@@ -485,25 +566,6 @@ __device__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int
     const float* bias = P.bias ? P.bias + (size_t)layer * P.n_qkv : nullptr;
     const int Nq = P.n_q * HD, Nkv = P.n_kv * HD;
 
-    // ---- query tile: normalise, add bias, rotate, round to bf16
-    for (int idx = wtid; idx < RP * HD2; idx += kWorkerThreads) {
-        const int r = idx / HD2, i = idx % HD2;
-        float q0 = 0.f, q1 = 0.f;
-        if (r < R) {
-            const int hl = r / M, j = r % M, col = (hk * P.g + hl) * HD + i;
-            const float rs = rsqrtf(__ldcg(sumsq + j) / (float)P.d + P.eps);
-            float a = rs * __ldcg(P.qkv_acc + (size_t)j * P.n_qkv + col);
-            float b = rs * __ldcg(P.qkv_acc + (size_t)j * P.n_qkv + col + HD2);
-            if (bias) { a += bias[col]; b += bias[col + HD2]; }
-            const float2 cs = __ldg(P.rope + (size_t)(L + j) * HD2 + i);
-            q0 = a * cs.x - b * cs.y;
-            q1 = b * cs.x + a * cs.y;
-        }
-        const int c0 = i, c1 = i + HD2;
-        *reinterpret_cast<__nv_bfloat16*>(Qs + (c0 >> 6) * (RP * 128) + swz_off(r, c0 & 63)) = __float2bfloat16(q0);
-        *reinterpret_cast<__nv_bfloat16*>(Qs + (c1 >> 6) * (RP * 128) + swz_off(r, c1 & 63)) = __float2bfloat16(q1);
-    }
-
     int t_begin = 0, nkeys = M;
     if (!is_new) {
         t_begin = s * kps;
@@ -512,6 +574,89 @@ __device__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int
     }
     const int nblk = (nkeys + kAttnBlockKeys - 1) / kAttnBlockKeys;
     const size_t cache_row0 = ((size_t)layer * P.n_kv + hk) * P.max_seq;
+
+    // ---- cached keys: the first block's loads are in flight while the query tile is built
+    uint4 kreg[UPT], vreg[UPT];
+    auto issue_block = [&](int blk) {
+#pragma unroll
+        for (int t = 0; t < UPT; ++t) {
+            const int u = wtid + t * kWorkerThreads;
+            const int key = u / UNITS, q16 = u % UNITS, kk = blk * kAttnBlockKeys + key;
+            kreg[t] = make_uint4(0, 0, 0, 0);
+            vreg[t] = make_uint4(0, 0, 0, 0);
+            if (u < kAttnBlockKeys * UNITS && kk < nkeys) {
+                const size_t off = (cache_row0 + t_begin + kk) * HD + q16 * 8;
+                kreg[t] = ldcg_u4(P.kcache + off);
+                vreg[t] = ldcg_u4(P.vcache + off);
+            }
+        }
+    };
+    auto store_block = [&]() {
+#pragma unroll
+        for (int t = 0; t < UPT; ++t) {
+            const int u = wtid + t * kWorkerThreads;
+            if (u < kAttnBlockKeys * UNITS) {
+                const int key = u / UNITS, q16 = u % UNITS;
+                const uint32_t so = (q16 >> 3) * (kAttnBlockKeys * 128) + swz_unit(key, q16 & 7);
+                *reinterpret_cast<uint4*>(Ks + so) = kreg[t];
+                *reinterpret_cast<uint4*>(Vs + so) = vreg[t];
+            }
+        }
+    };
+    if (!is_new && nblk > 0) issue_block(0);
+
+    // ---- query tile: normalise, add bias, rotate, round to bf16; 4 rotary pairs per item
+    {
+        const int items = RP * (HD2 / 4);
+        for (int base = wtid; base < items; base += 2 * kWorkerThreads) {
+            float4 qa[2], qb[2], c0[2], c1[2];
+            float ssq[2];
+            int rr[2], ii[2];
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const int idx = base + t * kWorkerThreads;
+                rr[t] = idx / (HD2 / 4);
+                ii[t] = (idx % (HD2 / 4)) * 4;
+                ssq[t] = 0.f;
+                qa[t] = qb[t] = c0[t] = c1[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (idx < items && rr[t] < R) {
+                    const int hl = rr[t] / M, j = rr[t] % M, col = (hk * P.g + hl) * HD + ii[t];
+                    ssq[t] = __ldcg(sumsq + j);
+                    qa[t] = ldcg_f4(P.qkv_acc + (size_t)j * P.n_qkv + col);
+                    qb[t] = ldcg_f4(P.qkv_acc + (size_t)j * P.n_qkv + col + HD2);
+                    const float4* rp = reinterpret_cast<const float4*>(P.rope + (size_t)(L + j) * HD2 + ii[t]);
+                    c0[t] = __ldg(rp);
+                    c1[t] = __ldg(rp + 1);
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const int idx = base + t * kWorkerThreads;
+                if (idx >= items) continue;
+                const int r = rr[t], i = ii[t];
+                uint2 lo = make_uint2(0, 0), hi = make_uint2(0, 0);
+                if (r < R) {
+                    const float rs = rsqrtf(ssq[t] / (float)P.d + P.eps);
+                    float a[4] = {qa[t].x * rs, qa[t].y * rs, qa[t].z * rs, qa[t].w * rs};
+                    float b[4] = {qb[t].x * rs, qb[t].y * rs, qb[t].z * rs, qb[t].w * rs};
+                    if (bias) {
+                        const int col = (hk * P.g + r / M) * HD + i;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) { a[e] += bias[col + e]; b[e] += bias[col + HD2 + e]; }
+                    }
+                    const float cs[4] = {c0[t].x, c0[t].z, c1[t].x, c1[t].z}, sn[4] = {c0[t].y, c0[t].w, c1[t].y, c1[t].w};
+                    float x0[4], x1[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) { x0[e] = a[e] * cs[e] - b[e] * sn[e]; x1[e] = b[e] * cs[e] + a[e] * sn[e]; }
+                    lo = make_uint2(pack_bf16(x0[0], x0[1]), pack_bf16(x0[2], x0[3]));
+                    hi = make_uint2(pack_bf16(x1[0], x1[1]), pack_bf16(x1[2], x1[3]));
+                }
+                const int cA = i, cB = i + HD2;
+                *reinterpret_cast<uint2*>(Qs + (cA >> 6) * (RP * 128) + swz_off(r, cA & 63)) = lo;
+                *reinterpret_cast<uint2*>(Qs + (cB >> 6) * (RP * 128) + swz_off(r, cB & 63)) = hi;
+            }
+        }
+    }
 
     const int g = lane >> 2, q2 = (lane & 3) * 2;
     const int r_lo = warp * 16 + g, r_hi = r_lo + 8;
@@ -522,112 +667,124 @@ __device__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int
     for (int n = 0; n < HD / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
 
     for (int blk = 0; blk < nblk; ++blk) {
-        named_bar_sync(1, kWorkerThreads);  // previous block consumed (and, first time, Q tile written)
-        for (int u = wtid; u < kAttnBlockKeys * UNITS; u += kWorkerThreads) {
-            const int key = u / UNITS, q16 = u % UNITS, kk = blk * kAttnBlockKeys + key;
-            uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
-            if (kk < nkeys) {
-                if (is_new) {
+        if (is_new) {
+            // K and V rows of the new tokens: finish the projection, rotate K, append to the cache
+            for (int u = wtid; u < kAttnBlockKeys * UNITS; u += kWorkerThreads) {
+                const int key = u / UNITS, q16 = u % UNITS, kk = blk * kAttnBlockKeys + key;
+                uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
+                if (kk < nkeys) {
                     const float rs = rsqrtf(__ldcg(sumsq + kk) / (float)P.d + P.eps);
                     const float* accrow = P.qkv_acc + (size_t)kk * P.n_qkv;
-                    float kvals[8], vvals[8];
+                    const int colb = q16 * 8, ib = colb % HD2;  // 8 columns share one half of the rotary pairing
+                    const float* pa = accrow + Nq + hk * HD + ib;
+                    const float4 a0 = ldcg_f4(pa), a1 = ldcg_f4(pa + 4), b0 = ldcg_f4(pa + HD2), b1 = ldcg_f4(pa + HD2 + 4);
+                    const float* pv = accrow + Nq + Nkv + hk * HD + colb;
+                    const float4 v0 = ldcg_f4(pv), v1 = ldcg_f4(pv + 4);
+                    const float4* rp = reinterpret_cast<const float4*>(P.rope + (size_t)(L + kk) * HD2 + ib);
+                    const float4 r0 = __ldg(rp), r1 = __ldg(rp + 1), r2 = __ldg(rp + 2), r3 = __ldg(rp + 3);
+                    float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                    float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                    float v[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+                    const float cs[8] = {r0.x, r0.z, r1.x, r1.z, r2.x, r2.z, r3.x, r3.z};
+                    const float sn[8] = {r0.y, r0.w, r1.y, r1.w, r2.y, r2.w, r3.y, r3.w};
+                    float kvals[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
-                        const int col = q16 * 8 + e, i = col % HD2;
-                        const int ka = Nq + hk * HD + i, kb = ka + HD2, vc = Nq + Nkv + hk * HD + col;
-                        float a = rs * __ldcg(accrow + ka), b = rs * __ldcg(accrow + kb), v = rs * __ldcg(accrow + vc);
-                        if (bias) { a += bias[ka]; b += bias[kb]; v += bias[vc]; }
-                        const float2 cs = __ldg(P.rope + (size_t)(L + kk) * HD2 + i);
-                        kvals[e] = (col < HD2) ? (a * cs.x - b * cs.y) : (b * cs.x + a * cs.y);
-                        vvals[e] = v;
+                        a[e] *= rs; b[e] *= rs; v[e] *= rs;
+                        if (bias) {
+                            a[e] += bias[Nq + hk * HD + ib + e];
+                            b[e] += bias[Nq + hk * HD + ib + HD2 + e];
+                            v[e] += bias[Nq + Nkv + hk * HD + colb + e];
+                        }
+                        kvals[e] = (colb < HD2) ? (a[e] * cs[e] - b[e] * sn[e]) : (b[e] * cs[e] + a[e] * sn[e]);
                     }
                     kv4 = make_uint4(pack_bf16(kvals[0], kvals[1]), pack_bf16(kvals[2], kvals[3]),
                                      pack_bf16(kvals[4], kvals[5]), pack_bf16(kvals[6], kvals[7]));
-                    vv4 = make_uint4(pack_bf16(vvals[0], vvals[1]), pack_bf16(vvals[2], vvals[3]),
-                                     pack_bf16(vvals[4], vvals[5]), pack_bf16(vvals[6], vvals[7]));
+                    vv4 = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]),
+                                     pack_bf16(v[6], v[7]));
                     const size_t off = (cache_row0 + L + kk) * HD + q16 * 8;
                     *reinterpret_cast<uint4*>(P.kcache + off) = kv4;
                     *reinterpret_cast<uint4*>(P.vcache + off) = vv4;
-                } else {
-                    const size_t off = (cache_row0 + t_begin + kk) * HD + q16 * 8;
-                    kv4 = ldcg_u4(P.kcache + off);
-                    vv4 = ldcg_u4(P.vcache + off);
+                }
+                const uint32_t so = (q16 >> 3) * (kAttnBlockKeys * 128) + swz_unit(key, q16 & 7);
+                *reinterpret_cast<uint4*>(Ks + so) = kv4;
+                *reinterpret_cast<uint4*>(Vs + so) = vv4;
+            }
+        } else {
+            store_block();
+        }
+        named_bar_sync(1, kWorkerThreads);  // K/V block (and, first time, the Q tile) are in place
+        if (!is_new && blk + 1 < nblk) issue_block(blk + 1);
+        if (warp < MT) {
+            // ---- S = Q K^T for 16 rows x 32 keys
+            float sc[4][4];
+#pragma unroll
+            for (int n = 0; n < 4; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
+            const uint32_t qb = smem_u32(Qs), kb = smem_u32(Ks), vb = smem_u32(Vs);
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+                uint32_t a0, a1, a2, a3;
+                ldsm_x4(qb + (ks >> 2) * (RP * 128) + swz_unit(warp * 16 + (lane & 15), (ks & 3) * 2 + (lane >> 4)), a0,
+                        a1, a2, a3);
+#pragma unroll
+                for (int np = 0; np < 2; ++np) {
+                    uint32_t b0, b1, b2, b3;
+                    const int row = np * 16 + (lane & 7) + ((lane >> 4) << 3);
+                    ldsm_x4(kb + (ks >> 2) * (kAttnBlockKeys * 128) + swz_unit(row, (ks & 3) * 2 + ((lane >> 3) & 1)), b0,
+                            b1, b2, b3);
+                    mma_bf16_16816(sc[2 * np], a0, a1, a2, a3, b0, b1);
+                    mma_bf16_16816(sc[2 * np + 1], a0, a1, a2, a3, b2, b3);
                 }
             }
-            const uint32_t so = (q16 >> 3) * (kAttnBlockKeys * 128) + swz_unit(key, q16 & 7);
-            *reinterpret_cast<uint4*>(Ks + so) = kv4;
-            *reinterpret_cast<uint4*>(Vs + so) = vv4;
-        }
-        named_bar_sync(1, kWorkerThreads);
-        if (warp >= MT) continue;
-
-        // ---- S = Q K^T for 16 rows x 32 keys
-        float sc[4][4];
+            // ---- mask, online softmax (log2 domain)
+            float mx_lo = -CUDART_INF_F, mx_hi = -CUDART_INF_F;
 #pragma unroll
-        for (int n = 0; n < 4; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
-        const uint32_t qb = smem_u32(Qs), kb = smem_u32(Ks), vb = smem_u32(Vs);
+            for (int n = 0; n < 4; ++n)
 #pragma unroll
-        for (int ks = 0; ks < KSTEPS; ++ks) {
-            uint32_t a0, a1, a2, a3;
-            ldsm_x4(qb + (ks >> 2) * (RP * 128) + swz_unit(warp * 16 + (lane & 15), (ks & 3) * 2 + (lane >> 4)), a0, a1,
-                    a2, a3);
+                for (int e = 0; e < 4; ++e) {
+                    const int key = blk * kAttnBlockKeys + n * 8 + q2 + (e & 1);
+                    const bool hi = e >= 2;
+                    const int row = hi ? r_hi : r_lo, j = hi ? j_hi : j_lo;
+                    const bool ok = key < nkeys && row < R && (!is_new || key <= j);
+                    const float v = ok ? sc[n][e] * P.scale_log2e : -CUDART_INF_F;
+                    sc[n][e] = v;
+                    if (hi) mx_hi = fmaxf(mx_hi, v); else mx_lo = fmaxf(mx_lo, v);
+                }
+            mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+            mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+            mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+            mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+            const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+            const float use_lo = (mn_lo == -CUDART_INF_F) ? 0.f : mn_lo, use_hi = (mn_hi == -CUDART_INF_F) ? 0.f : mn_hi;
+            const float corr_lo = exp2f(m_lo - use_lo), corr_hi = exp2f(m_hi - use_hi);
+            m_lo = mn_lo; m_hi = mn_hi;
+            l_lo *= corr_lo; l_hi *= corr_hi;
 #pragma unroll
-            for (int np = 0; np < 2; ++np) {
-                uint32_t b0, b1, b2, b3;
-                const int row = np * 16 + (lane & 7) + ((lane >> 4) << 3);
-                ldsm_x4(kb + (ks >> 2) * (kAttnBlockKeys * 128) + swz_unit(row, (ks & 3) * 2 + ((lane >> 3) & 1)), b0, b1,
-                        b2, b3);
-                mma_bf16_16816(sc[2 * np], a0, a1, a2, a3, b0, b1);
-                mma_bf16_16816(sc[2 * np + 1], a0, a1, a2, a3, b2, b3);
+            for (int n = 0; n < HD / 8; ++n) { o[n][0] *= corr_lo; o[n][1] *= corr_lo; o[n][2] *= corr_hi; o[n][3] *= corr_hi; }
+            uint32_t pa[2][4];
+#pragma unroll
+            for (int n = 0; n < 4; ++n) {
+                const float p0 = exp2f(sc[n][0] - use_lo), p1 = exp2f(sc[n][1] - use_lo);
+                const float p2 = exp2f(sc[n][2] - use_hi), p3 = exp2f(sc[n][3] - use_hi);
+                l_lo += p0 + p1; l_hi += p2 + p3;
+                pa[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
+                pa[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
+            }
+            // ---- O += P V
+#pragma unroll
+            for (int kk2 = 0; kk2 < 2; ++kk2) {
+#pragma unroll
+                for (int np = 0; np < HD / 16; ++np) {
+                    uint32_t b0, b1, b2, b3;
+                    const int key = kk2 * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+                    const int cu = np * 2 + (lane >> 4);
+                    ldsm_x4_trans(vb + (cu >> 3) * (kAttnBlockKeys * 128) + swz_unit(key, cu & 7), b0, b1, b2, b3);
+                    mma_bf16_16816(o[2 * np], pa[kk2][0], pa[kk2][1], pa[kk2][2], pa[kk2][3], b0, b1);
+                    mma_bf16_16816(o[2 * np + 1], pa[kk2][0], pa[kk2][1], pa[kk2][2], pa[kk2][3], b2, b3);
+                }
             }
         }
-        // ---- mask, online softmax (log2 domain)
-        float mx_lo = -CUDART_INF_F, mx_hi = -CUDART_INF_F;
-#pragma unroll
-        for (int n = 0; n < 4; ++n)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int key = blk * kAttnBlockKeys + n * 8 + q2 + (e & 1);
-                const bool hi = e >= 2;
-                const int row = hi ? r_hi : r_lo, j = hi ? j_hi : j_lo;
-                const bool ok = key < nkeys && row < R && (!is_new || key <= j);
-                const float v = ok ? sc[n][e] * P.scale_log2e : -CUDART_INF_F;
-                sc[n][e] = v;
-                if (hi) mx_hi = fmaxf(mx_hi, v); else mx_lo = fmaxf(mx_lo, v);
-            }
-        mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
-        mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
-        mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
-        mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
-        const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
-        const float use_lo = (mn_lo == -CUDART_INF_F) ? 0.f : mn_lo, use_hi = (mn_hi == -CUDART_INF_F) ? 0.f : mn_hi;
-        const float corr_lo = exp2f(m_lo - use_lo), corr_hi = exp2f(m_hi - use_hi);
-        m_lo = mn_lo; m_hi = mn_hi;
-        l_lo *= corr_lo; l_hi *= corr_hi;
-#pragma unroll
-        for (int n = 0; n < HD / 8; ++n) { o[n][0] *= corr_lo; o[n][1] *= corr_lo; o[n][2] *= corr_hi; o[n][3] *= corr_hi; }
-        uint32_t pa[2][4];
-#pragma unroll
-        for (int n = 0; n < 4; ++n) {
-            const float p0 = exp2f(sc[n][0] - use_lo), p1 = exp2f(sc[n][1] - use_lo);
-            const float p2 = exp2f(sc[n][2] - use_hi), p3 = exp2f(sc[n][3] - use_hi);
-            l_lo += p0 + p1; l_hi += p2 + p3;
-            pa[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
-            pa[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
-        }
-        // ---- O += P V
-#pragma unroll
-        for (int kk2 = 0; kk2 < 2; ++kk2) {
-#pragma unroll
-            for (int np = 0; np < HD / 16; ++np) {
-                uint32_t b0, b1, b2, b3;
-                const int key = kk2 * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
-                const int cu = np * 2 + (lane >> 4);
-                ldsm_x4_trans(vb + (cu >> 3) * (kAttnBlockKeys * 128) + swz_unit(key, cu & 7), b0, b1, b2, b3);
-                mma_bf16_16816(o[2 * np], pa[kk2][0], pa[kk2][1], pa[kk2][2], pa[kk2][3], b0, b1);
-                mma_bf16_16816(o[2 * np + 1], pa[kk2][0], pa[kk2][1], pa[kk2][2], pa[kk2][3], b2, b3);
-            }
-        }
+        named_bar_sync(1, kWorkerThreads);  // the block has been consumed
     }
 
     // ---- un-normalised partial result of this key range
@@ -653,14 +810,67 @@ __device__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int
 }
 
 __device__ void attention_phase(const FwdParams& P, int layer, uint8_t* att, int wtid) {
-    const int S = attn_splits(P.L), S1 = S + 1;
-    const int kps = S ? attn_keys_per_split(P.L, S) : 0;
+    int S, kps;
+    attn_split(P, S, kps);
+    const int S1 = S + 1;
     const int nunits = P.n_kv * S1;
     for (int unit = blockIdx.x; unit < nunits; unit += P.G) {
         const int hk = unit / S1, s = unit % S1;
         if (P.hd == 128) attention_unit<128>(P, layer, hk, s, S, kps, att, wtid);
         else attention_unit<64>(P, layer, hk, s, S, kps, att, wtid);
         named_bar_sync(1, kWorkerThreads);  // the unit's shared-memory tiles are free again
+    }
+}
+
+// Merge of the split-KV partial results into the output projection's bf16 operand.  One warp per
+// (query head, row, 8 columns); lanes run over the splits.
+template <int NT>
+__device__ __forceinline__ void combine_phase(const FwdParams& P, int wtid) {
+    constexpr int A_CHUNK = SmemLayout<NT>::A_CHUNK;
+    int S, kps;
+    attn_split(P, S, kps);
+    const int S1 = S + 1;
+    const int warp = wtid >> 5, lane = wtid & 31;
+    const int U8 = P.hd / 8, nwarps = kWorkerThreads / 32;
+    const int items = P.n_q * P.M * U8;
+    for (int item = blockIdx.x * nwarps + warp; item < items; item += P.G * nwarps) {
+        const int hq = item / (P.M * U8), j = (item / U8) % P.M, c8 = item % U8;
+        const size_t base = ((size_t)hq * (kMaxSplits + 1)) * kMaxRows + j;
+        float m[2], l[2];
+        float4 a[2], b[2];
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const int s = lane + 32 * t;
+            m[t] = -CUDART_INF_F; l[t] = 0.f;
+            a[t] = b[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (s < S1) {
+                const size_t row = base + (size_t)s * kMaxRows;
+                const float2 ml = __ldcg(reinterpret_cast<const float2*>(P.part_ml + row * 2));
+                m[t] = ml.x; l[t] = ml.y;
+                const float* op = P.part_o + row * P.hd + c8 * 8;
+                a[t] = ldcg_f4(op);
+                b[t] = ldcg_f4(op + 4);
+            }
+        }
+        float mmax = fmaxf(m[0], m[1]);
+#pragma unroll
+        for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
+        const float w0 = exp2f(m[0] - mmax), w1 = exp2f(m[1] - mmax);  // 0 for splits that saw no key
+        float v[9];
+        v[0] = w0 * a[0].x + w1 * a[1].x; v[1] = w0 * a[0].y + w1 * a[1].y; v[2] = w0 * a[0].z + w1 * a[1].z;
+        v[3] = w0 * a[0].w + w1 * a[1].w; v[4] = w0 * b[0].x + w1 * b[1].x; v[5] = w0 * b[0].y + w1 * b[1].y;
+        v[6] = w0 * b[0].z + w1 * b[1].z; v[7] = w0 * b[0].w + w1 * b[1].w; v[8] = w0 * l[0] + w1 * l[1];
+#pragma unroll
+        for (int e = 0; e < 9; ++e)
+#pragma unroll
+            for (int off = 16; off; off >>= 1) v[e] += __shfl_xor_sync(0xffffffffu, v[e], off);
+        if (lane == 0) {
+            const float inv = 1.f / v[8];
+            const int col = hq * P.hd + c8 * 8;
+            const uint4 out = make_uint4(pack_bf16(v[0] * inv, v[1] * inv), pack_bf16(v[2] * inv, v[3] * inv),
+                                         pack_bf16(v[4] * inv, v[5] * inv), pack_bf16(v[6] * inv, v[7] * inv));
+            *reinterpret_cast<uint4*>(P.attn_op + (size_t)(col >> 6) * A_CHUNK + swz_unit(j, (col & 63) >> 3)) = out;
+        }
     }
 }
 
@@ -701,6 +911,7 @@ template <int NT>
 __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_constant__ FwdParams P) {
     using SL = SmemLayout<NT>;
     static_assert(SL::NSTAGE >= 4 && SL::NSTAGE <= 16, "ring depth");
+    static_assert(kConsumerWarps * SL::MP * 16 * 4 <= kAttnSmemBytes, "staged epilogue buffer");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     Misc* misc = reinterpret_cast<Misc*>(smem + SL::MISC_OFF);
@@ -709,7 +920,7 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
     if (tid == 0) {
         for (int s = 0; s < SL::NSTAGE; ++s) {
             mbar_init(&misc->full_w[s], 1);
-            mbar_init(&misc->full_a[s], 1);
+            mbar_init(&misc->full_a[s], kMaxKW);
             mbar_init(&misc->empty[s], kConsumerWarps);
         }
         mbar_init(&misc->rstd_bar, kLoaderWarps);
@@ -725,12 +936,13 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
     }
 
     const int wtid = tid;  // 0 .. kWorkerThreads-1
-    uint32_t it = 0, norm_uses = 0;
+    uint32_t it = 0, ci = 0, norm_uses = 0;
     int nbar = 0;
     bool skip = false;
     for (int ph = P.ph_begin; ph < P.ph_end; ++ph) {
         int layer;
         const int kind = decode_phase(ph, P.n_layers, layer);
+        if (P.prof && wtid == 0) P.prof[((size_t)(ph - P.ph_begin) * P.G + blockIdx.x) * kProfWords] = global_timer_ns();
         // after an abandoned wait the remaining phases do no work but still meet at every barrier
         if (skip) {
         } else if (kind == PH_EMBED) {
@@ -738,13 +950,27 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
             zero_qkv_acc(P, 0, wtid);
         } else if (kind == PH_ATTN) {
             attention_phase(P, layer, smem + SL::ATT_OFF, wtid);
+        } else if (kind == PH_COMB) {
+            combine_phase<NT>(P, wtid);
         } else {
             if (kind == PH_O) zero_qkv_acc(P, (layer + 1) & 1, wtid);
-            const Part pt = get_part(P.op[phase_op(kind)], blockIdx.x, P.G);
+            const OpDesc& od = P.op[phase_op(kind)];
+            const Part pt = get_part(od, blockIdx.x, P.G);
             if (pt.ntiles > 0) {
-                if (warp < kConsumerWarps) consumer_phase<NT>(P, kind, layer, pt, smem, misc, it, norm_uses, warp, lane);
-                else loader_phase<NT>(P, kind, layer, pt, smem, misc, it, warp - kConsumerWarps, lane);
+                unsigned long long* pp =
+                    P.prof ? P.prof + ((size_t)(ph - P.ph_begin) * P.G + blockIdx.x) * kProfWords : nullptr;
+                if (warp < kConsumerWarps) {
+                    consumer_phase<NT>(P, kind, layer, od, pt, smem, misc, it, ci, norm_uses, warp, lane, pp);
+                } else {
+                    const bool norm = (kind == PH_QKV || kind == PH_GU || kind == PH_LM);
+                    if (norm) loader_phase<NT, true>(P, kind, layer, od, pt, smem, misc, it, ci, warp - kConsumerWarps, lane, pp);
+                    else loader_phase<NT, false>(P, kind, layer, od, pt, smem, misc, it, ci, warp - kConsumerWarps, lane, pp);
+                }
             }
+        }
+        if (P.prof) {
+            named_bar_sync(1, kWorkerThreads);
+            if (wtid == 0) P.prof[((size_t)(ph - P.ph_begin) * P.G + blockIdx.x) * kProfWords + 1] = global_timer_ns();
         }
         if (ph + 1 < P.ph_end) {
             ++nbar;

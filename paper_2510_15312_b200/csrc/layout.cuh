@@ -3,10 +3,11 @@
 // Weight streaming layout.  Every linear layer W[N][K] (bf16) is cut into tiles of 16 rows x 64
 // columns (2 KB, 128-byte rows with XOR-swizzled 16-byte units).  An operation's tile grid
 // (T = N/16 row tiles, C = K/64 column chunks) is split into P_row x P_k rectangular
-// partitions, one per thread block; a block walks its partition in passes of at most 8 row
-// tiles (one per MMA warp) and, inside a pass, chunk by chunk.  Tiles are stored in exactly that
-// order, so every pipeline stage (<= 8 tiles of one chunk = <= 16 KB) is one contiguous bulk
-// copy and a block's whole share of an operation is one contiguous byte range.
+// partitions, one per thread block.  The block's 8 MMA warps form an RW x KW grid (RW * KW = 8):
+// it walks its partition in passes of at most RW row tiles and, inside a pass, in stages of KW
+// consecutive chunks, so one stage is RW x KW tiles (<= 16 KB), one per warp.  Tiles are stored
+// pass by pass, chunk by chunk, tile by tile: every stage is one contiguous bulk copy and a
+// block's whole share of an operation is one contiguous byte range.
 #pragma once
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -20,13 +21,14 @@ constexpr int kThreads = kWorkerThreads + 32;                        // 384 with
 constexpr int kTileBytes = 2048;                                     // 16 rows x 64 cols bf16
 constexpr int kStageWeightBytes = kConsumerWarps * kTileBytes;       // 16 KB
 constexpr int kMaxRows = 32;                                         // token rows a buffer is sized for
-constexpr int kMaxSplits = 12;                                       // KV splits per head (+1 unit for new rows)
-constexpr int kSplitTargetKeys = 256;
+constexpr int kMaxSplits = 40;                                       // KV splits per head (+1 unit for new rows)
+constexpr int kMaxKW = 4;                                             // chunks per stage at most
 constexpr int kAttnBlockKeys = 32;
 constexpr int kSmemBudget = 232448;                                  // 227 KB
 constexpr int kAttnSmemBytes = 32768 + 2 * 8192;                     // Q tile (128 x 128) + K and V blocks
 constexpr int kMiscSmemBytes = 4096;
 constexpr int kMaxDraftWords = 32;
+constexpr int kProfWords = 8;                                        // timestamps per (phase, block)
 
 enum OpIndex { OP_QKV = 0, OP_O = 1, OP_GU = 2, OP_DOWN = 3, OP_LM = 4, OP_RAW = 5, OP_COUNT = 6 };
 
@@ -36,7 +38,7 @@ struct OpDesc {
     int P_row;   // partitions along rows
     int P_k;     // partitions along columns (> 1: partial sums meet by atomic adds)
     int rot;     // block index that owns partition 0 (spreads idle blocks over operations)
-    int pad;
+    int RW;      // row tiles per pass (8, 4 or 2); KW = 8 / RW chunks per stage
     unsigned long long w_off;  // byte offset of the operation inside its weight region
 };
 
@@ -78,14 +80,14 @@ __host__ __device__ inline Part get_part(const OpDesc& o, int cta, int G) {
             ((unsigned long long)p.tile0 * o.C + (unsigned long long)p.ntiles * p.chunk0);
     return p;
 }
-__host__ __device__ inline int part_passes(const Part& p) { return (p.ntiles + kConsumerWarps - 1) / kConsumerWarps; }
+__host__ __device__ inline int part_passes(const Part& p, int RW) { return (p.ntiles + RW - 1) / RW; }
 
 // Byte offset (from the operation's base) of tile t, chunk c: the inverse view used when packing.
 __host__ __device__ inline unsigned long long tile_offset(const OpDesc& o, int t, int c) {
     const int pr = even_find(o.T, o.P_row, t), pk = even_find(o.C, o.P_k, c);
     const int tile0 = even_start(o.T, o.P_row, pr), ntiles = even_count(o.T, o.P_row, pr);
     const int chunk0 = even_start(o.C, o.P_k, pk), nchunks = even_count(o.C, o.P_k, pk);
-    const int npass = (ntiles + kConsumerWarps - 1) / kConsumerWarps;
+    const int npass = (ntiles + o.RW - 1) / o.RW;
     const int lt = t - tile0;
     const int p = even_find(ntiles, npass, lt);
     const int start = even_start(ntiles, npass, p), cnt = even_count(ntiles, npass, p);
@@ -127,6 +129,7 @@ struct FwdParams {
     float* qkv_acc;    // [kMaxRows][n_qkv] un-normalised q|k|v sums
     float* sumsq;      // [2][kMaxRows] sum of squares of h rows for the attention-side norm
     uint8_t* act;      // bf16 [f/64][rows][64] swizzled: SwiGLU output, the down projection's operand
+    uint8_t* attn_op;  // bf16 [n_q*hd/64][rows][64] swizzled: attention output, the o projection's operand
     float* part_o;     // [n_q][kMaxSplits+1][kMaxRows][hd] un-normalised split outputs
     float* part_ml;    // [n_q][kMaxSplits+1][kMaxRows][2]  (running max in log2 units, sum)
     float* cand_val;   // [G][kMaxRows] per-block best logit
@@ -137,6 +140,7 @@ struct FwdParams {
     int* state;
     const int* hist;
     int* bar;          // grid barrier counter
+    unsigned long long* prof;  // optional [phase][block][kProfWords] timestamps (ns)
     // per launch
     int L;             // committed KV length = position of row 0
     int M;             // rows computed (1..8*NT)
@@ -144,6 +148,7 @@ struct FwdParams {
     int ph_begin, ph_end;
     int bar_base;      // barrier counter value before this launch
     int store_logits;
+    int ahead;         // weight stages the streamer may run ahead of the MMA warps (<= ring size)
     unsigned long long wait_limit_ns;
 };
 

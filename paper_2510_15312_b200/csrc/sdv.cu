@@ -23,7 +23,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Regions {
     size_t state, bar, never, hist, rope, norm_w, bias, wlayers, wlm, emb, kcache, vcache, h, qkv_acc, sumsq, act,
-        part_o, part_ml, cand_val, cand_idx, logits, raw_out, staging, wraw, xstage, total;
+        attn_op, part_o, part_ml, cand_val, cand_idx, logits, raw_out, staging, wraw, xstage, prof, total;
     size_t layer_stride, staging_bytes, act_k;
 };
 
@@ -78,6 +78,7 @@ Regions carve(const sdv_config* c) {
     if (nq > act_k) act_k = nq;
     r.act_k = act_k;
     r.act = take(act_k / 64 * kMaxRows * 128);
+    r.attn_op = take(nq / 64 * kMaxRows * 128);
     r.part_o = take((size_t)c->n_q_heads * (kMaxSplits + 1) * kMaxRows * hd * 4);
     r.part_ml = take((size_t)c->n_q_heads * (kMaxSplits + 1) * kMaxRows * 2 * 4);
     r.cand_val = take((size_t)kMaxGrid * kMaxRows * 4);
@@ -92,33 +93,42 @@ Regions carve(const sdv_config* c) {
     r.wraw = take(st);
     r.raw_out = take((size_t)kMaxRows * (st / 128) * 4);  // N <= staging / (2 bytes * 64 columns)
     r.xstage = take((size_t)kMaxRows * act_k * 4);
+    r.prof = take((size_t)(3 + kPhasesPerLayer * c->n_layers) * kMaxGrid * kProfWords * 8);
     r.total = off;
     return r;
 }
 
-// Chooses how an operation's tile grid is cut among the blocks: minimise the largest per-block
-// share, then the number of sequential pipeline stages, then the number of column partitions.
+// Chooses how an operation's tile grid is cut among the blocks and how a block's 8 MMA warps are
+// arranged (RW row tiles x KW column chunks per stage).  Model of a block's time in microseconds:
+// the larger of streaming its share (at a fair share of HBM bandwidth) and walking its pipeline
+// stages, plus a charge per column partition for the atomic adds that merge partial sums.
+// Operations whose epilogue needs complete sums (full_k) keep all columns in one block.
 void choose_partition(OpDesc& o, int G, bool full_k) {
-    long long best_cost = -1;
-    int best_stages = 0, bp_row = 1, bp_k = 1;
-    for (int pr = 1; pr <= o.T && pr <= G; ++pr) {
-        const int pk_max = full_k ? 1 : (G / pr < o.C ? G / pr : o.C);
-        for (int pk = 1; pk <= pk_max; ++pk) {
-            const int tiles = (o.T + pr - 1) / pr, chunks = (o.C + pk - 1) / pk;
-            const int passes = (tiles + kConsumerWarps - 1) / kConsumerWarps;
-            const long long cost = (long long)tiles * chunks;
-            const int stages = passes * chunks;
-            if (best_cost < 0 || cost < best_cost || (cost == best_cost && stages < best_stages) ||
-                (cost == best_cost && stages == best_stages && pk < bp_k)) {
-                best_cost = cost;
-                best_stages = stages;
-                bp_row = pr;
-                bp_k = pk;
+    double best_t = -1.0;
+    o.RW = kConsumerWarps;
+    o.P_row = 1;
+    o.P_k = 1;
+    const int rw_first = kConsumerWarps, rw_last = full_k ? kConsumerWarps : kConsumerWarps / kMaxKW;
+    for (int RW = rw_first; RW >= rw_last; RW /= 2) {
+        const int KW = kConsumerWarps / RW;
+        for (int pr = 1; pr <= o.T && pr <= G; ++pr) {
+            const int pk_max = full_k ? 1 : (G / pr < o.C ? G / pr : o.C);
+            for (int pk = 1; pk <= pk_max; ++pk) {
+                const int tiles = (o.T + pr - 1) / pr, chunks = (o.C + pk - 1) / pk;
+                const int passes = (tiles + RW - 1) / RW;
+                const int stages = passes * ((chunks + KW - 1) / KW);
+                const double stream = (double)tiles * chunks * kTileBytes / 44000.0;
+                const double walk = 0.25 * stages;
+                const double t = (stream > walk ? stream : walk) + (pk > 1 ? 0.2 * pk : 0.0);
+                if (best_t < 0 || t < best_t - 1e-9) {
+                    best_t = t;
+                    o.RW = RW;
+                    o.P_row = pr;
+                    o.P_k = pk;
+                }
             }
         }
     }
-    o.P_row = bp_row;
-    o.P_k = bp_k;
 }
 
 }  // namespace
@@ -140,6 +150,8 @@ struct sdv_ctx {
     int last_rows;  // rows of the last verify
     int bar_base;
     int parity;
+    int profile;
+    int ahead;
     int last_cuda;
     long long launches;
     bool have_verify_time;
@@ -181,6 +193,8 @@ int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph
     P.ph_end = ph_end;
     P.bar_base = ctx->bar_base;
     P.store_logits = ctx->parity;
+    P.ahead = ctx->ahead;
+    P.prof = ctx->profile ? (unsigned long long*)(ctx->ws + ctx->r.prof) : nullptr;
     const int nbar = ph_end - ph_begin - 1;
     ctx->bar_base += nbar * ctx->G;
     const int NT = (rows + 7) / 8;
@@ -299,6 +313,10 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
     if (sms > kMaxGrid) sms = kMaxGrid;
     ctx->G = sms;  // one persistent block per SM
     ctx->r = carve(cfg);
+    {
+        const char* e_ahead = getenv("SDV_AHEAD");
+        ctx->ahead = e_ahead ? atoi(e_ahead) : 0;
+    }
     e = cudaHostAlloc((void**)&ctx->pinned, 4096, cudaHostAllocDefault);
     if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev0);
     if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev1);
@@ -346,6 +364,7 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
     P.qkv_acc = (float*)(ws + ctx->r.qkv_acc);
     P.sumsq = (float*)(ws + ctx->r.sumsq);
     P.act = ws + ctx->r.act;
+    P.attn_op = ws + ctx->r.attn_op;
     P.part_o = (float*)(ws + ctx->r.part_o);
     P.part_ml = (float*)(ws + ctx->r.part_ml);
     P.cand_val = (float*)(ws + ctx->r.cand_val);
@@ -501,7 +520,7 @@ int sdv_prefill_chunk(sdv_ctx* ctx, const int32_t* host_tokens, int n, int is_la
     if (tile > 24) tile = 24;
     tile = tile / 8 * 8;
     if (tile < 8) tile = 8;
-    const int n_ph = 1 + 5 * c.n_layers;
+    const int n_ph = 1 + kPhasesPerLayer * c.n_layers;
     int done = 0;
     while (done < n) {
         const int rows = (n - done < tile) ? n - done : tile;
@@ -576,7 +595,7 @@ int sdv_verify(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, int32_t* 
         ctx->launches++;
         CK(cudaGetLastError());
     }
-    int rc = launch_forward(ctx, rows, ctx->kv_len, 0, 0, 2 + 5 * c.n_layers, true);
+    int rc = launch_forward(ctx, rows, ctx->kv_len, 0, 0, 2 + kPhasesPerLayer * c.n_layers, true);
     if (rc) return rc;
     accept_kernel<<<1, 32 * rows, 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0);
     ctx->launches++;
@@ -748,7 +767,7 @@ int sdv_debug_gemm(sdv_ctx* ctx, const float* host_x, const uint16_t* host_w, fl
     const int saved_N = ctx->P.raw_N;
     ctx->P.op[OP_RAW] = o;
     ctx->P.raw_N = N;
-    const int ph = 2 + 5 * c.n_layers;
+    const int ph = 2 + kPhasesPerLayer * c.n_layers;
     rc = launch_forward(ctx, M, 0, 1, ph, ph + 1, true);
     ctx->P.op[OP_RAW] = saved;
     ctx->P.raw_N = saved_N;
@@ -758,6 +777,21 @@ int sdv_debug_gemm(sdv_ctx* ctx, const float* host_x, const uint16_t* host_w, fl
     if (rc) return rc;
     if (dev_ms) CK(cudaEventElapsedTime(dev_ms, ctx->ev0, ctx->ev1));
     return SDV_OK;
+}
+
+int sdv_debug_profile(sdv_ctx* ctx, int on, unsigned long long* host_out, int n_phases) {
+    if (!ctx) return SDV_EINVAL;
+    if (host_out) {
+        if (n_phases < 1 || n_phases > 3 + kPhasesPerLayer * ctx->cfg.n_layers) return SDV_EINVAL;
+        CK(cudaMemcpyAsync(host_out, ctx->ws + ctx->r.prof, (size_t)n_phases * ctx->G * kProfWords * 8, cudaMemcpyDeviceToHost,
+                           ctx->stream));
+        CK(cudaStreamSynchronize(ctx->stream));
+    }
+    if (on)
+        CK(cudaMemsetAsync(ctx->ws + ctx->r.prof, 0,
+                           (size_t)(3 + kPhasesPerLayer * ctx->cfg.n_layers) * kMaxGrid * kProfWords * 8, ctx->stream));
+    ctx->profile = on ? 1 : 0;
+    return ctx->G;
 }
 
 int sdv_debug_timeout_probe(sdv_ctx* ctx) {
