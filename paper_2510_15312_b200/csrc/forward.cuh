@@ -73,6 +73,8 @@ struct Misc {
     float ss_part[4][kMaxRows];
     float best_v[kConsumerWarps][kMaxRows];
     int best_i[kConsumerWarps][kMaxRows];
+    Part part[OP_COUNT];  // this block's share of every operation
+    FwdParams P;  // block-local copy of the launch parameters (cheap to reach from out-of-line code)
 };
 static_assert(sizeof(Misc) <= kMiscSmemBytes, "misc shared memory");
 
@@ -84,7 +86,7 @@ __device__ __forceinline__ bool grid_barrier(const FwdParams& P, int target, Mis
     named_bar_sync(1, kWorkerThreads);
     if (wtid == 0) {
         __threadfence();
-        atomicAdd(P.bar, 1);
+        red_add_s32(P.bar, 1);  // no return value to wait for: polling starts at once
         const uint64_t t0 = global_timer_ns();
         uint32_t spins = 0;
         while ((int)(ld_acquire_gpu(P.bar) - target) < 0) {
@@ -106,9 +108,8 @@ __device__ __forceinline__ bool grid_barrier(const FwdParams& P, int target, Mis
 // ------------------------------------------------------------------------------------------
 // Weight streamer (one thread).
 template <int NT>
-__device__ __forceinline__ void producer_loop(const FwdParams& P, uint8_t* smem, Misc* misc) {
+__device__ __noinline__ void producer_loop(const FwdParams& P, uint8_t* smem, Misc* misc) {
     using SL = SmemLayout<NT>;
-    const int cta = blockIdx.x;
     const uint64_t policy = l2_policy_evict_first();
     uint32_t it = 0;
     const uint32_t ahead = (P.ahead >= 1 && P.ahead <= SL::NSTAGE) ? (uint32_t)P.ahead : (uint32_t)SL::NSTAGE;
@@ -118,15 +119,13 @@ __device__ __forceinline__ void producer_loop(const FwdParams& P, uint8_t* smem,
         const int kind = decode_phase(ph, P.n_layers, layer);
         const int op = phase_op(kind);
         if (op < 0) continue;
-        const OpDesc& od = P.op[op];
-        const Part pt = get_part(od, cta, P.G);
+        const Part& pt = misc->part[op];
         if (pt.ntiles == 0) continue;
-        const int KW = kConsumerWarps / od.RW;
+        const int KW = 1 << pt.lkw;
         const uint8_t* src = op_weights(P, kind, layer) + pt.off;
-        const int npass = part_passes(pt, od.RW);
-        const int nst = (pt.nchunks + KW - 1) / KW;
+        const int npass = pt.npass, nst = pt.nst;
         for (int p = 0; p < npass && ok; ++p) {
-            const int pcount = even_count(pt.ntiles, npass, p);
+            const int pcount = pass_count(pt, p);
             for (int st = 0; st < nst; ++st, ++it) {
                 const int kcnt = min(KW, pt.nchunks - st * KW);
                 const uint32_t bytes = (uint32_t)(pcount * kcnt) * kTileBytes;
@@ -160,164 +159,180 @@ __device__ __forceinline__ void producer_loop(const FwdParams& P, uint8_t* smem,
 }
 
 // ------------------------------------------------------------------------------------------
-// Activation loaders.  The operand chunks of a phase are dealt round-robin to the three loader
-// warps; each warp keeps two chunks' loads in flight (registers) and stores a chunk into its
-// stage's slot once the slot is free.
-template <int NT, bool NORM>
-struct ChunkRegs {
-    // NORM: fp32 residual values of 2*NT (token, 8-column) units + the 8 norm weights of the lane's
-    // column group; otherwise 2*NT ready-made 16-byte bf16 units.
-    float4 h[NORM ? 2 * NT : 1][2];
-    float4 w[2];
-    uint4 v[NORM ? 1 : 2 * NT];
-};
+// Activation loaders.  The operand chunks ([rows x 64] bf16 each) of a phase are dealt round-robin
+// to the three loader warps.
+//  - Ready-made operands (SwiGLU output, merged attention output) are already stored chunk by
+//    chunk in the shared-memory image: one lane issues a bulk asynchronous copy per chunk straight
+//    into the stage's slot, as far ahead as free slots allow.
+//  - Operands that still need the RMSNorm scale: the chunk's fp32 residual rows and norm weights
+//    are first staged in shared memory by 16-byte asynchronous copies (up to three chunks in flight
+//    per warp, no registers held), then scaled, rounded to bf16 and stored into the slot.  The
+//    row sums of squares fall out of the first pass.
+constexpr int kRedBytes = 16384;  // staged-epilogue buffer at the start of the attention region
+constexpr int kStageBufBytes = (kAttnSmemBytes - kRedBytes) / kLoaderWarps / 256 * 256;
 
-template <int NT, bool NORM>
-__device__ __forceinline__ void chunk_issue(const FwdParams& P, ChunkRegs<NT, NORM>& r, const float* wn,
-                                            const uint8_t* src_op, int chunk, int lane) {
-    if (NORM) {
-        const int q = lane & 7;
-        r.w[0] = __ldg(reinterpret_cast<const float4*>(wn + chunk * 64 + q * 8));
-        r.w[1] = __ldg(reinterpret_cast<const float4*>(wn + chunk * 64 + q * 8 + 4));
-#pragma unroll
-        for (int i = 0; i < 2 * NT; ++i) {
-            const int tok = (lane + 32 * i) >> 3;
-            if (tok < P.M) {
-                const float* hp = P.h + (size_t)tok * P.d + chunk * 64 + q * 8;
-                r.h[NORM ? i : 0][0] = ldcg_f4(hp);
-                r.h[NORM ? i : 0][1] = ldcg_f4(hp + 4);
-            }
-        }
-    } else {
-        const uint8_t* src = src_op + (size_t)chunk * SmemLayout<NT>::A_CHUNK;
-#pragma unroll
-        for (int i = 0; i < 2 * NT; ++i) r.v[NORM ? 0 : i] = ldcg_u4(src + (lane + 32 * i) * 16);
-    }
+__device__ __forceinline__ uint32_t chunk_arrivals(int c, int nchunks, int KW) {
+    uint32_t cnt = kMaxKW / KW;
+    if (c == nchunks - 1) cnt *= (uint32_t)(KW - ((nchunks - 1) & (KW - 1)));  // the last chunk covers a ragged stage
+    return cnt;
 }
 
-template <int NT, bool NORM>
-__device__ __forceinline__ void chunk_store(const FwdParams& P, const ChunkRegs<NT, NORM>& r, uint8_t* dst, int lane,
-                                            float (&ss)[2 * NT], bool accumulate) {
-    if (NORM) {
-        const int q = lane & 7;
-#pragma unroll
-        for (int i = 0; i < 2 * NT; ++i) {
-            const int tok = (lane + 32 * i) >> 3;
-            uint4 out = make_uint4(0, 0, 0, 0);
-            if (tok < P.M) {
-                const float4 a = r.h[NORM ? i : 0][0], b = r.h[NORM ? i : 0][1];
-                if (accumulate)
-                    ss[i] += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w + b.x * b.x + b.y * b.y + b.z * b.z +
-                             b.w * b.w;
-                out.x = pack_bf16(a.x * r.w[0].x, a.y * r.w[0].y);
-                out.y = pack_bf16(a.z * r.w[0].z, a.w * r.w[0].w);
-                out.z = pack_bf16(b.x * r.w[1].x, b.y * r.w[1].y);
-                out.w = pack_bf16(b.z * r.w[1].z, b.w * r.w[1].w);
+template <int NT>
+__device__ __noinline__ void loader_copy(const FwdParams& P, int kind, const OpDesc& od, const Part& pt, uint8_t* smem,
+                                         Misc* misc, uint32_t& it, uint32_t& ci, int lw, int lane,
+                                         unsigned long long* prof) {
+    using SL = SmemLayout<NT>;
+    const int KW = 1 << pt.lkw, lkw = pt.lkw;
+    const int npass = pt.npass, nst = pt.nst;
+    const int nchunks = pt.nchunks;
+    const uint8_t* src_op = (kind == PH_O) ? P.attn_op : P.act;
+    const uint32_t it0 = it, ci0 = ci;
+    const int total = npass * nchunks;
+    const int x0 = (int)((lw + kLoaderWarps - (ci0 % kLoaderWarps)) % kLoaderWarps);
+    if (prof && lw == 0 && lane == 0) prof[6] = global_timer_ns();
+    if (lane == 0) {
+        bool dead = *(volatile int*)&misc->abort_flag != 0;
+        int p_ = 0, c_ = x0;
+        for (int x = x0; x < total && !dead; x += kLoaderWarps, c_ += kLoaderWarps) {
+            while (c_ >= nchunks) { c_ -= nchunks; ++p_; }
+            const uint32_t sidx = it0 + (uint32_t)(p_ * nst + (c_ >> lkw));
+            const uint32_t slot = sidx % SL::NSTAGE, use = sidx / SL::NSTAGE;
+            if (use > 0 &&
+                !mbar_wait_bounded(&misc->empty[slot], (use - 1) & 1, &misc->abort_flag, P.wait_limit_ns)) {
+                dead = true;
+                break;
             }
-            *reinterpret_cast<uint4*>(dst + swz_unit(tok, q)) = out;
+            const uint32_t cnt = chunk_arrivals(c_, nchunks, KW);
+            if (cnt > 1) mbar_arrive_cnt(&misc->full_a[slot], cnt - 1);
+            mbar_arrive_expect_tx(&misc->full_a[slot], SL::A_CHUNK);
+            bulk_g2s_plain(smem + SL::A_OFF + slot * SL::A_STAGE + (c_ & (KW - 1)) * SL::A_CHUNK,
+                           src_op + (size_t)(pt.chunk0 + c_) * SL::A_CHUNK, SL::A_CHUNK, &misc->full_a[slot]);
+            if (prof && lw == 0 && x == x0) prof[7] = global_timer_ns();
         }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 2 * NT; ++i) *reinterpret_cast<uint4*>(dst + (lane + 32 * i) * 16) = r.v[NORM ? 0 : i];
     }
+    __syncwarp();
+    if (prof && lw == 0 && lane == 0) prof[5] = global_timer_ns();
+    it = it0 + (uint32_t)(npass * nst);
+    ci = ci0 + (uint32_t)total;
 }
 
 // A bounded wait that ran out marks the warp "dead": it stops touching the pipeline but still
-// walks the control flow, so that every named barrier is reached by all of its threads.
-template <int NT, bool NORM>
-__device__ __forceinline__ void loader_phase(const FwdParams& P, int kind, int layer, const OpDesc& od, const Part& pt, uint8_t* smem,
-                             Misc* misc, uint32_t& it, uint32_t& ci, int lw, int lane, unsigned long long* prof) {
+// walks the control flow to the end.
+template <int NT>
+__device__ __noinline__ void loader_norm(const FwdParams& P, int kind, int layer, const OpDesc& od, const Part& pt,
+                                         uint8_t* smem, Misc* misc, uint32_t& it, uint32_t& ci, int lw, int lane,
+                                         unsigned long long* prof) {
     using SL = SmemLayout<NT>;
-    const int KW = kConsumerWarps / od.RW;
-    const int npass = part_passes(pt, od.RW);
-    const int nst = (pt.nchunks + KW - 1) / KW;
+    const int KW = 1 << pt.lkw, lkw = pt.lkw;
+    const int npass = pt.npass, nst = pt.nst;
     const int nchunks = pt.nchunks;
-    const float* wn = nullptr;
-    if (kind == PH_QKV) wn = P.norm_w + (size_t)(layer * 2 + 0) * P.d;
-    if (kind == PH_GU) wn = P.norm_w + (size_t)(layer * 2 + 1) * P.d;
-    if (kind == PH_LM) wn = P.norm_w + (size_t)(P.n_layers * 2) * P.d;
-    const uint8_t* src_op = (kind == PH_O) ? P.attn_op : P.act;
+    const int M = P.M, d = P.d;
+    const float* wn = P.norm_w + (size_t)(kind == PH_QKV ? layer * 2 : (kind == PH_GU ? layer * 2 + 1 : P.n_layers * 2)) * d;
+    const float* hbase = P.h;
     float ss[2 * NT];
 #pragma unroll
     for (int i = 0; i < 2 * NT; ++i) ss[i] = 0.f;
     bool dead = *(volatile int*)&misc->abort_flag != 0;
     const uint32_t it0 = it, ci0 = ci;
     const int total = npass * nchunks;  // chunk visits of this phase, pass-major
-    // first visit handled by this warp
     const int x0 = (int)((lw + kLoaderWarps - (ci0 % kLoaderWarps)) % kLoaderWarps);
-
-    // Publish this warp's share of the per-row sums of squares as soon as its first-pass chunks are
-    // done: the MMA warps need them at the end of the first pass, before later passes can drain.
-    bool published = false;
-#define SDV_PUBLISH()                                                                                             \
-    do {                                                                                                          \
-        published = true;                                                                                         \
-        _Pragma("unroll") for (int i = 0; i < 2 * NT; ++i) {                                                      \
-            float v = ss[i];                                                                                      \
-            v += __shfl_xor_sync(0xffffffffu, v, 1);                                                              \
-            v += __shfl_xor_sync(0xffffffffu, v, 2);                                                              \
-            v += __shfl_xor_sync(0xffffffffu, v, 4);                                                              \
-            const int tok = (lane + 32 * i) >> 3;                                                                 \
-            if ((lane & 7) == 0) {                                                                                \
-                if (kind == PH_QKV) {                                                                             \
-                    /* the attention step normalises q, k, v; only one row partition reports */                  \
-                    if (pt.pr == 0 && tok < P.M && !dead) atomicAdd(P.sumsq + (layer & 1) * kMaxRows + tok, v);   \
-                } else {                                                                                          \
-                    misc->ss_part[lw][tok] = v;                                                                   \
-                }                                                                                                 \
-            }                                                                                                     \
-        }                                                                                                         \
-        if (kind != PH_QKV) {                                                                                     \
-            __syncwarp();                                                                                         \
-            if (lane == 0) mbar_arrive(&misc->rstd_bar);                                                          \
-        }                                                                                                         \
-    } while (0)
-
+    const int nmine = (x0 < total) ? (total - x0 + kLoaderWarps - 1) / kLoaderWarps : 0;
+    const int entry = (M + 1) * 256;  // M rows of 64 floats, then the 64 norm weights
+    int D = kStageBufBytes / entry;
+    if (D > 3) D = 3;
+    if (D < 1) D = 1;
+    uint8_t* stage = smem + SL::ATT_OFF + kRedBytes + lw * kStageBufBytes;
     if (prof && lw == 0 && lane == 0) prof[6] = global_timer_ns();
-    bool first_done = false;
-    ChunkRegs<NT, NORM> ra, rb;
-    int xa = x0, xb = -1;
-    if (NORM && x0 >= nchunks) SDV_PUBLISH();  // no first-pass chunk falls to this warp
-    if (xa < total && !dead) chunk_issue<NT, NORM>(P, ra, wn, src_op, pt.chunk0 + xa % nchunks, lane);
-    // finish a chunk: wait for its slot, transform + store, signal
-#define SDV_FINISH(REGS, XV)                                                                                      \
-    do {                                                                                                          \
-        const int p_ = (XV) / nchunks, c_ = (XV) % nchunks;                                                       \
-        const uint32_t sidx = it0 + (uint32_t)(p_ * nst + c_ / KW);                                               \
-        const uint32_t slot = sidx % SL::NSTAGE, use = sidx / SL::NSTAGE;                                         \
-        if (!dead && use > 0) {                                                                                   \
-            const bool got =                                                                                      \
-                mbar_wait_bounded(&misc->empty[slot], (use - 1) & 1, &misc->abort_flag, P.wait_limit_ns);         \
-            if (!__all_sync(0xffffffffu, got)) dead = true;                                                       \
-        }                                                                                                         \
-        if (!dead) {                                                                                              \
-            uint8_t* dst = smem + SL::A_OFF + slot * SL::A_STAGE + (c_ % KW) * SL::A_CHUNK;                       \
-            chunk_store<NT, NORM>(P, REGS, dst, lane, ss, p_ == 0);                                               \
-            __syncwarp();                                                                                         \
-            if (lane == 0) {                                                                                      \
-                uint32_t cnt = kMaxKW / KW;                                                                       \
-                if (c_ == nchunks - 1) cnt *= (uint32_t)(KW - (nchunks - 1) % KW); /* ragged last stage */        \
-                mbar_arrive_cnt(&misc->full_a[slot], cnt);                                                        \
-            }                                                                                                     \
-        }                                                                                                         \
-        if (prof && !first_done && lw == 0 && lane == 0) { prof[7] = global_timer_ns(); }                        \
-        first_done = true;                                                                                        \
-        if (NORM && !published && (XV) + kLoaderWarps >= nchunks) SDV_PUBLISH();                                  \
-    } while (0)
 
-    while (xa < total) {
-        xb = xa + kLoaderWarps;
-        if (xb < total && !dead) chunk_issue<NT, NORM>(P, rb, wn, src_op, pt.chunk0 + xb % nchunks, lane);
-        SDV_FINISH(ra, xa);
-        if (xb >= total) break;
-        xa = xb + kLoaderWarps;
-        if (xa < total && !dead) chunk_issue<NT, NORM>(P, ra, wn, src_op, pt.chunk0 + xa % nchunks, lane);
-        SDV_FINISH(rb, xb);
+    int ic = x0;  // chunk index (within the partition) of the next visit to issue, kept below nchunks
+    while (ic >= nchunks) ic -= nchunks;
+    auto issue = [&](int k) {
+        if (k < nmine) {
+            const int chunk = pt.chunk0 + ic;
+            ic += kLoaderWarps;
+            while (ic >= nchunks) ic -= nchunks;
+            uint8_t* dst = stage + (k % D) * entry;
+            const int units = (M + 1) * 16;
+            for (int u = lane; u < units; u += 32) {
+                const int row = u >> 4, part = u & 15;
+                const float* src = (row < M ? hbase + (size_t)row * d : wn) + chunk * 64 + part * 4;
+                cp_async_16(dst + u * 16, src);
+            }
+        }
+        cp_async_commit();  // possibly empty: keeps the group count uniform
+    };
+    auto publish = [&]() {
+        // this warp's share of the per-row sums of squares (its first-pass chunks)
+#pragma unroll
+        for (int i = 0; i < 2 * NT; ++i) {
+            float v = ss[i];
+            v += __shfl_xor_sync(0xffffffffu, v, 1);
+            v += __shfl_xor_sync(0xffffffffu, v, 2);
+            v += __shfl_xor_sync(0xffffffffu, v, 4);
+            const int tok = (lane + 32 * i) >> 3;
+            if ((lane & 7) == 0) {
+                if (kind == PH_QKV) {
+                    // the attention step normalises q, k, v; only one row partition reports
+                    if (pt.pr == 0 && tok < M && !dead) atomicAdd(P.sumsq + (layer & 1) * kMaxRows + tok, v);
+                } else {
+                    misc->ss_part[lw][tok] = v;
+                }
+            }
+        }
+        if (kind != PH_QKV) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&misc->rstd_bar);
+        }
+    };
+
+    bool published = false;
+    if (x0 >= nchunks) { publish(); published = true; }  // no first-pass chunk falls to this warp
+    for (int k = 0; k < D; ++k) issue(k);
+    int p_ = 0, c_ = x0;
+    for (int k = 0; k < nmine; ++k, c_ += kLoaderWarps) {
+        const int x = x0 + k * kLoaderWarps;
+        while (c_ >= nchunks) { c_ -= nchunks; ++p_; }
+        if (D == 3) cp_async_wait<2>(); else if (D == 2) cp_async_wait<1>(); else cp_async_wait<0>();
+        __syncwarp();
+        const uint32_t sidx = it0 + (uint32_t)(p_ * nst + (c_ >> lkw));
+        const uint32_t slot = sidx % SL::NSTAGE, use = sidx / SL::NSTAGE;
+        if (!dead && use > 0) {
+            const bool got = mbar_wait_bounded(&misc->empty[slot], (use - 1) & 1, &misc->abort_flag, P.wait_limit_ns);
+            if (!__all_sync(0xffffffffu, got)) dead = true;
+        }
+        if (!dead) {
+            const uint8_t* src = stage + (k % D) * entry;
+            uint8_t* dst = smem + SL::A_OFF + slot * SL::A_STAGE + (c_ & (KW - 1)) * SL::A_CHUNK;
+            const int q = lane & 7;
+            const float4 w0 = *reinterpret_cast<const float4*>(src + M * 256 + q * 32);
+            const float4 w1 = *reinterpret_cast<const float4*>(src + M * 256 + q * 32 + 16);
+#pragma unroll
+            for (int i = 0; i < 2 * NT; ++i) {
+                const int tok = (lane + 32 * i) >> 3;
+                uint4 out = make_uint4(0, 0, 0, 0);
+                if (tok < M) {
+                    const float4 a = *reinterpret_cast<const float4*>(src + tok * 256 + q * 32);
+                    const float4 b = *reinterpret_cast<const float4*>(src + tok * 256 + q * 32 + 16);
+                    if (p_ == 0)
+                        ss[i] += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w + b.x * b.x + b.y * b.y + b.z * b.z +
+                                 b.w * b.w;
+                    out.x = pack_bf16(a.x * w0.x, a.y * w0.y);
+                    out.y = pack_bf16(a.z * w0.z, a.w * w0.w);
+                    out.z = pack_bf16(b.x * w1.x, b.y * w1.y);
+                    out.w = pack_bf16(b.z * w1.z, b.w * w1.w);
+                }
+                *reinterpret_cast<uint4*>(dst + swz_unit(tok, q)) = out;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cnt(&misc->full_a[slot], chunk_arrivals(c_, nchunks, KW));
+            if (prof && k == 0 && lw == 0 && lane == 0) prof[7] = global_timer_ns();
+        }
+        __syncwarp();   // every lane is done with the staging entry before it is refilled
+        issue(k + D);
+        if (!published && x + kLoaderWarps >= nchunks) { publish(); published = true; }
     }
-#undef SDV_FINISH
-
-    if (NORM && !published) SDV_PUBLISH();
-#undef SDV_PUBLISH
+    cp_async_wait<0>();
+    if (!published) publish();
     if (prof && lw == 0 && lane == 0) prof[5] = global_timer_ns();
     it = it0 + (uint32_t)(npass * nst);
     ci = ci0 + (uint32_t)total;
@@ -326,15 +341,14 @@ __device__ __forceinline__ void loader_phase(const FwdParams& P, int kind, int l
 // ------------------------------------------------------------------------------------------
 // MMA warps.
 template <int NT>
-__device__ __forceinline__ void consumer_phase(const FwdParams& P, int kind, int layer, const OpDesc& od, const Part& pt, uint8_t* smem,
+__device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int layer, const OpDesc& od, const Part& pt, uint8_t* smem,
                                Misc* misc, uint32_t& it, uint32_t& ci, uint32_t& norm_uses, int warp, int lane,
                                unsigned long long* prof) {
     using SL = SmemLayout<NT>;
     constexpr int MP = SL::MP;
-    const int RW = od.RW, KW = kConsumerWarps / RW;
-    const int rw = warp % RW, kw = warp / RW;
-    const int npass = part_passes(pt, RW);
-    const int nst = (pt.nchunks + KW - 1) / KW;
+    const int RW = od.RW, KW = 1 << pt.lkw;
+    const int rw = warp & (RW - 1), kw = warp >> (3 - pt.lkw);
+    const int npass = pt.npass, nst = pt.nst;
     const int g = lane >> 2, q2 = (lane & 3) * 2;
     const bool need_rstd = (kind == PH_GU || kind == PH_LM);
     const bool staged = (kind == PH_QKV || kind == PH_O || kind == PH_DOWN || kind == PH_RAW);
@@ -355,8 +369,8 @@ __device__ __forceinline__ void consumer_phase(const FwdParams& P, int kind, int
     ci += (uint32_t)(npass * pt.nchunks);
 
     for (int p = 0; p < npass; ++p) {
-        const int pcount = even_count(pt.ntiles, npass, p);
-        const int tile_base = pt.tile0 + even_start(pt.ntiles, npass, p);
+        const int pcount = pass_count(pt, p);
+        const int tile_base = pt.tile0 + pass_start(pt, p);
         const int tile = tile_base + rw;
         float acc[NT][4];
 #pragma unroll
@@ -550,7 +564,7 @@ __device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps)
 }
 
 template <int HD>
-__device__ __forceinline__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int S, int kps, uint8_t* att, int wtid) {
+__device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int S, int kps, uint8_t* att, int wtid) {
     constexpr int HD2 = HD / 2;
     constexpr int KSTEPS = HD / 16;
     constexpr int UNITS = HD / 8;  // 16-byte units per K/V row
@@ -825,7 +839,7 @@ __device__ void attention_phase(const FwdParams& P, int layer, uint8_t* att, int
 // Merge of the split-KV partial results into the output projection's bf16 operand.  One warp per
 // (query head, row, 8 columns); lanes run over the splits.
 template <int NT>
-__device__ __forceinline__ void combine_phase(const FwdParams& P, int wtid) {
+__device__ __noinline__ void combine_phase(const FwdParams& P, int wtid) {
     constexpr int A_CHUNK = SmemLayout<NT>::A_CHUNK;
     int S, kps;
     attn_split(P, S, kps);
@@ -908,14 +922,22 @@ __device__ void zero_qkv_acc(const FwdParams& P, int sumsq_buf, int wtid) {
 
 // ------------------------------------------------------------------------------------------
 template <int NT>
-__global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_constant__ FwdParams P) {
+__global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_constant__ FwdParams Pg) {
     using SL = SmemLayout<NT>;
     static_assert(SL::NSTAGE >= 4 && SL::NSTAGE <= 16, "ring depth");
-    static_assert(kConsumerWarps * SL::MP * 16 * 4 <= kAttnSmemBytes, "staged epilogue buffer");
+    static_assert(kConsumerWarps * SL::MP * 16 * 4 <= kRedBytes, "staged epilogue buffer");
+    static_assert(sizeof(FwdParams) % 4 == 0, "parameter block is copied word by word");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     Misc* misc = reinterpret_cast<Misc*>(smem + SL::MISC_OFF);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    {
+        const int* src = reinterpret_cast<const int*>(&Pg);
+        int* dst = reinterpret_cast<int*>(&misc->P);
+        for (int i = tid; i < (int)(sizeof(FwdParams) / 4); i += kThreads) dst[i] = src[i];
+    }
+    const FwdParams& P = misc->P;
+    if (tid >= 32 && tid < 32 + OP_COUNT) misc->part[tid - 32] = get_part(Pg.op[tid - 32], blockIdx.x, Pg.G);
 
     if (tid == 0) {
         for (int s = 0; s < SL::NSTAGE; ++s) {
@@ -955,7 +977,7 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
         } else {
             if (kind == PH_O) zero_qkv_acc(P, (layer + 1) & 1, wtid);
             const OpDesc& od = P.op[phase_op(kind)];
-            const Part pt = get_part(od, blockIdx.x, P.G);
+            const Part& pt = misc->part[phase_op(kind)];
             if (pt.ntiles > 0) {
                 unsigned long long* pp =
                     P.prof ? P.prof + ((size_t)(ph - P.ph_begin) * P.G + blockIdx.x) * kProfWords : nullptr;
@@ -963,8 +985,8 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
                     consumer_phase<NT>(P, kind, layer, od, pt, smem, misc, it, ci, norm_uses, warp, lane, pp);
                 } else {
                     const bool norm = (kind == PH_QKV || kind == PH_GU || kind == PH_LM);
-                    if (norm) loader_phase<NT, true>(P, kind, layer, od, pt, smem, misc, it, ci, warp - kConsumerWarps, lane, pp);
-                    else loader_phase<NT, false>(P, kind, layer, od, pt, smem, misc, it, ci, warp - kConsumerWarps, lane, pp);
+                    if (norm) loader_norm<NT>(P, kind, layer, od, pt, smem, misc, it, ci, warp - kConsumerWarps, lane, pp);
+                    else loader_copy<NT>(P, kind, od, pt, smem, misc, it, ci, warp - kConsumerWarps, lane, pp);
                 }
             }
         }

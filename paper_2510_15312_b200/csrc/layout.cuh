@@ -45,7 +45,14 @@ struct OpDesc {
 struct Part {
     int tile0, ntiles, chunk0, nchunks, pr, pk;
     unsigned long long off;  // byte offset of this partition from the operation's base
+    // derived once per launch so that the per-stage code needs no integer division
+    int npass, nst;          // passes over the row tiles; stages (groups of KW chunks) per pass
+    int pbase, prem;         // tiles per pass: pbase + (p < prem)
+    int lkw;                 // log2(KW)
+    int pad;
 };
+__host__ __device__ inline int pass_count(const Part& p, int i) { return p.pbase + (i < p.prem ? 1 : 0); }
+__host__ __device__ inline int pass_start(const Part& p, int i) { return i * p.pbase + (i < p.prem ? i : p.prem); }
 
 __host__ __device__ inline int even_start(int total, int parts, int i) {
     const int b = total / parts, r = total % parts;
@@ -65,6 +72,7 @@ __host__ __device__ inline Part get_part(const OpDesc& o, int cta, int G) {
     Part p;
     int idx = cta - o.rot;
     if (idx < 0) idx += G;
+    p.npass = p.nst = p.pbase = p.prem = p.lkw = p.pad = 0;
     if (idx >= o.P_row * o.P_k) {
         p.tile0 = p.ntiles = p.chunk0 = p.nchunks = p.pr = p.pk = 0;
         p.off = 0;
@@ -78,6 +86,12 @@ __host__ __device__ inline Part get_part(const OpDesc& o, int cta, int G) {
     p.nchunks = even_count(o.C, o.P_k, p.pk);
     p.off = (unsigned long long)kTileBytes *
             ((unsigned long long)p.tile0 * o.C + (unsigned long long)p.ntiles * p.chunk0);
+    const int KW = kConsumerWarps / o.RW;
+    p.lkw = KW == 4 ? 2 : (KW == 2 ? 1 : 0);
+    p.npass = (p.ntiles + o.RW - 1) / o.RW;
+    p.nst = (p.nchunks + KW - 1) / KW;
+    p.pbase = p.ntiles / p.npass;
+    p.prem = p.ntiles % p.npass;
     return p;
 }
 __host__ __device__ inline int part_passes(const Part& p, int RW) { return (p.ntiles + RW - 1) / RW; }

@@ -101,9 +101,10 @@ Regions carve(const sdv_config* c) {
 // Chooses how an operation's tile grid is cut among the blocks and how a block's 8 MMA warps are
 // arranged (RW row tiles x KW column chunks per stage).  Model of a block's time in microseconds:
 // the larger of streaming its share (at a fair share of HBM bandwidth) and walking its pipeline
-// stages, plus a charge per column partition for the atomic adds that merge partial sums.
+// stages or loading its operand chunks (costlier when the RMSNorm scale is applied on the way),
+// plus a charge per column partition for the atomic adds that merge partial sums.
 // Operations whose epilogue needs complete sums (full_k) keep all columns in one block.
-void choose_partition(OpDesc& o, int G, bool full_k) {
+void choose_partition(OpDesc& o, int G, bool full_k, bool norm_operand) {
     double best_t = -1.0;
     o.RW = kConsumerWarps;
     o.P_row = 1;
@@ -118,8 +119,11 @@ void choose_partition(OpDesc& o, int G, bool full_k) {
                 const int passes = (tiles + RW - 1) / RW;
                 const int stages = passes * ((chunks + KW - 1) / KW);
                 const double stream = (double)tiles * chunks * kTileBytes / 44000.0;
-                const double walk = 0.25 * stages;
-                const double t = (stream > walk ? stream : walk) + (pk > 1 ? 0.2 * pk : 0.0);
+                const double walk = 0.15 * stages;
+                const double load = (double)passes * chunks * (norm_operand ? 0.28 : 0.05);  // operand chunk visits
+                double t = stream > walk ? stream : walk;
+                if (load > t) t = load;
+                if (pk > 1) t += 0.3 + 0.05 * pk;
                 if (best_t < 0 || t < best_t - 1e-9) {
                     best_t = t;
                     o.RW = RW;
@@ -343,7 +347,7 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
         OpDesc& o = P.op[ops[i].idx];
         o.T = ops[i].N / 16;
         o.C = ops[i].K / 64;
-        choose_partition(o, ctx->G, ops[i].full_k);
+        choose_partition(o, ctx->G, ops[i].full_k, ops[i].idx != OP_O && ops[i].idx != OP_DOWN);
         o.rot = rot % ctx->G;
         rot += o.P_row * o.P_k;
         o.w_off = (ops[i].idx == OP_LM) ? 0 : woff;
@@ -752,7 +756,7 @@ int sdv_debug_gemm(sdv_ctx* ctx, const float* host_x, const uint16_t* host_w, fl
     memset(&o, 0, sizeof(o));
     o.T = N / 16;
     o.C = K / 64;
-    choose_partition(o, ctx->G, false);
+    choose_partition(o, ctx->G, false, false);
     const int NT = (M + 7) / 8;
     CK(cudaMemcpyAsync(ws + ctx->r.staging, host_w, (size_t)N * K * 2, cudaMemcpyDefault, s));
     int rc = pack_op(ctx, o, ws + ctx->r.wraw, (const uint16_t*)(ws + ctx->r.staging), N, nullptr, 0, nullptr, K, 0, 0,
