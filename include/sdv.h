@@ -188,9 +188,10 @@ int sdv_debug_gemm(sdv_ctx *ctx, const float *host_x, const uint16_t *host_w, fl
 int sdv_debug_timeout_probe(sdv_ctx *ctx);
 
 /* Per-phase timing of the forward kernel.  host_out != NULL: copies the timestamps recorded by the
- * last profiled launch, uint64 nanoseconds [n_phases][blocks][8] per thread block: phase work
- * begin, end, first pipeline stage ready, last stage consumed, epilogue done, loaders done (the
- * last four only in GEMM phases; two spare) (phase 0 = embedding, then 6 per layer: qkv, attention, split merge, o, gate|up,
+ * last profiled launch, uint64 nanoseconds [n_phases][blocks][12] per thread block: phase work
+ * begin, end, first pipeline stage ready, last stage consumed, epilogue done, loaders done, loader
+ * entry, first operand chunk stored, total wait for weights, total wait for operands (GEMM phases
+ * only; two spare) (phase 0 = embedding, then 6 per layer: qkv, attention, split merge, o, gate|up,
  * down; last = LM head).  Then switches recording on or off for later launches (it adds a block-wide barrier
  * per phase, so timed runs keep it off).  Returns the number of thread blocks, or an error. */
 int sdv_debug_profile(sdv_ctx *ctx, int on, unsigned long long *host_out, int n_phases);

@@ -259,14 +259,14 @@ class Sdv:
 
     def debug_profile(self, on: bool, n_phases: int = 0) -> Optional[np.ndarray]:
         """Switches per-phase timestamps on/off; with n_phases > 0 first returns the last recording
-        as uint64 [n_phases, blocks, 8]."""
+        as uint64 [n_phases, blocks, 12]."""
         L = lib()
         G = L.sdv_debug_profile(self._h, int(on), None, 0)
         if G < 0:
             raise SdvError(G, "sdv_debug_profile")
         if n_phases <= 0:
             return None
-        out = np.zeros((n_phases, G, 8), dtype=np.uint64)
+        out = np.zeros((n_phases, G, 12), dtype=np.uint64)
         rc = L.sdv_debug_profile(self._h, int(on), out.ctypes.data, n_phases)
         if rc < 0:
             raise SdvError(rc, "sdv_debug_profile")

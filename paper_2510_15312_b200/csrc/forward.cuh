@@ -181,39 +181,39 @@ template <int NT>
 __device__ __noinline__ void loader_copy(const FwdParams& P, int kind, const OpDesc& od, const Part& pt, uint8_t* smem,
                                          Misc* misc, uint32_t& it, uint32_t& ci, int lw, int lane,
                                          unsigned long long* prof) {
+    // The chunks of a stage are adjacent both in the operand buffer and in the stage's slot: one
+    // bulk copy per stage, issued by one lane as far ahead as free slots allow.
     using SL = SmemLayout<NT>;
-    const int KW = 1 << pt.lkw, lkw = pt.lkw;
+    const int KW = 1 << pt.lkw;
     const int npass = pt.npass, nst = pt.nst;
-    const int nchunks = pt.nchunks;
     const uint8_t* src_op = (kind == PH_O) ? P.attn_op : P.act;
-    const uint32_t it0 = it, ci0 = ci;
-    const int total = npass * nchunks;
-    const int x0 = (int)((lw + kLoaderWarps - (ci0 % kLoaderWarps)) % kLoaderWarps);
+    const uint32_t it0 = it;
     if (prof && lw == 0 && lane == 0) prof[6] = global_timer_ns();
-    if (lane == 0) {
+    if (lw == 0 && lane == 0) {
         bool dead = *(volatile int*)&misc->abort_flag != 0;
-        int p_ = 0, c_ = x0;
-        for (int x = x0; x < total && !dead; x += kLoaderWarps, c_ += kLoaderWarps) {
-            while (c_ >= nchunks) { c_ -= nchunks; ++p_; }
-            const uint32_t sidx = it0 + (uint32_t)(p_ * nst + (c_ >> lkw));
-            const uint32_t slot = sidx % SL::NSTAGE, use = sidx / SL::NSTAGE;
-            if (use > 0 &&
-                !mbar_wait_bounded(&misc->empty[slot], (use - 1) & 1, &misc->abort_flag, P.wait_limit_ns)) {
-                dead = true;
-                break;
+        uint32_t sidx = it0;
+        for (int p = 0; p < npass && !dead; ++p) {
+            for (int st = 0; st < nst; ++st, ++sidx) {
+                const uint32_t slot = sidx % SL::NSTAGE, use = sidx / SL::NSTAGE;
+                if (use > 0 &&
+                    !mbar_wait_bounded(&misc->empty[slot], (use - 1) & 1, &misc->abort_flag, P.wait_limit_ns)) {
+                    dead = true;
+                    break;
+                }
+                const int kcnt = min(KW, pt.nchunks - st * KW);
+                const uint32_t bytes = (uint32_t)kcnt * SL::A_CHUNK;
+                mbar_arrive_cnt(&misc->full_a[slot], kMaxKW - 1);
+                mbar_arrive_expect_tx(&misc->full_a[slot], bytes);
+                bulk_g2s_plain(smem + SL::A_OFF + slot * SL::A_STAGE,
+                               src_op + (size_t)(pt.chunk0 + st * KW) * SL::A_CHUNK, bytes, &misc->full_a[slot]);
+                if (prof && sidx == it0) prof[7] = global_timer_ns();
             }
-            const uint32_t cnt = chunk_arrivals(c_, nchunks, KW);
-            if (cnt > 1) mbar_arrive_cnt(&misc->full_a[slot], cnt - 1);
-            mbar_arrive_expect_tx(&misc->full_a[slot], SL::A_CHUNK);
-            bulk_g2s_plain(smem + SL::A_OFF + slot * SL::A_STAGE + (c_ & (KW - 1)) * SL::A_CHUNK,
-                           src_op + (size_t)(pt.chunk0 + c_) * SL::A_CHUNK, SL::A_CHUNK, &misc->full_a[slot]);
-            if (prof && lw == 0 && x == x0) prof[7] = global_timer_ns();
         }
     }
     __syncwarp();
     if (prof && lw == 0 && lane == 0) prof[5] = global_timer_ns();
     it = it0 + (uint32_t)(npass * nst);
-    ci = ci0 + (uint32_t)total;
+    ci += (uint32_t)(npass * pt.nchunks);
 }
 
 // A bounded wait that ran out marks the warp "dead": it stops touching the pipeline but still
@@ -366,21 +366,32 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
         bi[nt][0] = bi[nt][1] = 0x7fffffff;
     }
     float* red = reinterpret_cast<float*>(smem + SL::ATT_OFF);  // [8 warps][MP][16] partial tiles (staged epilogue)
+    uint64_t wait_w = 0, wait_a = 0;
     ci += (uint32_t)(npass * pt.nchunks);
 
     for (int p = 0; p < npass; ++p) {
         const int pcount = pass_count(pt, p);
         const int tile_base = pt.tile0 + pass_start(pt, p);
         const int tile = tile_base + rw;
-        float acc[NT][4];
+        // one accumulator set per k-step of a stage: four independent MMA chains instead of one
+        float acck[4][NT][4];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+        for (int ks = 0; ks < 4; ++ks)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) acck[ks][nt][0] = acck[ks][nt][1] = acck[ks][nt][2] = acck[ks][nt][3] = 0.f;
 
         for (int st = 0; st < nst; ++st, ++it) {
             const uint32_t slot = it % SL::NSTAGE, par = (it / SL::NSTAGE) & 1;
             if (!dead) {
-                const bool got = mbar_wait_bounded(&misc->full_w[slot], par, &misc->abort_flag, P.wait_limit_ns) &&
-                                 mbar_wait_bounded(&misc->full_a[slot], par, &misc->abort_flag, P.wait_limit_ns);
+                const uint64_t tw0 = prof ? global_timer_ns() : 0;
+                bool got = mbar_wait_bounded(&misc->full_w[slot], par, &misc->abort_flag, P.wait_limit_ns);
+                const uint64_t tw1 = prof ? global_timer_ns() : 0;
+                got = got && mbar_wait_bounded(&misc->full_a[slot], par, &misc->abort_flag, P.wait_limit_ns);
+                if (prof && warp == 0 && lane == 0) {
+                    const uint64_t tw2 = global_timer_ns();
+                    wait_w += tw1 - tw0;
+                    wait_a += tw2 - tw1;
+                }
                 if (!__all_sync(0xffffffffu, got)) dead = true;
             }
             if (dead) continue;
@@ -399,14 +410,14 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
                         uint32_t b0, b1, b2, b3;
                         const int row = np * 16 + (lane & 7) + ((lane >> 4) << 3);
                         ldsm_x4(abase + swz_unit(row, ks * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
-                        mma_bf16_16816(acc[2 * np], a0, a1, a2, a3, b0, b1);
-                        mma_bf16_16816(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
+                        mma_bf16_16816(acck[ks][2 * np], a0, a1, a2, a3, b0, b1);
+                        mma_bf16_16816(acck[ks][2 * np + 1], a0, a1, a2, a3, b2, b3);
                     }
                     if (NT & 1) {
                         uint32_t b0, b1;
                         const int row = (NT - 1) * 8 + (lane & 7);
                         ldsm_x2(abase + swz_unit(row, ks * 2 + ((lane >> 3) & 1)), b0, b1);
-                        mma_bf16_16816(acc[NT - 1], a0, a1, a2, a3, b0, b1);
+                        mma_bf16_16816(acck[ks][NT - 1], a0, a1, a2, a3, b0, b1);
                     }
                 }
             }
@@ -414,6 +425,11 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
             if (lane == 0) mbar_arrive(&misc->empty[slot]);
         }
 
+        float acc[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[nt][e] = (acck[0][nt][e] + acck[1][nt][e]) + (acck[2][nt][e] + acck[3][nt][e]);
         if (prof && p == npass - 1 && warp == 0 && lane == 0) prof[3] = global_timer_ns();
         if (need_rstd && !have_rstd && !dead) {
             const bool got = mbar_wait_bounded(&misc->rstd_bar, norm_uses & 1, &misc->abort_flag, P.wait_limit_ns);
@@ -510,7 +526,11 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
                 }
         }
     }
-    if (prof && warp == 0 && lane == 0) prof[4] = global_timer_ns();
+    if (prof && warp == 0 && lane == 0) {
+        prof[4] = global_timer_ns();
+        prof[8] = wait_w;
+        prof[9] = wait_a;
+    }
     if (need_rstd) ++norm_uses;
 
     if (kind == PH_LM) {

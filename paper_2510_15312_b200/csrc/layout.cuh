@@ -28,7 +28,7 @@ constexpr int kSmemBudget = 232448;                                  // 227 KB
 constexpr int kAttnSmemBytes = 32768 + 2 * 8192;                     // Q tile (128 x 128) + K and V blocks
 constexpr int kMiscSmemBytes = 4096;
 constexpr int kMaxDraftWords = 32;
-constexpr int kProfWords = 8;                                        // timestamps per (phase, block)
+constexpr int kProfWords = 12;                                       // timestamps per (phase, block)
 
 enum OpIndex { OP_QKV = 0, OP_O = 1, OP_GU = 2, OP_DOWN = 3, OP_LM = 4, OP_RAW = 5, OP_COUNT = 6 };
 
