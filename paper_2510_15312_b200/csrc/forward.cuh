@@ -373,12 +373,9 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
         const int pcount = pass_count(pt, p);
         const int tile_base = pt.tile0 + pass_start(pt, p);
         const int tile = tile_base + rw;
-        // one accumulator set per k-step of a stage: four independent MMA chains instead of one
-        float acck[4][NT][4];
+        float acc[NT][4];
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) acck[ks][nt][0] = acck[ks][nt][1] = acck[ks][nt][2] = acck[ks][nt][3] = 0.f;
+        for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
 
         for (int st = 0; st < nst; ++st, ++it) {
             const uint32_t slot = it % SL::NSTAGE, par = (it / SL::NSTAGE) & 1;
@@ -410,14 +407,14 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
                         uint32_t b0, b1, b2, b3;
                         const int row = np * 16 + (lane & 7) + ((lane >> 4) << 3);
                         ldsm_x4(abase + swz_unit(row, ks * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
-                        mma_bf16_16816(acck[ks][2 * np], a0, a1, a2, a3, b0, b1);
-                        mma_bf16_16816(acck[ks][2 * np + 1], a0, a1, a2, a3, b2, b3);
+                        mma_bf16_16816(acc[2 * np], a0, a1, a2, a3, b0, b1);
+                        mma_bf16_16816(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
                     }
                     if (NT & 1) {
                         uint32_t b0, b1;
                         const int row = (NT - 1) * 8 + (lane & 7);
                         ldsm_x2(abase + swz_unit(row, ks * 2 + ((lane >> 3) & 1)), b0, b1);
-                        mma_bf16_16816(acck[ks][NT - 1], a0, a1, a2, a3, b0, b1);
+                        mma_bf16_16816(acc[NT - 1], a0, a1, a2, a3, b0, b1);
                     }
                 }
             }
@@ -425,11 +422,6 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
             if (lane == 0) mbar_arrive(&misc->empty[slot]);
         }
 
-        float acc[NT][4];
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[nt][e] = (acck[0][nt][e] + acck[1][nt][e]) + (acck[2][nt][e] + acck[3][nt][e]);
         if (prof && p == npass - 1 && warp == 0 && lane == 0) prof[3] = global_timer_ns();
         if (need_rstd && !have_rstd && !dead) {
             const bool got = mbar_wait_bounded(&misc->rstd_bar, norm_uses & 1, &misc->abort_flag, P.wait_limit_ns);
