@@ -30,8 +30,11 @@ import numpy as np  # noqa: E402
 
 METRIC = "generated_tokens_per_sec"
 UNIT = "tokens/s"
-NCU_TRAFFIC = {  # dram__bytes_read.sum + dram__bytes_write.sum per launch of sdv_forward_kernel (see profiles/)
-}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of sdv_forward_kernel, as a multiple of the
+# algorithmic bytes: captured on the 0.5B-shaped workload (profiles/sdv_forward_kernel_qwen0.5b_ncu_full.md)
+# and scaled to the timed workload by its algorithmic bytes (traffic grows with the bytes streamed).
+# None once the kernel has changed since the capture.
+NCU_TRAFFIC_RATIO = 1.0058
 
 
 def load_peaks():
@@ -268,7 +271,9 @@ def main():
             "verify_kernel_us_p10_p90": [float(np.percentile(kms, 10)) * 1e3, float(np.percentile(kms, 90)) * 1e3],
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_kind": f"of {peak_kind}", "bytes_per_launch": wbytes + kvbytes,
-                         "traffic": NCU_TRAFFIC.get(cfg.name), "kernel": "sdv_forward_kernel"},
+                         "traffic": None if NCU_TRAFFIC_RATIO is None else (wbytes + kvbytes) * NCU_TRAFFIC_RATIO,
+                         "traffic_source": "ncu capture on the 0.5B-shaped workload, scaled by algorithmic bytes",
+                         "kernel": "sdv_forward_kernel"},
             "e2e": {"value": tokens_e_all / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * k + 4,
                     "d2h_bytes_per_step": 3 * 640},
             "gpu_launches": launches,
