@@ -37,7 +37,8 @@ enum {
     SDV_ECAPACITY = -3, /* KV cache / history would exceed max_seq */
     SDV_ESTATE = -4,    /* call order: e.g. verify before prefill finished, commit without verify */
     SDV_ECUDA = -5,     /* CUDA runtime error, see sdv_last_cuda_error() */
-    SDV_ETIMEOUT = -6   /* a bounded device-side wait ran out; the context must be re-created */
+    SDV_ETIMEOUT = -6,  /* a bounded device-side wait ran out; the context must be re-created */
+    SDV_ETOOBIG = -7    /* sdv_gemm_noalloc: the problem exceeds its fixed scratch area */
 };
 
 #define SDV_K_MAX 16 /* longest draft per verify step (M = k+1 <= 17 rows) */
@@ -202,6 +203,35 @@ long long sdv_launch_count(const sdv_ctx *ctx);
 /* Device time in milliseconds of the last forward kernel launched by sdv_verify (CUDA events on
  * the context's stream; synchronises on the closing event). */
 int sdv_last_verify_ms(sdv_ctx *ctx, float *ms);
+
+/* The same GEMM as sdv_debug_gemm, Y[M][N] = X[M][K] * W[N][K]^T (operands rounded to bf16, fp32
+ * accumulate), for callers that may not allocate.  The paper has no counterpart: this is a
+ * library convenience.  It needs no context and asks the CUDA runtime for no memory at any point,
+ * so it can be used where an allocation is unwelcome or impossible: inside a serving loop whose
+ * memory is fully handed out to the KV cache, from a plug-in that was given a fixed budget, or at
+ * a point where the implicit device synchronisation of cudaMalloc / cudaFree would stall other
+ * streams.
+ *
+ * All three buffers are DEVICE pointers on the current device and stay owned by the caller:
+ * dev_x fp32 [M][K], dev_w bf16 bits [N][K] row-major, dev_y fp32 [M][N] (overwritten).
+ * cuda_stream is a cudaStream_t (NULL = the default stream); the work is queued on it and the
+ * call returns after it has finished (it synchronises that stream).
+ *
+ * Scratch (the weights in streaming order, the bf16 operand, the accumulators, an error word)
+ * lives in a fixed array of about 2.8 MB inside the library's device image, present on every GPU
+ * that loads the library for as long as it stays loaded.  Hence the limits: M <= 32, N <= 4096,
+ * K <= 4096, N % 16 == 0, K % 64 == 0 and N * K * 2 <= 2 MiB; a larger problem returns
+ * SDV_ETOOBIG and touches nothing, a malformed one SDV_EINVAL.  The array keeps whatever the last
+ * call left in it; each call clears the parts that must start at zero (accumulators, error word)
+ * itself.  There is one array per GPU, so two calls that overlap in time on one GPU (different
+ * streams or threads) race on it: serialise them.
+ *
+ * The first call on each device looks up the array's device address (a one-time set-up step that
+ * also makes the runtime load the library's device code if it has not yet); make that first call
+ * before starting any stream capture.  Returns SDV_OK, SDV_EINVAL, SDV_ETOOBIG, SDV_ECUDA, or
+ * SDV_ETIMEOUT if a bounded device-side wait ran out. */
+int sdv_gemm_noalloc(const float *dev_x, const uint16_t *dev_w, float *dev_y, int M, int N, int K,
+                     void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -6,7 +6,7 @@ and streams.  There is no CPU fallback: importing works without a GPU, creating 
 does not.
 """
 from .binding import (SdvError, Sdv, SdvConfig, lib, load_library, EXPORTS, OK, EINVAL, ENOMEM, ECAPACITY,
-                      ESTATE, ECUDA, ETIMEOUT)
+                      ESTATE, ECUDA, ETIMEOUT, ETOOBIG, gemm_noalloc)
 
 __all__ = ["SdvError", "Sdv", "SdvConfig", "lib", "load_library", "EXPORTS", "OK", "EINVAL", "ENOMEM",
-           "ECAPACITY", "ESTATE", "ECUDA", "ETIMEOUT"]
+           "ECAPACITY", "ESTATE", "ECUDA", "ETIMEOUT", "ETOOBIG", "gemm_noalloc"]

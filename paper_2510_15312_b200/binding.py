@@ -9,7 +9,7 @@ import numpy as np
 
 from .build import LIB_PATH, build
 
-OK, EINVAL, ENOMEM, ECAPACITY, ESTATE, ECUDA, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
+OK, EINVAL, ENOMEM, ECAPACITY, ESTATE, ECUDA, ETIMEOUT, ETOOBIG = 0, -1, -2, -3, -4, -5, -6, -7
 K_MAX = 16
 
 EXPORTS = [
@@ -18,6 +18,7 @@ EXPORTS = [
     "sdv_strerror", "sdv_last_cuda_error", "sdv_step_bytes", "sdv_debug_set_history", "sdv_debug_accept",
     "sdv_debug_force_commit", "sdv_debug_read_kv", "sdv_debug_read_hidden", "sdv_debug_gemm",
     "sdv_debug_timeout_probe", "sdv_debug_profile", "sdv_launch_count", "sdv_last_verify_ms",
+    "sdv_gemm_noalloc",
 ]
 
 
@@ -84,6 +85,7 @@ def load_library(path: Optional[str] = None):
     L.sdv_launch_count.argtypes = [vp]
     L.sdv_launch_count.restype = C.c_longlong
     L.sdv_last_verify_ms.argtypes = [vp, C.POINTER(C.c_float)]
+    L.sdv_gemm_noalloc.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp]
     for name in EXPORTS:
         if name not in ("sdv_workspace_bytes", "sdv_strerror", "sdv_launch_count"):
             getattr(L, name).restype = C.c_int
@@ -274,3 +276,22 @@ class Sdv:
 
     def debug_timeout_probe(self) -> int:
         return lib().sdv_debug_timeout_probe(self._h)
+
+
+def gemm_noalloc(x, w_bits, y, stream=None) -> int:
+    """y[M][N] = x[M][K] * w[N][K]^T on device tensors, through the entry point that allocates no
+    memory.  x: CUDA float32 [M][K]; w_bits: CUDA tensor of bf16 values (dtype bfloat16, or their
+    bits as int16 / uint16) [N][K]; y: CUDA float32 [M][N], overwritten.  All contiguous and on the
+    current device.  Returns the library's status code (OK, ETOOBIG, ...): marshalling only."""
+    import torch
+    for t in (x, w_bits, y):
+        if not (t.is_cuda and t.is_contiguous()):
+            raise ValueError("gemm_noalloc takes contiguous CUDA tensors")
+    if x.dtype != torch.float32 or y.dtype != torch.float32 or w_bits.element_size() != 2:
+        raise ValueError("gemm_noalloc: x and y float32, w 16-bit")
+    M, K = x.shape
+    N = w_bits.shape[0]
+    if tuple(w_bits.shape) != (N, K) or tuple(y.shape) != (M, N):
+        raise ValueError("gemm_noalloc: shapes do not agree")
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return lib().sdv_gemm_noalloc(x.data_ptr(), w_bits.data_ptr(), y.data_ptr(), M, N, K, s.cuda_stream)

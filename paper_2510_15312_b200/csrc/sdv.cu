@@ -281,6 +281,7 @@ const char* sdv_strerror(int code) {
         case SDV_ESTATE: return "call not valid in the current state";
         case SDV_ECUDA: return "CUDA runtime error";
         case SDV_ETIMEOUT: return "a bounded device-side wait ran out";
+        case SDV_ETOOBIG: return "problem larger than the fixed scratch area of the no-allocation entry point";
         default: return "unknown error";
     }
 }
@@ -809,6 +810,104 @@ int sdv_debug_timeout_probe(sdv_ctx* ctx) {
     CK(cudaMemsetAsync(ctx->P.state + ST_ERR, 0, 4, ctx->stream));
     CK(cudaStreamSynchronize(ctx->stream));
     return err == 2 ? SDV_ETIMEOUT : SDV_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// Stand-alone GEMM without any allocation (see include/sdv.h, sdv_gemm_noalloc).
+//
+// Its scratch memory is a fixed array in the library's device image.  Host code must not hand the
+// array's name to a kernel (there it is only a host-side stand-in); the device address is looked
+// up once per device with cudaGetSymbolAddress and passed on.
+namespace {
+constexpr size_t kNaWeightBytes = (size_t)2 << 20;              // packed weights: N * K * 2 <= 2 MiB
+constexpr int kNaMaxK = 4096, kNaMaxN = 4096;
+constexpr size_t kNaActOff = kNaWeightBytes;                    // operand chunks: K/64 * 32 rows * 128 B
+constexpr size_t kNaActBytes = (size_t)kNaMaxK / 64 * kMaxRows * 128;
+constexpr size_t kNaOutOff = kNaActOff + kNaActBytes;           // fp32 accumulators [32][N]
+constexpr size_t kNaOutBytes = (size_t)kMaxRows * kNaMaxN * 4;
+constexpr size_t kNaStateOff = kNaOutOff + kNaOutBytes;         // state words (error flag)
+constexpr size_t kNaTotal = kNaStateOff + 1024;
+constexpr int kNaMaxDevices = 64;
+uint8_t* g_na_ptr[kNaMaxDevices];  // device address of the scratch array, per device (0 = not looked up yet)
+}  // namespace
+
+static __device__ __align__(256) uint8_t g_na_scratch[kNaTotal];  // ~2.8 MB per GPU that loads the library
+
+namespace {
+template <int NT>
+cudaError_t launch_raw_nt(const FwdParams& P, cudaStream_t stream) {
+    using SL = SmemLayout<NT>;
+    cudaError_t e = cudaFuncSetAttribute(sdv_forward_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::TOTAL);
+    if (e != cudaSuccess) return e;
+    void* args[] = {(void*)&P};
+    return cudaLaunchKernel((const void*)sdv_forward_kernel<NT>, dim3(P.G), dim3(kThreads), args, SL::TOTAL, stream);
+}
+}  // namespace
+
+extern "C" {
+
+int sdv_gemm_noalloc(const float* dev_x, const uint16_t* dev_w, float* dev_y, int M, int N, int K, void* cuda_stream) {
+    if (!dev_x || !dev_w || !dev_y) return SDV_EINVAL;
+    if (M < 1 || N < 16 || N % 16 || K < 64 || K % 64) return SDV_EINVAL;
+    if (M > kMaxRows || N > kNaMaxN || K > kNaMaxK || (size_t)N * K * 2 > kNaWeightBytes) return SDV_ETOOBIG;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNaMaxDevices) return SDV_ECUDA;
+    if (!g_na_ptr[dev]) {
+        // first call on this device: look the array's device address up (do this before any stream capture)
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_na_scratch) != cudaSuccess || !p) return SDV_ECUDA;
+        g_na_ptr[dev] = (uint8_t*)p;
+    }
+    uint8_t* sc = g_na_ptr[dev];
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return SDV_ECUDA;
+    if (sms > kMaxGrid) sms = kMaxGrid;
+
+    FwdParams P;
+    memset(&P, 0, sizeof(P));
+    P.G = sms;
+    OpDesc& o = P.op[OP_RAW];
+    o.T = N / 16;
+    o.C = K / 64;
+    choose_partition(o, sms, false, false);
+    P.wraw = sc;
+    P.act = sc + kNaActOff;
+    P.raw_out = (float*)(sc + kNaOutOff);
+    P.raw_N = N;
+    P.state = (int*)(sc + kNaStateOff);
+    P.bar = P.state + 200;  // unused by a one-phase launch, kept inside the cleared words
+    P.M = M;
+    P.mode = 1;
+    P.ph_begin = 2;  // with n_layers = 0 phase 2 is the stand-alone GEMM
+    P.ph_end = 3;
+    P.wait_limit_ns = 2000000000ull;
+    const int NT = (M + 7) / 8;
+
+    // the array keeps the previous call's contents: clear what must start at zero
+    if (cudaMemsetAsync(sc + kNaOutOff, 0, (size_t)kMaxRows * N * 4, s) != cudaSuccess) return SDV_ECUDA;
+    if (cudaMemsetAsync(sc + kNaStateOff, 0, 1024, s) != cudaSuccess) return SDV_ECUDA;
+    const long long total = (long long)o.T * o.C * 128;
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    pack_weights_kernel<<<blocks, 256, 0, s>>>(o, sc, dev_w, N, nullptr, 0, nullptr, K, 0, 0, o.T, 0);
+    stage_operand_kernel<<<64, 256, 0, s>>>(dev_x, sc + kNaActOff, M, K, 8 * NT);
+    if (cudaGetLastError() != cudaSuccess) return SDV_ECUDA;
+    cudaError_t e;
+    switch (NT) {
+        case 1: e = launch_raw_nt<1>(P, s); break;
+        case 2: e = launch_raw_nt<2>(P, s); break;
+        case 3: e = launch_raw_nt<3>(P, s); break;
+        default: e = launch_raw_nt<4>(P, s); break;
+    }
+    if (e != cudaSuccess) return SDV_ECUDA;
+    if (cudaMemcpyAsync(dev_y, sc + kNaOutOff, (size_t)M * N * 4, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return SDV_ECUDA;
+    int err = 0;
+    if (cudaMemcpyAsync(&err, sc + kNaStateOff + ST_ERR * 4, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SDV_ECUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return SDV_ECUDA;
+    return err ? SDV_ETIMEOUT : SDV_OK;
 }
 
 }  // extern "C"
