@@ -817,7 +817,9 @@ int sdv_debug_timeout_probe(sdv_ctx* ctx) {
 // ------------------------------------------------------------------------------------------
 // Stand-alone GEMM without any allocation (see include/sdv.h, sdv_gemm_noalloc).
 //
-// Its scratch memory is a fixed array in the library's device image.  Host code must not hand the
+// For callers that have no memory left to give or cannot afford the device-wide stall an
+// allocation or a free brings (a serving loop whose memory is all KV cache, a plug-in with a fixed
+// budget): nothing below asks the runtime for memory.  Its scratch memory is a fixed array in the library's device image.  Host code must not hand the
 // array's name to a kernel (there it is only a host-side stand-in); the device address is looked
 // up once per device with cudaGetSymbolAddress and passed on.
 namespace {
