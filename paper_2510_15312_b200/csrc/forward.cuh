@@ -366,7 +366,7 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
         bi[nt][0] = bi[nt][1] = 0x7fffffff;
     }
     float* red = reinterpret_cast<float*>(smem + SL::ATT_OFF);  // [8 warps][MP][16] partial tiles (staged epilogue)
-    uint64_t wait_w = 0, wait_a = 0;
+    uint64_t wait_w = 0, wait_a = 0, mma_cycles = 0, mma_stages = 0;
     ci += (uint32_t)(npass * pt.nchunks);
 
     for (int p = 0; p < npass; ++p) {
@@ -393,6 +393,7 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
             }
             if (dead) continue;
             if (prof && p == 0 && st == 0 && warp == 0 && lane == 0) prof[2] = global_timer_ns();
+            const long long c0 = prof ? clock64() : 0;
             const int kcnt = min(KW, pt.nchunks - st * KW);
             if (rw < pcount && kw < kcnt) {
                 const uint32_t wbase =
@@ -420,6 +421,7 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&misc->empty[slot]);
+            if (prof) { mma_cycles += (uint64_t)(clock64() - c0); ++mma_stages; }
         }
 
         if (prof && p == npass - 1 && warp == 0 && lane == 0) prof[3] = global_timer_ns();
@@ -522,6 +524,8 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
         prof[4] = global_timer_ns();
         prof[8] = wait_w;
         prof[9] = wait_a;
+        prof[10] = mma_cycles;  // SM clock cycles between the waits' end and the slot's release, all stages
+        prof[11] = mma_stages;
     }
     if (need_rstd) ++norm_uses;
 
@@ -576,7 +580,8 @@ __device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps)
 }
 
 template <int HD>
-__device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int S, int kps, uint8_t* att, int wtid) {
+__device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int S, int kps, uint8_t* att, int wtid,
+                                            unsigned long long* prof) {
     constexpr int HD2 = HD / 2;
     constexpr int KSTEPS = HD / 16;
     constexpr int UNITS = HD / 8;  // 16-byte units per K/V row
@@ -629,6 +634,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
             }
         }
     };
+    if (prof && wtid == 0) prof[2] = global_timer_ns();
     if (!is_new && nblk > 0) issue_block(0);
 
     // ---- query tile: normalise, add bias, rotate, round to bf16; 4 rotary pairs per item
@@ -684,6 +690,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
         }
     }
 
+    if (prof && wtid == 0) prof[3] = global_timer_ns();
     const int g = lane >> 2, q2 = (lane & 3) * 2;
     const int r_lo = warp * 16 + g, r_hi = r_lo + 8;
     const int j_lo = r_lo % M, j_hi = r_hi % M;
@@ -740,6 +747,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
             store_block();
         }
         named_bar_sync(1, kWorkerThreads);  // K/V block (and, first time, the Q tile) are in place
+        if (prof && wtid == 0 && blk == 0) prof[4] = global_timer_ns();
         if (!is_new && blk + 1 < nblk) issue_block(blk + 1);
         if (warp < MT) {
             // ---- S = Q K^T for 16 rows x 32 keys
@@ -814,6 +822,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
     }
 
     // ---- un-normalised partial result of this key range
+    if (prof && wtid == 0) prof[5] = global_timer_ns();
     if (warp < MT) {
         l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
         l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
@@ -835,16 +844,17 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
     }
 }
 
-__device__ void attention_phase(const FwdParams& P, int layer, uint8_t* att, int wtid) {
+__device__ void attention_phase(const FwdParams& P, int layer, uint8_t* att, int wtid, unsigned long long* prof) {
     int S, kps;
     attn_split(P, S, kps);
     const int S1 = S + 1;
     const int nunits = P.n_kv * S1;
     for (int unit = blockIdx.x; unit < nunits; unit += P.G) {
         const int hk = unit / S1, s = unit % S1;
-        if (P.hd == 128) attention_unit<128>(P, layer, hk, s, S, kps, att, wtid);
-        else attention_unit<64>(P, layer, hk, s, S, kps, att, wtid);
+        if (P.hd == 128) attention_unit<128>(P, layer, hk, s, S, kps, att, wtid, prof);
+        else attention_unit<64>(P, layer, hk, s, S, kps, att, wtid, prof);
         named_bar_sync(1, kWorkerThreads);  // the unit's shared-memory tiles are free again
+        if (prof && wtid == 0) { prof[6] = global_timer_ns(); prof[7] = (unsigned long long)(s == S); }
     }
 }
 
@@ -983,7 +993,8 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
             embed_phase(P, wtid);
             zero_qkv_acc(P, 0, wtid);
         } else if (kind == PH_ATTN) {
-            attention_phase(P, layer, smem + SL::ATT_OFF, wtid);
+            attention_phase(P, layer, smem + SL::ATT_OFF, wtid,
+                            P.prof ? P.prof + ((size_t)(ph - P.ph_begin) * P.G + blockIdx.x) * kProfWords : nullptr);
         } else if (kind == PH_COMB) {
             combine_phase<NT>(P, wtid);
         } else {

@@ -119,7 +119,7 @@ void choose_partition(OpDesc& o, int G, bool full_k, bool norm_operand) {
                 const int passes = (tiles + RW - 1) / RW;
                 const int stages = passes * ((chunks + KW - 1) / KW);
                 const double stream = (double)tiles * chunks * kTileBytes / 44000.0;
-                const double walk = 0.15 * stages;
+                const double walk = 0.24 * stages;  // an MMA warp needs about 450 cycles per stage
                 const double load = (double)passes * chunks * (norm_operand ? 0.28 : 0.05);  // operand chunk visits
                 double t = stream > walk ? stream : walk;
                 if (load > t) t = load;
