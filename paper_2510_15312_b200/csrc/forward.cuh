@@ -179,7 +179,7 @@ __device__ __forceinline__ uint32_t chunk_arrivals(int c, int nchunks, int KW) {
 
 template <int NT>
 __device__ __noinline__ void loader_copy(const FwdParams& P, int kind, const OpDesc& od, const Part& pt, uint8_t* smem,
-                                         Misc* misc, uint32_t& it, uint32_t& ci, int lw, int lane,
+                                         Misc* misc, uint32_t it, uint32_t ci, int lw, int lane,
                                          unsigned long long* prof) {
     // The chunks of a stage are adjacent both in the operand buffer and in the stage's slot: one
     // bulk copy per stage, issued by one lane as far ahead as free slots allow.
@@ -212,15 +212,13 @@ __device__ __noinline__ void loader_copy(const FwdParams& P, int kind, const OpD
     }
     __syncwarp();
     if (prof && lw == 0 && lane == 0) prof[5] = global_timer_ns();
-    it = it0 + (uint32_t)(npass * nst);
-    ci += (uint32_t)(npass * pt.nchunks);
 }
 
 // A bounded wait that ran out marks the warp "dead": it stops touching the pipeline but still
 // walks the control flow to the end.
 template <int NT>
 __device__ __noinline__ void loader_norm(const FwdParams& P, int kind, int layer, const OpDesc& od, const Part& pt,
-                                         uint8_t* smem, Misc* misc, uint32_t& it, uint32_t& ci, int lw, int lane,
+                                         uint8_t* smem, Misc* misc, uint32_t it, uint32_t ci, int lw, int lane,
                                          unsigned long long* prof) {
     using SL = SmemLayout<NT>;
     const int KW = 1 << pt.lkw, lkw = pt.lkw;
@@ -334,15 +332,13 @@ __device__ __noinline__ void loader_norm(const FwdParams& P, int kind, int layer
     cp_async_wait<0>();
     if (!published) publish();
     if (prof && lw == 0 && lane == 0) prof[5] = global_timer_ns();
-    it = it0 + (uint32_t)(npass * nst);
-    ci = ci0 + (uint32_t)total;
 }
 
 // ------------------------------------------------------------------------------------------
 // MMA warps.
 template <int NT>
 __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int layer, const OpDesc& od, const Part& pt, uint8_t* smem,
-                               Misc* misc, uint32_t& it, uint32_t& ci, uint32_t& norm_uses, int warp, int lane,
+                               Misc* misc, uint32_t it, uint32_t norm_uses, int warp, int lane,
                                unsigned long long* prof) {
     using SL = SmemLayout<NT>;
     constexpr int MP = SL::MP;
@@ -367,7 +363,6 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
     }
     float* red = reinterpret_cast<float*>(smem + SL::ATT_OFF);  // [8 warps][MP][16] partial tiles (staged epilogue)
     uint64_t wait_w = 0, wait_a = 0, mma_cycles = 0, mma_stages = 0;
-    ci += (uint32_t)(npass * pt.nchunks);
 
     for (int p = 0; p < npass; ++p) {
         const int pcount = pass_count(pt, p);
@@ -527,7 +522,6 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
         prof[10] = mma_cycles;  // SM clock cycles between the waits' end and the slot's release, all stages
         prof[11] = mma_stages;
     }
-    if (need_rstd) ++norm_uses;
 
     if (kind == PH_LM) {
         // best over the 8 row groups of the warp, then over the 8 warps
@@ -570,6 +564,17 @@ __device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int la
 // query rows of the head group to range s; unit (kv head, S) covers the M new rows: it finishes
 // their K/V projection (norm scale, bias, rotary), appends them to the cache and attends to them
 // under the causal mask (row j sees new keys 0..j).  Partial results are merged afterwards.
+//
+// Inside a unit the R = (query heads per KV head) x M rows form MT tiles of 16 rows and the keys
+// come in blocks of KB (64 while the row tile leaves room, else 32).  A block takes three short
+// steps, each spread over all 11 worker warps as independent tasks so that no warp runs a long
+// dependent chain:
+//   A  scores: task (row tile, 16 keys) = Q K^T on tensor cores, scaled and masked, kept in
+//      registers; per-row maxima of the 16 keys go to shared memory;
+//   B  same tasks: block maximum per row from the partial maxima, probabilities exp2(s - m),
+//      written as bf16 over the K block (no longer needed), partial row sums to shared memory;
+//   C  output: task (row tile, 16 head columns) = rescale the running output, add P V.
+// Running maximum, sum and rescale factor per row live in shared memory.
 __device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps) {
     if (P.L <= 0) { S = 0; kps = 0; return; }
     int cap = P.G / P.n_kv - 1;
@@ -579,20 +584,34 @@ __device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps)
     S = (P.L + kps - 1) / kps;
 }
 
-template <int HD>
+constexpr int kAttnStatsOff = 49152;  // row statistics behind the Q | K | V tiles
+
+template <int HD, bool BIG>  // BIG: more than 64 query rows (4 row tiles)
 __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int S, int kps, uint8_t* att, int wtid,
                                             unsigned long long* prof) {
     constexpr int HD2 = HD / 2;
     constexpr int KSTEPS = HD / 16;
-    constexpr int UNITS = HD / 8;  // 16-byte units per K/V row
-    constexpr int UPT = (kAttnBlockKeys * UNITS + kWorkerThreads - 1) / kWorkerThreads;  // units per thread
+    constexpr int UNITS = HD / 8;   // 16-byte units per K/V row
+    constexpr int CG = HD / 16;     // 16-column groups of the output
+    constexpr int NWARPS = kWorkerThreads / 32;
+    constexpr int TA_MAX = 2;                                // score tasks per warp (at most 16 tasks)
+    constexpr int TC_MAX = ((BIG ? 8 : 4) * CG + NWARPS - 1) / NWARPS;  // output tasks per warp
+    constexpr int KB = BIG ? 32 : 64, lng = BIG ? 1 : 2, NG = 1 << lng;  // keys per block; 16-key groups
     const int warp = wtid >> 5, lane = wtid & 31;
     const int M = P.M, L = P.L, R = P.g * M;
     const int MT = (R + 15) >> 4, RP = MT * 16;
     const bool is_new = (s == S);
     uint8_t* Qs = att;
-    uint8_t* Ks = att + 32768;
-    uint8_t* Vs = att + 32768 + 8192;
+    uint8_t* Ks = att + RP * HD * 2;
+    uint8_t* Vs = Ks + KB * HD * 2;
+    // probabilities: over the keys once the scores are done (head_dim 128, where the tiles fill the
+    // region), else in the free space behind the tiles
+    uint8_t* Pb = (HD == 128) ? Ks : att + 32768;
+    float* st_m = reinterpret_cast<float*>(att + kAttnStatsOff);  // [2][128] running maximum, by block parity
+    float* st_l = st_m + 256;                                     // [128] running sum
+    float* st_corr = st_l + 128;                                  // [128] rescale factor of this block
+    float* st_pmax = st_corr + 128;                               // [RP][NG] per-task maxima
+    float* st_psum = st_pmax + 256;                               // [RP][NG] per-task sums
     const float* sumsq = P.sumsq + (layer & 1) * kMaxRows;
     const float* bias = P.bias ? P.bias + (size_t)layer * P.n_qkv : nullptr;
     const int Nq = P.n_q * HD, Nkv = P.n_kv * HD;
@@ -603,39 +622,27 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
         const int t_end = min(L, t_begin + kps);
         nkeys = max(0, t_end - t_begin);
     }
-    const int nblk = (nkeys + kAttnBlockKeys - 1) / kAttnBlockKeys;
+    const int nblk = (nkeys + KB - 1) / KB;
     const size_t cache_row0 = ((size_t)layer * P.n_kv + hk) * P.max_seq;
 
-    // ---- cached keys: the first block's loads are in flight while the query tile is built
-    uint4 kreg[UPT], vreg[UPT];
-    auto issue_block = [&](int blk) {
-#pragma unroll
-        for (int t = 0; t < UPT; ++t) {
-            const int u = wtid + t * kWorkerThreads;
-            const int key = u / UNITS, q16 = u % UNITS, kk = blk * kAttnBlockKeys + key;
-            kreg[t] = make_uint4(0, 0, 0, 0);
-            vreg[t] = make_uint4(0, 0, 0, 0);
-            if (u < kAttnBlockKeys * UNITS && kk < nkeys) {
-                const size_t off = (cache_row0 + t_begin + kk) * HD + q16 * 8;
-                kreg[t] = ldcg_u4(P.kcache + off);
-                vreg[t] = ldcg_u4(P.vcache + off);
-            }
+    // cached keys and values of one block: 16-byte asynchronous copies, rows past the range zero-filled
+    auto load_block = [&](int blk) {
+        for (int u = wtid; u < KB * UNITS; u += kWorkerThreads) {
+            const int key = u / UNITS, q16 = u % UNITS, kk = blk * KB + key;
+            const bool valid = kk < nkeys;
+            const size_t off = (cache_row0 + t_begin + (valid ? kk : 0)) * HD + q16 * 8;
+            const uint32_t so = (q16 >> 3) * (KB * 128) + swz_unit(key, q16 & 7);
+            cp_async_16_zfill(Ks + so, P.kcache + off, valid);
+            cp_async_16_zfill(Vs + so, P.vcache + off, valid);
         }
-    };
-    auto store_block = [&]() {
-#pragma unroll
-        for (int t = 0; t < UPT; ++t) {
-            const int u = wtid + t * kWorkerThreads;
-            if (u < kAttnBlockKeys * UNITS) {
-                const int key = u / UNITS, q16 = u % UNITS;
-                const uint32_t so = (q16 >> 3) * (kAttnBlockKeys * 128) + swz_unit(key, q16 & 7);
-                *reinterpret_cast<uint4*>(Ks + so) = kreg[t];
-                *reinterpret_cast<uint4*>(Vs + so) = vreg[t];
-            }
-        }
+        cp_async_commit();
     };
     if (prof && wtid == 0) prof[2] = global_timer_ns();
-    if (!is_new && nblk > 0) issue_block(0);
+    if (!is_new && nblk > 0) load_block(0);
+    if (wtid < 128) {
+        st_m[wtid] = -CUDART_INF_F;
+        st_l[wtid] = 0.f;
+    }
 
     // ---- query tile: normalise, add bias, rotate, round to bf16; 4 rotary pairs per item
     {
@@ -689,158 +696,217 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
             }
         }
     }
-
-    if (prof && wtid == 0) prof[3] = global_timer_ns();
-    const int g = lane >> 2, q2 = (lane & 3) * 2;
-    const int r_lo = warp * 16 + g, r_hi = r_lo + 8;
-    const int j_lo = r_lo % M, j_hi = r_hi % M;
-    float m_lo = -CUDART_INF_F, m_hi = -CUDART_INF_F, l_lo = 0.f, l_hi = 0.f;
-    float o[HD / 8][4];
+    // the new rows' own keys and values fit one block (M <= 32 <= KB)
+    if (is_new) {
+        // K and V rows of the new tokens: finish the projection, rotate K, append to the cache
+        for (int u = wtid; u < KB * UNITS; u += kWorkerThreads) {
+            const int key = u / UNITS, q16 = u % UNITS, kk = key;
+            uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
+            if (kk < nkeys) {
+                const float rs = rsqrtf(__ldcg(sumsq + kk) / (float)P.d + P.eps);
+                const float* accrow = P.qkv_acc + (size_t)kk * P.n_qkv;
+                const int colb = q16 * 8, ib = colb % HD2;  // 8 columns share one half of the rotary pairing
+                const float* pa = accrow + Nq + hk * HD + ib;
+                const float4 a0 = ldcg_f4(pa), a1 = ldcg_f4(pa + 4), b0 = ldcg_f4(pa + HD2), b1 = ldcg_f4(pa + HD2 + 4);
+                const float* pv = accrow + Nq + Nkv + hk * HD + colb;
+                const float4 v0 = ldcg_f4(pv), v1 = ldcg_f4(pv + 4);
+                const float4* rp = reinterpret_cast<const float4*>(P.rope + (size_t)(L + kk) * HD2 + ib);
+                const float4 r0 = __ldg(rp), r1 = __ldg(rp + 1), r2 = __ldg(rp + 2), r3 = __ldg(rp + 3);
+                float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                float v[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+                const float cs[8] = {r0.x, r0.z, r1.x, r1.z, r2.x, r2.z, r3.x, r3.z};
+                const float sn[8] = {r0.y, r0.w, r1.y, r1.w, r2.y, r2.w, r3.y, r3.w};
+                float kvals[8];
 #pragma unroll
-    for (int n = 0; n < HD / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+                for (int e = 0; e < 8; ++e) {
+                    a[e] *= rs; b[e] *= rs; v[e] *= rs;
+                    if (bias) {
+                        a[e] += bias[Nq + hk * HD + ib + e];
+                        b[e] += bias[Nq + hk * HD + ib + HD2 + e];
+                        v[e] += bias[Nq + Nkv + hk * HD + colb + e];
+                    }
+                    kvals[e] = (colb < HD2) ? (a[e] * cs[e] - b[e] * sn[e]) : (b[e] * cs[e] + a[e] * sn[e]);
+                }
+                kv4 = make_uint4(pack_bf16(kvals[0], kvals[1]), pack_bf16(kvals[2], kvals[3]),
+                                 pack_bf16(kvals[4], kvals[5]), pack_bf16(kvals[6], kvals[7]));
+                vv4 = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]),
+                                 pack_bf16(v[6], v[7]));
+                const size_t off = (cache_row0 + L + kk) * HD + q16 * 8;
+                *reinterpret_cast<uint4*>(P.kcache + off) = kv4;
+                *reinterpret_cast<uint4*>(P.vcache + off) = vv4;
+            }
+            const uint32_t so = (q16 >> 3) * (KB * 128) + swz_unit(key, q16 & 7);
+            *reinterpret_cast<uint4*>(Ks + so) = kv4;
+            *reinterpret_cast<uint4*>(Vs + so) = vv4;
+        }
+    }
+    if (prof && wtid == 0) prof[3] = global_timer_ns();
+
+    const int g = lane >> 2, q2 = (lane & 3) * 2;
+    const int ntaskA = MT << lng, ntaskC = MT * CG;
+    // byte offset of 16-byte unit `unit` of row r in the probability tile (swizzled against bank conflicts)
+    auto p_unit = [&](uint32_t r, uint32_t unit) -> uint32_t {
+        return KB == 64 ? swz_unit(r, unit) : r * 64u + (((unit ^ (r >> 1)) & 3u) << 4);
+    };
+    float o[TC_MAX][2][4];
+#pragma unroll
+    for (int t = 0; t < TC_MAX; ++t)
+#pragma unroll
+        for (int n = 0; n < 2; ++n) o[t][n][0] = o[t][n][1] = o[t][n][2] = o[t][n][3] = 0.f;
 
     for (int blk = 0; blk < nblk; ++blk) {
-        if (is_new) {
-            // K and V rows of the new tokens: finish the projection, rotate K, append to the cache
-            for (int u = wtid; u < kAttnBlockKeys * UNITS; u += kWorkerThreads) {
-                const int key = u / UNITS, q16 = u % UNITS, kk = blk * kAttnBlockKeys + key;
-                uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
-                if (kk < nkeys) {
-                    const float rs = rsqrtf(__ldcg(sumsq + kk) / (float)P.d + P.eps);
-                    const float* accrow = P.qkv_acc + (size_t)kk * P.n_qkv;
-                    const int colb = q16 * 8, ib = colb % HD2;  // 8 columns share one half of the rotary pairing
-                    const float* pa = accrow + Nq + hk * HD + ib;
-                    const float4 a0 = ldcg_f4(pa), a1 = ldcg_f4(pa + 4), b0 = ldcg_f4(pa + HD2), b1 = ldcg_f4(pa + HD2 + 4);
-                    const float* pv = accrow + Nq + Nkv + hk * HD + colb;
-                    const float4 v0 = ldcg_f4(pv), v1 = ldcg_f4(pv + 4);
-                    const float4* rp = reinterpret_cast<const float4*>(P.rope + (size_t)(L + kk) * HD2 + ib);
-                    const float4 r0 = __ldg(rp), r1 = __ldg(rp + 1), r2 = __ldg(rp + 2), r3 = __ldg(rp + 3);
-                    float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-                    float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-                    float v[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-                    const float cs[8] = {r0.x, r0.z, r1.x, r1.z, r2.x, r2.z, r3.x, r3.z};
-                    const float sn[8] = {r0.y, r0.w, r1.y, r1.w, r2.y, r2.w, r3.y, r3.w};
-                    float kvals[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        a[e] *= rs; b[e] *= rs; v[e] *= rs;
-                        if (bias) {
-                            a[e] += bias[Nq + hk * HD + ib + e];
-                            b[e] += bias[Nq + hk * HD + ib + HD2 + e];
-                            v[e] += bias[Nq + Nkv + hk * HD + colb + e];
-                        }
-                        kvals[e] = (colb < HD2) ? (a[e] * cs[e] - b[e] * sn[e]) : (b[e] * cs[e] + a[e] * sn[e]);
-                    }
-                    kv4 = make_uint4(pack_bf16(kvals[0], kvals[1]), pack_bf16(kvals[2], kvals[3]),
-                                     pack_bf16(kvals[4], kvals[5]), pack_bf16(kvals[6], kvals[7]));
-                    vv4 = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]),
-                                     pack_bf16(v[6], v[7]));
-                    const size_t off = (cache_row0 + L + kk) * HD + q16 * 8;
-                    *reinterpret_cast<uint4*>(P.kcache + off) = kv4;
-                    *reinterpret_cast<uint4*>(P.vcache + off) = vv4;
-                }
-                const uint32_t so = (q16 >> 3) * (kAttnBlockKeys * 128) + swz_unit(key, q16 & 7);
-                *reinterpret_cast<uint4*>(Ks + so) = kv4;
-                *reinterpret_cast<uint4*>(Vs + so) = vv4;
-            }
-        } else {
-            store_block();
+        const int par = blk & 1;
+        if (!is_new) {
+            if (blk > 0) load_block(blk);
+            cp_async_wait<0>();
         }
-        named_bar_sync(1, kWorkerThreads);  // K/V block (and, first time, the Q tile) are in place
+        named_bar_sync(1, kWorkerThreads);  // K/V block (and, first time, the Q tile and the row statistics) are in place
         if (prof && wtid == 0 && blk == 0) prof[4] = global_timer_ns();
-        if (!is_new && blk + 1 < nblk) issue_block(blk + 1);
-        if (warp < MT) {
-            // ---- S = Q K^T for 16 rows x 32 keys
-            float sc[4][4];
+
+        // ---- A: scores of (row tile, 16 keys), kept in registers
+        float sc[TA_MAX][2][4];
+        const uint32_t qb = smem_u32(Qs), kb = smem_u32(Ks), vb = smem_u32(Vs), pb = smem_u32(Pb);
 #pragma unroll
-            for (int n = 0; n < 4; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
-            const uint32_t qb = smem_u32(Qs), kb = smem_u32(Ks), vb = smem_u32(Vs);
+        for (int ti = 0; ti < TA_MAX; ++ti) {
+            const int task = warp + ti * NWARPS;
+            if (task >= ntaskA) continue;
+            const int mt = task >> lng, kg = task & (NG - 1);
+#pragma unroll
+            for (int n = 0; n < 2; ++n) sc[ti][n][0] = sc[ti][n][1] = sc[ti][n][2] = sc[ti][n][3] = 0.f;
 #pragma unroll
             for (int ks = 0; ks < KSTEPS; ++ks) {
-                uint32_t a0, a1, a2, a3;
-                ldsm_x4(qb + (ks >> 2) * (RP * 128) + swz_unit(warp * 16 + (lane & 15), (ks & 3) * 2 + (lane >> 4)), a0,
-                        a1, a2, a3);
-#pragma unroll
-                for (int np = 0; np < 2; ++np) {
-                    uint32_t b0, b1, b2, b3;
-                    const int row = np * 16 + (lane & 7) + ((lane >> 4) << 3);
-                    ldsm_x4(kb + (ks >> 2) * (kAttnBlockKeys * 128) + swz_unit(row, (ks & 3) * 2 + ((lane >> 3) & 1)), b0,
-                            b1, b2, b3);
-                    mma_bf16_16816(sc[2 * np], a0, a1, a2, a3, b0, b1);
-                    mma_bf16_16816(sc[2 * np + 1], a0, a1, a2, a3, b2, b3);
-                }
+                uint32_t a0, a1, a2, a3, b0, b1, b2, b3;
+                ldsm_x4(qb + (ks >> 2) * (RP * 128) + swz_unit(mt * 16 + (lane & 15), (ks & 3) * 2 + (lane >> 4)), a0, a1, a2,
+                        a3);
+                const int row = kg * 16 + (lane & 7) + ((lane >> 4) << 3);
+                ldsm_x4(kb + (ks >> 2) * (KB * 128) + swz_unit(row, (ks & 3) * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
+                mma_bf16_16816(sc[ti][0], a0, a1, a2, a3, b0, b1);
+                mma_bf16_16816(sc[ti][1], a0, a1, a2, a3, b2, b3);
             }
-            // ---- mask, online softmax (log2 domain)
+            const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
+            const int j_lo = r_lo % M, j_hi = r_hi % M;
             float mx_lo = -CUDART_INF_F, mx_hi = -CUDART_INF_F;
 #pragma unroll
-            for (int n = 0; n < 4; ++n)
+            for (int n = 0; n < 2; ++n)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const int key = blk * kAttnBlockKeys + n * 8 + q2 + (e & 1);
+                    const int key = blk * KB + kg * 16 + n * 8 + q2 + (e & 1);
                     const bool hi = e >= 2;
                     const int row = hi ? r_hi : r_lo, j = hi ? j_hi : j_lo;
                     const bool ok = key < nkeys && row < R && (!is_new || key <= j);
-                    const float v = ok ? sc[n][e] * P.scale_log2e : -CUDART_INF_F;
-                    sc[n][e] = v;
+                    const float v = ok ? sc[ti][n][e] * P.scale_log2e : -CUDART_INF_F;
+                    sc[ti][n][e] = v;
                     if (hi) mx_hi = fmaxf(mx_hi, v); else mx_lo = fmaxf(mx_lo, v);
                 }
             mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
             mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
             mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
             mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
-            const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
-            const float use_lo = (mn_lo == -CUDART_INF_F) ? 0.f : mn_lo, use_hi = (mn_hi == -CUDART_INF_F) ? 0.f : mn_hi;
-            const float corr_lo = exp2f(m_lo - use_lo), corr_hi = exp2f(m_hi - use_hi);
-            m_lo = mn_lo; m_hi = mn_hi;
-            l_lo *= corr_lo; l_hi *= corr_hi;
-#pragma unroll
-            for (int n = 0; n < HD / 8; ++n) { o[n][0] *= corr_lo; o[n][1] *= corr_lo; o[n][2] *= corr_hi; o[n][3] *= corr_hi; }
-            uint32_t pa[2][4];
-#pragma unroll
-            for (int n = 0; n < 4; ++n) {
-                const float p0 = exp2f(sc[n][0] - use_lo), p1 = exp2f(sc[n][1] - use_lo);
-                const float p2 = exp2f(sc[n][2] - use_hi), p3 = exp2f(sc[n][3] - use_hi);
-                l_lo += p0 + p1; l_hi += p2 + p3;
-                pa[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
-                pa[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
+            if ((lane & 3) == 0) {
+                st_pmax[(r_lo << lng) + kg] = mx_lo;
+                st_pmax[(r_hi << lng) + kg] = mx_hi;
             }
-            // ---- O += P V
+        }
+        named_bar_sync(1, kWorkerThreads);  // partial maxima are visible; the K block has been read
+
+        // ---- B: probabilities
 #pragma unroll
-            for (int kk2 = 0; kk2 < 2; ++kk2) {
+        for (int ti = 0; ti < TA_MAX; ++ti) {
+            const int task = warp + ti * NWARPS;
+            if (task >= ntaskA) continue;
+            const int mt = task >> lng, kg = task & (NG - 1);
+            const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
+            float mb_lo = st_pmax[r_lo << lng], mb_hi = st_pmax[r_hi << lng];
+            for (int i = 1; i < NG; ++i) {
+                mb_lo = fmaxf(mb_lo, st_pmax[(r_lo << lng) + i]);
+                mb_hi = fmaxf(mb_hi, st_pmax[(r_hi << lng) + i]);
+            }
+            const float mo_lo = st_m[par * 128 + r_lo], mo_hi = st_m[par * 128 + r_hi];
+            const float mn_lo = fmaxf(mo_lo, mb_lo), mn_hi = fmaxf(mo_hi, mb_hi);
+            const float use_lo = (mn_lo == -CUDART_INF_F) ? 0.f : mn_lo, use_hi = (mn_hi == -CUDART_INF_F) ? 0.f : mn_hi;
+            float sum_lo = 0.f, sum_hi = 0.f;
 #pragma unroll
-                for (int np = 0; np < HD / 16; ++np) {
-                    uint32_t b0, b1, b2, b3;
-                    const int key = kk2 * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
-                    const int cu = np * 2 + (lane >> 4);
-                    ldsm_x4_trans(vb + (cu >> 3) * (kAttnBlockKeys * 128) + swz_unit(key, cu & 7), b0, b1, b2, b3);
-                    mma_bf16_16816(o[2 * np], pa[kk2][0], pa[kk2][1], pa[kk2][2], pa[kk2][3], b0, b1);
-                    mma_bf16_16816(o[2 * np + 1], pa[kk2][0], pa[kk2][1], pa[kk2][2], pa[kk2][3], b2, b3);
+            for (int n = 0; n < 2; ++n) {
+                const float p0 = exp2f(sc[ti][n][0] - use_lo), p1 = exp2f(sc[ti][n][1] - use_lo);
+                const float p2 = exp2f(sc[ti][n][2] - use_hi), p3 = exp2f(sc[ti][n][3] - use_hi);
+                sum_lo += p0 + p1;
+                sum_hi += p2 + p3;
+                const uint32_t unit = (uint32_t)(kg * 2 + n);
+                *reinterpret_cast<uint32_t*>(Pb + p_unit(r_lo, unit) + q2 * 2) = pack_bf16(p0, p1);
+                *reinterpret_cast<uint32_t*>(Pb + p_unit(r_hi, unit) + q2 * 2) = pack_bf16(p2, p3);
+            }
+            sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 1);
+            sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 2);
+            sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 1);
+            sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 2);
+            if ((lane & 3) == 0) {
+                st_psum[(r_lo << lng) + kg] = sum_lo;
+                st_psum[(r_hi << lng) + kg] = sum_hi;
+                if (kg == 0) {
+                    st_corr[r_lo] = exp2f(mo_lo - use_lo);
+                    st_corr[r_hi] = exp2f(mo_hi - use_hi);
+                    st_m[(par ^ 1) * 128 + r_lo] = mn_lo;
+                    st_m[(par ^ 1) * 128 + r_hi] = mn_hi;
                 }
             }
         }
-        named_bar_sync(1, kWorkerThreads);  // the block has been consumed
+        named_bar_sync(1, kWorkerThreads);  // probabilities, sums and rescale factors are visible
+
+        // ---- C: O = O * corr + P V for (row tile, 16 columns)
+#pragma unroll
+        for (int tj = 0; tj < TC_MAX; ++tj) {
+            const int task = warp + tj * NWARPS;
+            if (task >= ntaskC) continue;
+            const int mt = task / CG, cg = task % CG;
+            const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
+            const float c_lo = st_corr[r_lo], c_hi = st_corr[r_hi];
+#pragma unroll
+            for (int n = 0; n < 2; ++n) { o[tj][n][0] *= c_lo; o[tj][n][1] *= c_lo; o[tj][n][2] *= c_hi; o[tj][n][3] *= c_hi; }
+            for (int k2 = 0; k2 < NG; ++k2) {
+                uint32_t a0, a1, a2, a3, b0, b1, b2, b3;
+                ldsm_x4(pb + p_unit(mt * 16 + (lane & 15), k2 * 2 + (lane >> 4)), a0, a1, a2, a3);
+                const int key = k2 * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+                const int cu = cg * 2 + (lane >> 4);
+                ldsm_x4_trans(vb + (cu >> 3) * (KB * 128) + swz_unit(key, cu & 7), b0, b1, b2, b3);
+                mma_bf16_16816(o[tj][0], a0, a1, a2, a3, b0, b1);
+                mma_bf16_16816(o[tj][1], a0, a1, a2, a3, b2, b3);
+            }
+            if (cg == 0 && (lane & 3) == 0) {
+                float s_lo = 0.f, s_hi = 0.f;
+                for (int i = 0; i < NG; ++i) {
+                    s_lo += st_psum[(r_lo << lng) + i];
+                    s_hi += st_psum[(r_hi << lng) + i];
+                }
+                st_l[r_lo] = st_l[r_lo] * c_lo + s_lo;
+                st_l[r_hi] = st_l[r_hi] * c_hi + s_hi;
+            }
+        }
+        named_bar_sync(1, kWorkerThreads);  // the block has been consumed; row statistics are up to date
     }
 
     // ---- un-normalised partial result of this key range
     if (prof && wtid == 0) prof[5] = global_timer_ns();
-    if (warp < MT) {
-        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
-        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
-        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
-        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+#pragma unroll
+    for (int tj = 0; tj < TC_MAX; ++tj) {
+        const int task = warp + tj * NWARPS;
+        if (task >= ntaskC) continue;
+        const int mt = task / CG, cg = task % CG;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
-            const int r = half ? r_hi : r_lo;
+            const int r = mt * 16 + g + half * 8;
             if (r >= R) continue;
             const int hq = hk * P.g + r / M, j = r % M;
             const size_t row = ((size_t)hq * (kMaxSplits + 1) + s) * kMaxRows + j;
-            float* po = P.part_o + row * HD;
-#pragma unroll
-            for (int n = 0; n < HD / 8; ++n)
-                __stcg(reinterpret_cast<float2*>(po + n * 8 + q2), make_float2(o[n][half * 2], o[n][half * 2 + 1]));
-            if ((lane & 3) == 0)
-                __stcg(reinterpret_cast<float2*>(P.part_ml + row * 2), make_float2(half ? m_hi : m_lo, half ? l_hi : l_lo));
+            float* po = P.part_o + row * HD + cg * 16 + q2;
+            __stcg(reinterpret_cast<float2*>(po), make_float2(o[tj][0][half * 2], o[tj][0][half * 2 + 1]));
+            __stcg(reinterpret_cast<float2*>(po + 8), make_float2(o[tj][1][half * 2], o[tj][1][half * 2 + 1]));
         }
+    }
+    if (wtid < R) {
+        const int hq = hk * P.g + wtid / M, j = wtid % M;
+        const size_t row = ((size_t)hq * (kMaxSplits + 1) + s) * kMaxRows + j;
+        __stcg(reinterpret_cast<float2*>(P.part_ml + row * 2), make_float2(st_m[(nblk & 1) * 128 + wtid], st_l[wtid]));
     }
 }
 
@@ -851,8 +917,14 @@ __device__ void attention_phase(const FwdParams& P, int layer, uint8_t* att, int
     const int nunits = P.n_kv * S1;
     for (int unit = blockIdx.x; unit < nunits; unit += P.G) {
         const int hk = unit / S1, s = unit % S1;
-        if (P.hd == 128) attention_unit<128>(P, layer, hk, s, S, kps, att, wtid, prof);
-        else attention_unit<64>(P, layer, hk, s, S, kps, att, wtid, prof);
+        const bool big = P.g * P.M > 64;
+        if (P.hd == 128) {
+            if (big) attention_unit<128, true>(P, layer, hk, s, S, kps, att, wtid, prof);
+            else attention_unit<128, false>(P, layer, hk, s, S, kps, att, wtid, prof);
+        } else {
+            if (big) attention_unit<64, true>(P, layer, hk, s, S, kps, att, wtid, prof);
+            else attention_unit<64, false>(P, layer, hk, s, S, kps, att, wtid, prof);
+        }
         named_bar_sync(1, kWorkerThreads);  // the unit's shared-memory tiles are free again
         if (prof && wtid == 0) { prof[6] = global_timer_ns(); prof[7] = (unsigned long long)(s == S); }
     }
@@ -1005,12 +1077,16 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
                 unsigned long long* pp =
                     P.prof ? P.prof + ((size_t)(ph - P.ph_begin) * P.G + blockIdx.x) * kProfWords : nullptr;
                 if (warp < kConsumerWarps) {
-                    consumer_phase<NT>(P, kind, layer, od, pt, smem, misc, it, ci, norm_uses, warp, lane, pp);
+                    consumer_phase<NT>(P, kind, layer, od, pt, smem, misc, it, norm_uses, warp, lane, pp);
                 } else {
                     const bool norm = (kind == PH_QKV || kind == PH_GU || kind == PH_LM);
                     if (norm) loader_norm<NT>(P, kind, layer, od, pt, smem, misc, it, ci, warp - kConsumerWarps, lane, pp);
                     else loader_copy<NT>(P, kind, od, pt, smem, misc, it, ci, warp - kConsumerWarps, lane, pp);
                 }
+                // pipeline positions advance identically for every role
+                it += (uint32_t)(pt.npass * pt.nst);
+                ci += (uint32_t)(pt.npass * pt.nchunks);
+                if (kind == PH_GU || kind == PH_LM) ++norm_uses;
             }
         }
         if (P.prof) {

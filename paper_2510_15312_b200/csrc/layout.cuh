@@ -23,9 +23,8 @@ constexpr int kStageWeightBytes = kConsumerWarps * kTileBytes;       // 16 KB
 constexpr int kMaxRows = 32;                                         // token rows a buffer is sized for
 constexpr int kMaxSplits = 40;                                       // KV splits per head (+1 unit for new rows)
 constexpr int kMaxKW = 4;                                             // chunks per stage at most
-constexpr int kAttnBlockKeys = 32;
 constexpr int kSmemBudget = 232448;                                  // 227 KB
-constexpr int kAttnSmemBytes = 32768 + 2 * 8192;                     // Q tile (128 x 128) + K and V blocks
+constexpr int kAttnSmemBytes = 49152 + 4096;                         // Q tile + K and V blocks (48 KB), row statistics
 constexpr int kMiscSmemBytes = 4096;
 constexpr int kMaxDraftWords = 32;
 constexpr int kProfWords = 12;                                       // timestamps per (phase, block)
