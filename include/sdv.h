@@ -190,12 +190,27 @@ int sdv_debug_timeout_probe(sdv_ctx *ctx);
 
 /* Per-phase timing of the forward kernel.  host_out != NULL: copies the timestamps recorded by the
  * last profiled launch, uint64 nanoseconds [n_phases][blocks][12] per thread block: phase work
- * begin, end, first pipeline stage ready, last stage consumed, epilogue done, loaders done, loader
- * entry, first operand chunk stored, total wait for weights, total wait for operands (GEMM phases
- * only; two spare) (phase 0 = embedding, then 6 per layer: qkv, attention, split merge, o, gate|up,
- * down; last = LM head).  Then switches recording on or off for later launches (it adds a block-wide barrier
- * per phase, so timed runs keep it off).  Returns the number of thread blocks, or an error. */
+ * begin, end, token operand built, last tensor-core instruction issued, epilogue done (GEMM
+ * phases; the attention phase uses words 2..7 for its own steps; the rest spare) (phase 0 =
+ * embedding, then 4 per layer: qkv, attention, o, gate|up + down; last = LM head).  Then switches
+ * recording on or off for later launches (it adds a block-wide barrier per phase, so timed runs
+ * keep it off).  Returns the number of thread blocks, or an error. */
 int sdv_debug_profile(sdv_ctx *ctx, int on, unsigned long long *host_out, int n_phases);
+
+/* Host-only self-check of the weight streaming layout (no GPU needed): walks every thread block's
+ * share of an operation the way the kernel does and checks that every 16-byte unit of the matrix
+ * is met exactly once at the offset the packing step writes it to.  desc and gu_desc are
+ * {row tiles, column steps, row partitions, column partitions, tiles per pass, steps per stage,
+ * row granularity, follow flag}; gu_desc (the gate|up operation) is only read when the follow flag
+ * of desc is set.  Returns SDV_OK, SDV_EINVAL for a malformed description, or a code <= -100. */
+int sdv_debug_layout_check(const int *desc, const int *gu_desc, int n_blocks);
+
+/* Host-only: the work partition and the shared-memory plan a context of this configuration uses
+ * with n_blocks thread blocks and `rows` token rows.  out[8 * op + 0..7] as in
+ * sdv_debug_layout_check for QKV, O, gate|up, down, LM head; out[40..45] = row groups of the token
+ * operand, N of the tensor-core instruction, ring slots, operand region bytes, dynamic shared
+ * memory bytes, 1 if the plan fits. */
+int sdv_debug_plan(const sdv_config *cfg, int n_blocks, int rows, int *out);
 
 /* Number of kernels launched by this context since creation. */
 long long sdv_launch_count(const sdv_ctx *ctx);
@@ -217,8 +232,8 @@ int sdv_last_verify_ms(sdv_ctx *ctx, float *ms);
  * cuda_stream is a cudaStream_t (NULL = the default stream); the work is queued on it and the
  * call returns after it has finished (it synchronises that stream).
  *
- * Scratch (the weights in streaming order, the bf16 operand, the accumulators, an error word)
- * lives in a fixed array of about 2.8 MB inside the library's device image, present on every GPU
+ * Scratch (the weights in streaming order, the accumulators, an error word)
+ * lives in a fixed array of about 2.5 MB inside the library's device image, present on every GPU
  * that loads the library for as long as it stays loaded.  Hence the limits: M <= 32, N <= 4096,
  * K <= 4096, N % 16 == 0, K % 64 == 0 and N * K * 2 <= 2 MiB; a larger problem returns
  * SDV_ETOOBIG and touches nothing, a malformed one SDV_EINVAL.  The array keeps whatever the last

@@ -18,7 +18,7 @@ EXPORTS = [
     "sdv_strerror", "sdv_last_cuda_error", "sdv_step_bytes", "sdv_debug_set_history", "sdv_debug_accept",
     "sdv_debug_force_commit", "sdv_debug_read_kv", "sdv_debug_read_hidden", "sdv_debug_gemm",
     "sdv_debug_timeout_probe", "sdv_debug_profile", "sdv_launch_count", "sdv_last_verify_ms",
-    "sdv_gemm_noalloc",
+    "sdv_gemm_noalloc", "sdv_debug_layout_check", "sdv_debug_plan",
 ]
 
 
@@ -86,6 +86,8 @@ def load_library(path: Optional[str] = None):
     L.sdv_launch_count.restype = C.c_longlong
     L.sdv_last_verify_ms.argtypes = [vp, C.POINTER(C.c_float)]
     L.sdv_gemm_noalloc.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp]
+    L.sdv_debug_layout_check.argtypes = [C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_int]
+    L.sdv_debug_plan.argtypes = [C.POINTER(SdvConfig), C.c_int, C.c_int, C.POINTER(C.c_int)]
     for name in EXPORTS:
         if name not in ("sdv_workspace_bytes", "sdv_strerror", "sdv_launch_count"):
             getattr(L, name).restype = C.c_int
@@ -276,6 +278,23 @@ class Sdv:
 
     def debug_timeout_probe(self) -> int:
         return lib().sdv_debug_timeout_probe(self._h)
+
+
+def layout_check(desc: Sequence[int], gu_desc: Sequence[int], n_blocks: int) -> int:
+    """Host-only layout self-check (no GPU): returns the library's status code."""
+    a = (C.c_int * 8)(*desc)
+    b = (C.c_int * 8)(*gu_desc)
+    return lib().sdv_debug_layout_check(a, b, n_blocks)
+
+
+def plan(cconfig: SdvConfig, n_blocks: int, rows: int):
+    """Host-only: ([8 ints per operation] x 5, [NG, NB, ring slots, operand bytes, smem bytes, ok])."""
+    out = (C.c_int * 48)()
+    rc = lib().sdv_debug_plan(C.byref(cconfig), n_blocks, rows, out)
+    if rc != OK:
+        raise SdvError(rc, "sdv_debug_plan")
+    v = list(out)
+    return [v[i * 8:(i + 1) * 8] for i in range(5)], v[40:46]
 
 
 def gemm_noalloc(x, w_bits, y, stream=None) -> int:

@@ -1,4 +1,4 @@
-// The persistent forward kernel: one launch runs the decoder over M <= 8*NT token rows
+// The persistent forward kernel: one launch runs the decoder over M <= 32 token rows
 // (a verify step over [T, x_1..x_k], or one tile of a prefill chunk).
 //
 // One thread block per SM, 12 warps:
@@ -6,13 +6,18 @@
 //                and keeps a ring of 16 KB shared-memory stages full with bulk asynchronous copies.
 //                It never waits for activations or grid barriers, only for free ring slots, so HBM
 //                traffic continues across operation boundaries.
-//   warps 8..10  activation loaders: fill each stage's bf16 operand chunks ([rows x 64] each) from
-//                L2, two chunks in flight per warp, applying the RMSNorm scale where one is due.
-//   warps 0..7   MMA warps in an RW x KW grid: warp (rw, kw) multiplies row tile rw of the stage by
-//                operand chunk kw (weights are the MMA "A" operand, token rows the 8-wide "B"
-//                operand); epilogues are fused per operation.
-// Operations are separated by a bounded grid barrier; attention and the split-KV merge use all 11
-// non-producer warps.
+//   warp 10      its lane 0 issues the tensor-core instructions (tcgen05.mma, M = 128 weight rows
+//                x N = 16 or 32 token rows x K = 16 per instruction): the streamed stage is the A
+//                operand, the token rows, resident in shared memory for the whole operation, the
+//                B operand; accumulators live in tensor memory (two buffers, so the next pass
+//                starts while the previous one is read out).
+//   warps 0..3   read the accumulators back (tcgen05.ld) and run the fused epilogues.
+//   warps 0..10  together build the token operand at the start of an operation (RMSNorm scale,
+//                merge of the split-KV partial results, ...) and run the attention step.
+// A layer is four operations separated by a bounded grid barrier: QKV projection; attention;
+// output projection (+ residual); gate|up with SwiGLU followed, inside the same block and without
+// a barrier, by the slice of the down projection (+ residual) that consumes this block's SwiGLU
+// columns.
 #pragma once
 #include <math_constants.h>
 
@@ -21,11 +26,11 @@
 
 namespace sdv {
 
-enum PhaseKind { PH_EMBED = 0, PH_QKV, PH_ATTN, PH_COMB, PH_O, PH_GU, PH_DOWN, PH_LM, PH_RAW };
-constexpr int kPhasesPerLayer = 6;
+enum PhaseKind { PH_EMBED = 0, PH_QKV, PH_ATTN, PH_O, PH_GUD, PH_LM, PH_RAW };
+constexpr int kPhasesPerLayer = 4;
 
-// Phase numbering of a launch: 0 = embedding; 1 + 6*layer + {0..5} = QKV, attention, split merge,
-// output projection, gate|up, down; 1 + 6*n_layers = LM head; 2 + 6*n_layers = stand-alone GEMM.
+// Phase numbering of a launch: 0 = embedding; 1 + 4*layer + {0..3} = QKV, attention, output
+// projection, gate|up + down; 1 + 4*n_layers = LM head; 2 + 4*n_layers = stand-alone GEMM.
 __host__ __device__ __forceinline__ int decode_phase(int ph, int n_layers, int& layer) {
     layer = 0;
     if (ph == 0) return PH_EMBED;
@@ -34,59 +39,47 @@ __host__ __device__ __forceinline__ int decode_phase(int ph, int n_layers, int& 
     layer = (ph - 1) / kPhasesPerLayer;
     return PH_QKV + (ph - 1) % kPhasesPerLayer;
 }
-__device__ __forceinline__ int phase_op(int kind) {
+// The one or two streamed operations of a phase, in streaming order.
+__device__ __forceinline__ int phase_ops(int kind, int (&ops)[2]) {
     switch (kind) {
-        case PH_QKV: return OP_QKV;
-        case PH_O: return OP_O;
-        case PH_GU: return OP_GU;
-        case PH_DOWN: return OP_DOWN;
-        case PH_LM: return OP_LM;
-        case PH_RAW: return OP_RAW;
-        default: return -1;
+        case PH_QKV: ops[0] = OP_QKV; return 1;
+        case PH_O: ops[0] = OP_O; return 1;
+        case PH_GUD: ops[0] = OP_GU; ops[1] = OP_DOWN; return 2;
+        case PH_LM: ops[0] = OP_LM; return 1;
+        case PH_RAW: ops[0] = OP_RAW; return 1;
+        default: return 0;
     }
 }
-__device__ __forceinline__ const uint8_t* op_weights(const FwdParams& P, int kind, int layer) {
-    if (kind == PH_LM) return P.wlm + P.op[OP_LM].w_off;
-    if (kind == PH_RAW) return P.wraw + P.op[OP_RAW].w_off;
-    return P.wlayers + (unsigned long long)layer * P.layer_stride + P.op[phase_op(kind)].w_off;
+__device__ __forceinline__ const uint8_t* op_weights(const FwdParams& P, int op, int layer) {
+    if (op == OP_LM) return P.wlm + P.op[OP_LM].w_off;
+    if (op == OP_RAW) return P.wraw + P.op[OP_RAW].w_off;
+    return P.wlayers + (unsigned long long)layer * P.layer_stride + P.op[op].w_off;
 }
 
-template <int NT>
-struct SmemLayout {
-    static constexpr int MP = 8 * NT;
-    static constexpr int A_CHUNK = MP * 128;
-    static constexpr int A_STAGE = kMaxKW * A_CHUNK;
-    static constexpr int NSTAGE =
-        (kSmemBudget - 1024 - kAttnSmemBytes - kMiscSmemBytes) / (kStageWeightBytes + A_STAGE);
-    static constexpr int W_OFF = 0;
-    static constexpr int A_OFF = NSTAGE * kStageWeightBytes;
-    static constexpr int ATT_OFF = A_OFF + NSTAGE * A_STAGE;
-    static constexpr int MISC_OFF = ATT_OFF + kAttnSmemBytes;
-    static constexpr int TOTAL = MISC_OFF + kMiscSmemBytes + 1024;  // + slack for 1024-byte alignment
-};
-
 struct Misc {
-    uint64_t full_w[16], full_a[16], empty[16];
-    uint64_t rstd_bar;
+    uint64_t full[kMaxStages], empty[kMaxStages];
+    uint64_t tmem_full[2], tmem_empty[2];
+    uint64_t act_ready;   // the SwiGLU operand of this block is complete (one arrival per epilogue warp)
+    uint64_t done_bar;    // last tensor-core instruction of the launch has completed
+    uint32_t tmem_base;
     int abort_flag;
     int skip;  // block-uniform copy of abort_flag, refreshed inside every grid barrier
-    float ss_part[4][kMaxRows];
-    float best_v[kConsumerWarps][kMaxRows];
-    int best_i[kConsumerWarps][kMaxRows];
+    float sumsq[kMaxRows];  // sums of squares of the residual rows (this block's operand columns)
+    float best_v[kEpilogueWarps][kMaxRows];
+    int best_i[kEpilogueWarps][kMaxRows];
     Part part[OP_COUNT];  // this block's share of every operation
-    FwdParams P;  // block-local copy of the launch parameters (cheap to reach from out-of-line code)
+    FwdParams P;          // block-local copy of the launch parameters
 };
 static_assert(sizeof(Misc) <= kMiscSmemBytes, "misc shared memory");
 
 // ------------------------------------------------------------------------------------------
-// Grid barrier: every block adds one to a counter and waits (bounded) until all have.
-// Called by all worker threads.  Returns, identically for all of them, whether some bounded
+// Grid barrier: every block adds one to a counter (release) and waits (bounded, acquire) until all
+// have.  Called by all worker threads.  Returns, identically for all of them, whether some bounded
 // wait in this block has been abandoned (the remaining phases then do no work).
 __device__ __forceinline__ bool grid_barrier(const FwdParams& P, int target, Misc* misc, int wtid) {
     named_bar_sync(1, kWorkerThreads);
     if (wtid == 0) {
-        __threadfence();
-        red_add_s32(P.bar, 1);  // no return value to wait for: polling starts at once
+        red_release_add_s32(P.bar, 1);  // no return value to wait for: polling starts at once
         const uint64_t t0 = global_timer_ns();
         uint32_t spins = 0;
         while ((int)(ld_acquire_gpu(P.bar) - target) < 0) {
@@ -98,7 +91,6 @@ __device__ __forceinline__ bool grid_barrier(const FwdParams& P, int target, Mis
                 }
             }
         }
-        __threadfence();
         *(volatile int*)&misc->skip = *(volatile int*)&misc->abort_flag;
     }
     named_bar_sync(1, kWorkerThreads);
@@ -107,51 +99,46 @@ __device__ __forceinline__ bool grid_barrier(const FwdParams& P, int target, Mis
 
 // ------------------------------------------------------------------------------------------
 // Weight streamer (one thread).
-template <int NT>
 __device__ __noinline__ void producer_loop(const FwdParams& P, uint8_t* smem, Misc* misc) {
-    using SL = SmemLayout<NT>;
     const uint64_t policy = l2_policy_evict_first();
-    uint32_t it = 0;
-    const uint32_t ahead = (P.ahead >= 1 && P.ahead <= SL::NSTAGE) ? (uint32_t)P.ahead : (uint32_t)SL::NSTAGE;
+    const uint32_t nstage = (uint32_t)P.nstage;
+    uint32_t slot = 0, par = 0, issued = 0;  // ring position; parity of the current trip round the ring
     bool ok = true;
     for (int ph = P.ph_begin; ph < P.ph_end && ok; ++ph) {
-        int layer;
+        int layer, ops[2];
         const int kind = decode_phase(ph, P.n_layers, layer);
-        const int op = phase_op(kind);
-        if (op < 0) continue;
-        const Part& pt = misc->part[op];
-        if (pt.ntiles == 0) continue;
-        const int KW = 1 << pt.lkw;
-        const uint8_t* src = op_weights(P, kind, layer) + pt.off;
-        const int npass = pt.npass, nst = pt.nst;
-        for (int p = 0; p < npass && ok; ++p) {
-            const int pcount = pass_count(pt, p);
-            for (int st = 0; st < nst; ++st, ++it) {
-                const int kcnt = min(KW, pt.nchunks - st * KW);
-                const uint32_t bytes = (uint32_t)(pcount * kcnt) * kTileBytes;
-                const uint32_t slot = it % SL::NSTAGE;
-                // run at most `ahead` stages in front of the MMA warps: stage it - ahead must be consumed
-                if (it >= ahead) {
-                    const uint32_t j = it - ahead;
-                    if (!mbar_wait_bounded(&misc->empty[j % SL::NSTAGE], (j / SL::NSTAGE) & 1, &misc->abort_flag,
-                                           P.wait_limit_ns)) {
+        const int nops = phase_ops(kind, ops);
+        for (int oi = 0; oi < nops && ok; ++oi) {
+            const Part& pt = misc->part[ops[oi]];
+            if (pt.ntiles == 0 || pt.nk == 0) continue;
+            const uint8_t* src = op_weights(P, ops[oi], layer) + pt.off;
+            const int nst = pt.nst, SK = pt.SK, nk = pt.nk;
+            for (int p = 0; p < pt.npass && ok; ++p) {
+                const uint32_t pbytes = (uint32_t)pass_count(pt, p) * kStepBytes;
+                int kleft = nk;
+                for (int st = 0; st < nst; ++st, kleft -= SK) {
+                    const uint32_t bytes = pbytes * (uint32_t)min(SK, kleft);
+                    // the slot's previous contents must have been consumed (first trip: free at once)
+                    if (!mbar_wait_bounded(&misc->empty[slot], par ^ 1u, &misc->abort_flag, P.wait_limit_ns)) {
                         ok = false;
                         break;
                     }
+                    mbar_arrive_expect_tx(&misc->full[slot], bytes);
+                    bulk_g2s(smem + slot * kStageBytes, src, bytes, &misc->full[slot], policy);
+                    src += bytes;
+                    ++issued;
+                    if (++slot == nstage) { slot = 0; par ^= 1u; }
                 }
-                mbar_arrive_expect_tx(&misc->full_w[slot], bytes);
-                bulk_g2s(smem + SL::W_OFF + slot * kStageWeightBytes, src, bytes, &misc->full_w[slot], policy);
-                src += bytes;
             }
         }
     }
     if (!ok) {
         // Abandoned: wait (bounded) for the copies still in flight before the block may exit.
-        const uint32_t issued = it;
-        for (uint32_t back = 0; back < (uint32_t)SL::NSTAGE && back < issued; ++back) {
-            const uint32_t j = issued - 1 - back;
+        for (uint32_t back = 0; back < nstage && back < issued; ++back) {
+            if (slot == 0) { slot = nstage; par ^= 1u; }
+            --slot;
             const uint64_t t0 = global_timer_ns();
-            while (!mbar_try_wait(&misc->full_w[j % SL::NSTAGE], (j / SL::NSTAGE) & 1)) {
+            while (!mbar_try_wait(&misc->full[slot], par)) {
                 if (global_timer_ns() - t0 > P.wait_limit_ns) break;
             }
         }
@@ -159,422 +146,363 @@ __device__ __noinline__ void producer_loop(const FwdParams& P, uint8_t* smem, Mi
 }
 
 // ------------------------------------------------------------------------------------------
-// Activation loaders.  The operand chunks ([rows x 64] bf16 each) of a phase are dealt round-robin
-// to the three loader warps.
-//  - Ready-made operands (SwiGLU output, merged attention output) are already stored chunk by
-//    chunk in the shared-memory image: one lane issues a bulk asynchronous copy per chunk straight
-//    into the stage's slot, as far ahead as free slots allow.
-//  - Operands that still need the RMSNorm scale: the chunk's fp32 residual rows and norm weights
-//    are first staged in shared memory by 16-byte asynchronous copies (up to three chunks in flight
-//    per warp, no registers held), then scaled, rounded to bf16 and stored into the slot.  The
-//    row sums of squares fall out of the first pass.
-constexpr int kRedBytes = 16384;  // staged-epilogue buffer at the start of the attention region
-constexpr int kStageBufBytes = (kAttnSmemBytes - kRedBytes) / kLoaderWarps / 256 * 256;
-
-__device__ __forceinline__ uint32_t chunk_arrivals(int c, int nchunks, int KW) {
-    uint32_t cnt = kMaxKW / KW;
-    if (c == nchunks - 1) cnt *= (uint32_t)(KW - ((nchunks - 1) & (KW - 1)));  // the last chunk covers a ragged stage
-    return cnt;
+// Token operand of a GEMM, resident in shared memory for the whole operation, in a layout the
+// tensor core reads (K-major, no swizzle): for every 8 columns the M token rows, 16 bytes each:
+//     [8-column group][row 0..M-1][8 bf16].
+// An 8-row core matrix is 128 contiguous bytes, row groups are 128 bytes apart and the two halves
+// of a column step M * 16 bytes.  The instruction reads 16 or 32 rows: the ones past M belong to the
+// next column groups (or lie behind the operand, still inside shared memory) and only feed
+// accumulator columns nobody reads.
+__device__ __forceinline__ uint32_t operand_off(int k8, int row, int M) {
+    return (uint32_t)((k8 * M + row) * 16);
 }
 
-template <int NT>
-__device__ __noinline__ void loader_copy(const FwdParams& P, int kind, const OpDesc& od, const Part& pt, uint8_t* smem,
-                                         Misc* misc, uint32_t it, uint32_t ci, int lw, int lane,
-                                         unsigned long long* prof) {
-    // The chunks of a stage are adjacent both in the operand buffer and in the stage's slot: one
-    // bulk copy per stage, issued by one lane as far ahead as free slots allow.
-    using SL = SmemLayout<NT>;
-    const int KW = 1 << pt.lkw;
-    const int npass = pt.npass, nst = pt.nst;
-    const uint8_t* src_op = (kind == PH_O) ? P.attn_op : P.act;
-    const uint32_t it0 = it;
-    if (prof && lw == 0 && lane == 0) prof[6] = global_timer_ns();
-    if (lw == 0 && lane == 0) {
-        bool dead = *(volatile int*)&misc->abort_flag != 0;
-        uint32_t sidx = it0;
-        for (int p = 0; p < npass && !dead; ++p) {
-            for (int st = 0; st < nst; ++st, ++sidx) {
-                const uint32_t slot = sidx % SL::NSTAGE, use = sidx / SL::NSTAGE;
-                if (use > 0 &&
-                    !mbar_wait_bounded(&misc->empty[slot], (use - 1) & 1, &misc->abort_flag, P.wait_limit_ns)) {
-                    dead = true;
-                    break;
+// Operand = residual rows scaled by the RMSNorm weight (the per-row factor rsqrt(mean + eps)
+// commutes with the GEMM and is applied by the consumer of the result), or, for the stand-alone
+// GEMM, the caller's fp32 rows as they are.  Warp w converts rows w, w + 11, ...; all loads of a
+// batch are issued before the first use.  Leaves the rows' sums of squares over this block's
+// columns in misc->sumsq; QKV blocks of row partition 0 also add them to the global sums the
+// attention step reads.
+__device__ __noinline__ void build_norm_operand(const FwdParams& P, int kind, int layer, const Part& pt, uint8_t* U,
+                                                Misc* misc, int wtid) {
+    constexpr int UB = 12;  // 4-column units per lane and batch; a warp instruction reads 512 contiguous bytes
+    const int warp = wtid >> 5, lane = wtid & 31;
+    const int M = P.M;
+    const int k4_0 = pt.k0 * 4, nk4 = pt.nk * 4;
+    const bool raw = (kind == PH_RAW);
+    const int stride = raw ? P.raw_K : P.d;
+    const float* xbase = raw ? P.raw_x : P.h;
+    const float* wn = raw ? nullptr
+                          : P.norm_w + (size_t)(kind == PH_QKV ? layer * 2 : (kind == PH_GUD ? layer * 2 + 1 : P.n_layers * 2)) * P.d;
+    for (int row = warp; row < M; row += kWorkerWarps) {
+        const float4* src = reinterpret_cast<const float4*>(xbase + (size_t)row * stride) + k4_0;
+        const float4* wsrc = wn ? reinterpret_cast<const float4*>(wn) + k4_0 : nullptr;
+        float ss = 0.f;
+        for (int base = lane; base < nk4; base += 32 * UB) {
+            float4 a[UB], w[UB];
+#pragma unroll
+            for (int u = 0; u < UB; ++u) {
+                const int k4 = base + u * 32;
+                a[u] = w[u] = make_float4(1.f, 1.f, 1.f, 1.f);
+                if (k4 < nk4) {
+                    a[u] = ld_cg_f4_inorder(src + k4);
+                    if (wsrc) w[u] = ld_nc_f4_inorder(wsrc + k4);
                 }
-                const int kcnt = min(KW, pt.nchunks - st * KW);
-                const uint32_t bytes = (uint32_t)kcnt * SL::A_CHUNK;
-                mbar_arrive_cnt(&misc->full_a[slot], kMaxKW - 1);
-                mbar_arrive_expect_tx(&misc->full_a[slot], bytes);
-                bulk_g2s_plain(smem + SL::A_OFF + slot * SL::A_STAGE,
-                               src_op + (size_t)(pt.chunk0 + st * KW) * SL::A_CHUNK, bytes, &misc->full_a[slot]);
-                if (prof && sidx == it0) prof[7] = global_timer_ns();
+            }
+#pragma unroll
+            for (int u = 0; u < UB; ++u) {
+                const int k4 = base + u * 32;
+                if (k4 < nk4) {
+                    const float4 x = a[u];
+                    ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+                    const uint2 out = make_uint2(pack_bf16(x.x * w[u].x, x.y * w[u].y), pack_bf16(x.z * w[u].z, x.w * w[u].w));
+                    *reinterpret_cast<uint2*>(U + operand_off(k4 >> 1, row, M) + (k4 & 1) * 8) = out;
+                }
             }
         }
+#pragma unroll
+        for (int off = 16; off; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+        if (lane == 0) {
+            misc->sumsq[row] = ss;
+            if (kind == PH_QKV && pt.pr == 0) atomicAdd(P.sumsq + (layer & 1) * kMaxRows + row, ss);
+        }
     }
-    __syncwarp();
-    if (prof && lw == 0 && lane == 0) prof[5] = global_timer_ns();
 }
 
-// A bounded wait that ran out marks the warp "dead": it stops touching the pipeline but still
-// walks the control flow to the end.
-template <int NT>
-__device__ __noinline__ void loader_norm(const FwdParams& P, int kind, int layer, const OpDesc& od, const Part& pt,
-                                         uint8_t* smem, Misc* misc, uint32_t it, uint32_t ci, int lw, int lane,
-                                         unsigned long long* prof) {
-    using SL = SmemLayout<NT>;
-    const int KW = 1 << pt.lkw, lkw = pt.lkw;
-    const int npass = pt.npass, nst = pt.nst;
-    const int nchunks = pt.nchunks;
-    const int M = P.M, d = P.d;
-    const float* wn = P.norm_w + (size_t)(kind == PH_QKV ? layer * 2 : (kind == PH_GU ? layer * 2 + 1 : P.n_layers * 2)) * d;
-    const float* hbase = P.h;
-    float ss[2 * NT];
-#pragma unroll
-    for (int i = 0; i < 2 * NT; ++i) ss[i] = 0.f;
-    bool dead = *(volatile int*)&misc->abort_flag != 0;
-    const uint32_t it0 = it, ci0 = ci;
-    const int total = npass * nchunks;  // chunk visits of this phase, pass-major
-    const int x0 = (int)((lw + kLoaderWarps - (ci0 % kLoaderWarps)) % kLoaderWarps);
-    const int nmine = (x0 < total) ? (total - x0 + kLoaderWarps - 1) / kLoaderWarps : 0;
-    const int entry = (M + 1) * 256;  // M rows of 64 floats, then the 64 norm weights
-    int D = kStageBufBytes / entry;
-    if (D > 3) D = 3;
-    if (D < 1) D = 1;
-    uint8_t* stage = smem + SL::ATT_OFF + kRedBytes + lw * kStageBufBytes;
-    if (prof && lw == 0 && lane == 0) prof[6] = global_timer_ns();
+__device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps);
 
-    int ic = x0;  // chunk index (within the partition) of the next visit to issue, kept below nchunks
-    while (ic >= nchunks) ic -= nchunks;
-    auto issue = [&](int k) {
-        if (k < nmine) {
-            const int chunk = pt.chunk0 + ic;
-            ic += kLoaderWarps;
-            while (ic >= nchunks) ic -= nchunks;
-            uint8_t* dst = stage + (k % D) * entry;
-            const int units = (M + 1) * 16;
-            for (int u = lane; u < units; u += 32) {
-                const int row = u >> 4, part = u & 15;
-                const float* src = (row < M ? hbase + (size_t)row * d : wn) + chunk * 64 + part * 4;
-                cp_async_16(dst + u * 16, src);
-            }
-        }
-        cp_async_commit();  // possibly empty: keeps the group count uniform
-    };
-    auto publish = [&]() {
-        // this warp's share of the per-row sums of squares (its first-pass chunks)
+// Operand of the output projection = attention output of this block's columns: the split-KV
+// partial results (un-normalised sums with their running maximum and sum) are merged on the way.
+// Four lanes share one (row, 8 columns) item, each taking every fourth partial result.
+__device__ __noinline__ void build_merged_operand(const FwdParams& P, const Part& pt, uint8_t* U, int wtid) {
+    constexpr int TPL = (kMaxSplits + 1 + 3) / 4;  // partial results per lane at most
+    int S, kps;
+    attn_split(P, S, kps);
+    const int S1 = S + 1;
+    const int M = P.M, hd = P.hd;
+    const int k8_0 = pt.k0 * 2, nk8 = pt.nk * 2;
+    const int nitems = M * nk8, sub = wtid & 3;
+    for (int it0 = 0; it0 < nitems; it0 += kWorkerThreads / 4) {
+        const int item = it0 + (wtid >> 2);
+        const bool live = item < nitems;
+        const int j = live ? item / nk8 : 0, k8l = live ? item % nk8 : 0;
+        const int col = (k8_0 + k8l) * 8, hq = col / hd, c = col % hd;
+        const size_t base = ((size_t)hq * (kMaxSplits + 1)) * kMaxRows + j;
+        float m[TPL], l[TPL];
+        float4 a[TPL], b[TPL];
 #pragma unroll
-        for (int i = 0; i < 2 * NT; ++i) {
-            float v = ss[i];
-            v += __shfl_xor_sync(0xffffffffu, v, 1);
-            v += __shfl_xor_sync(0xffffffffu, v, 2);
-            v += __shfl_xor_sync(0xffffffffu, v, 4);
-            const int tok = (lane + 32 * i) >> 3;
-            if ((lane & 7) == 0) {
-                if (kind == PH_QKV) {
-                    // the attention step normalises q, k, v; only one row partition reports
-                    if (pt.pr == 0 && tok < M && !dead) atomicAdd(P.sumsq + (layer & 1) * kMaxRows + tok, v);
-                } else {
-                    misc->ss_part[lw][tok] = v;
-                }
+        for (int t = 0; t < TPL; ++t) {
+            const int s = sub + 4 * t;
+            m[t] = -CUDART_INF_F;
+            l[t] = 0.f;
+            a[t] = b[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (live && s < S1) {
+                const size_t row = base + (size_t)s * kMaxRows;
+                const float2 ml = ld_cg_f2_inorder(P.part_ml + row * 2);
+                m[t] = ml.x;
+                l[t] = ml.y;
+                const float* op = P.part_o + row * hd + c;
+                a[t] = ld_cg_f4_inorder(op);
+                b[t] = ld_cg_f4_inorder(op + 4);
             }
         }
-        if (kind != PH_QKV) {
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&misc->rstd_bar);
-        }
-    };
-
-    bool published = false;
-    if (x0 >= nchunks) { publish(); published = true; }  // no first-pass chunk falls to this warp
-    for (int k = 0; k < D; ++k) issue(k);
-    int p_ = 0, c_ = x0;
-    for (int k = 0; k < nmine; ++k, c_ += kLoaderWarps) {
-        const int x = x0 + k * kLoaderWarps;
-        while (c_ >= nchunks) { c_ -= nchunks; ++p_; }
-        if (D == 3) cp_async_wait<2>(); else if (D == 2) cp_async_wait<1>(); else cp_async_wait<0>();
-        __syncwarp();
-        const uint32_t sidx = it0 + (uint32_t)(p_ * nst + (c_ >> lkw));
-        const uint32_t slot = sidx % SL::NSTAGE, use = sidx / SL::NSTAGE;
-        if (!dead && use > 0) {
-            const bool got = mbar_wait_bounded(&misc->empty[slot], (use - 1) & 1, &misc->abort_flag, P.wait_limit_ns);
-            if (!__all_sync(0xffffffffu, got)) dead = true;
-        }
-        if (!dead) {
-            const uint8_t* src = stage + (k % D) * entry;
-            uint8_t* dst = smem + SL::A_OFF + slot * SL::A_STAGE + (c_ & (KW - 1)) * SL::A_CHUNK;
-            const int q = lane & 7;
-            const float4 w0 = *reinterpret_cast<const float4*>(src + M * 256 + q * 32);
-            const float4 w1 = *reinterpret_cast<const float4*>(src + M * 256 + q * 32 + 16);
+        float mmax = m[0];
 #pragma unroll
-            for (int i = 0; i < 2 * NT; ++i) {
-                const int tok = (lane + 32 * i) >> 3;
-                uint4 out = make_uint4(0, 0, 0, 0);
-                if (tok < M) {
-                    const float4 a = *reinterpret_cast<const float4*>(src + tok * 256 + q * 32);
-                    const float4 b = *reinterpret_cast<const float4*>(src + tok * 256 + q * 32 + 16);
-                    if (p_ == 0)
-                        ss[i] += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w + b.x * b.x + b.y * b.y + b.z * b.z +
-                                 b.w * b.w;
-                    out.x = pack_bf16(a.x * w0.x, a.y * w0.y);
-                    out.y = pack_bf16(a.z * w0.z, a.w * w0.w);
-                    out.z = pack_bf16(b.x * w1.x, b.y * w1.y);
-                    out.w = pack_bf16(b.z * w1.z, b.w * w1.w);
-                }
-                *reinterpret_cast<uint4*>(dst + swz_unit(tok, q)) = out;
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cnt(&misc->full_a[slot], chunk_arrivals(c_, nchunks, KW));
-            if (prof && k == 0 && lw == 0 && lane == 0) prof[7] = global_timer_ns();
+        for (int t = 1; t < TPL; ++t) mmax = fmaxf(mmax, m[t]);
+        mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, 1));
+        mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, 2));
+        const float ref = (mmax == -CUDART_INF_F) ? 0.f : mmax;
+        float v[9];
+#pragma unroll
+        for (int e = 0; e < 9; ++e) v[e] = 0.f;
+#pragma unroll
+        for (int t = 0; t < TPL; ++t) {
+            const float w = exp2f(m[t] - ref);  // 0 for partial results that saw no key
+            v[0] += w * a[t].x; v[1] += w * a[t].y; v[2] += w * a[t].z; v[3] += w * a[t].w;
+            v[4] += w * b[t].x; v[5] += w * b[t].y; v[6] += w * b[t].z; v[7] += w * b[t].w;
+            v[8] += w * l[t];
         }
-        __syncwarp();   // every lane is done with the staging entry before it is refilled
-        issue(k + D);
-        if (!published && x + kLoaderWarps >= nchunks) { publish(); published = true; }
+#pragma unroll
+        for (int e = 0; e < 9; ++e) {
+            v[e] += __shfl_xor_sync(0xffffffffu, v[e], 1);
+            v[e] += __shfl_xor_sync(0xffffffffu, v[e], 2);
+        }
+        if (live && sub == 0) {
+            const float inv = 1.f / v[8];
+            const uint4 out = make_uint4(pack_bf16(v[0] * inv, v[1] * inv), pack_bf16(v[2] * inv, v[3] * inv),
+                                         pack_bf16(v[4] * inv, v[5] * inv), pack_bf16(v[6] * inv, v[7] * inv));
+            *reinterpret_cast<uint4*>(U + operand_off(k8l, j, M)) = out;
+        }
     }
-    cp_async_wait<0>();
-    if (!published) publish();
-    if (prof && lw == 0 && lane == 0) prof[5] = global_timer_ns();
 }
 
 // ------------------------------------------------------------------------------------------
-// MMA warps.
-template <int NT>
-__device__ __noinline__ void consumer_phase(const FwdParams& P, int kind, int layer, const OpDesc& od, const Part& pt, uint8_t* smem,
-                               Misc* misc, uint32_t it, uint32_t norm_uses, int warp, int lane,
-                               unsigned long long* prof) {
-    using SL = SmemLayout<NT>;
-    constexpr int MP = SL::MP;
-    const int RW = od.RW, KW = 1 << pt.lkw;
-    const int rw = warp & (RW - 1), kw = warp >> (3 - pt.lkw);
-    const int npass = pt.npass, nst = pt.nst;
-    const int g = lane >> 2, q2 = (lane & 3) * 2;
-    const bool need_rstd = (kind == PH_GU || kind == PH_LM);
-    const bool staged = (kind == PH_QKV || kind == PH_O || kind == PH_DOWN || kind == PH_RAW);
-    float rstd[NT][2];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) rstd[nt][0] = rstd[nt][1] = 0.f;
-    bool have_rstd = false;
-    bool dead = *(volatile int*)&misc->abort_flag != 0;
-    // running arg-max for the LM head: token slots (nt, e)
-    float bv[NT][2];
-    int bi[NT][2];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-        bv[nt][0] = bv[nt][1] = -CUDART_INF_F;
-        bi[nt][0] = bi[nt][1] = 0x7fffffff;
-    }
-    float* red = reinterpret_cast<float*>(smem + SL::ATT_OFF);  // [8 warps][MP][16] partial tiles (staged epilogue)
-    uint64_t wait_w = 0, wait_a = 0, mma_cycles = 0, mma_stages = 0;
+// Tensor-core issue.  The whole warp walks the loop so that ring positions and operand descriptors
+// stay warp-uniform values; one elected lane issues the instructions.  Pipeline positions: (slot, par) is the ring position (slot
+// index and parity of the current trip round the ring), `q` counts accumulator passes; all advance
+// over the whole launch, identically in every role.  The issuing thread is bound by its own
+// instruction latency, so the loop keeps ready-made descriptors and advances them by additions.
+struct PipePos {
+    uint32_t slot, par, q, act_uses;
+    uint32_t w_full, w_acc;  // cycles the tensor-core thread waited for weights / for a free accumulator (profile)
+};
 
-    for (int p = 0; p < npass; ++p) {
+__device__ __forceinline__ void mma_op(const FwdParams& P, const Part& pt, uint8_t* smem, const uint8_t* B, Misc* misc,
+                                       PipePos& pos, bool& dead) {
+    const uint32_t nstage = (uint32_t)P.nstage;
+    const uint32_t idesc = umma_idesc_bf16_m128((uint32_t)P.NB);
+    const uint64_t wait_limit = P.wait_limit_ns;
+    const uint32_t lbo_b = (uint32_t)P.M * 16u;
+    const uint64_t bstep = (uint64_t)((2u * lbo_b) >> 4);       // one column step, in descriptor address units
+    const uint64_t bdesc0 = umma_smem_desc(smem_u32(B), lbo_b, 128u);
+    const uint32_t ring0 = smem_u32(smem);
+    const uint32_t tmem0 = misc->tmem_base;
+    const int nst = pt.nst, SK = pt.SK, nk = pt.nk;
+    for (int p = 0; p < pt.npass; ++p, ++pos.q) {
         const int pcount = pass_count(pt, p);
-        const int tile_base = pt.tile0 + pass_start(pt, p);
-        const int tile = tile_base + rw;
-        float acc[NT][4];
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-
-        for (int st = 0; st < nst; ++st, ++it) {
-            const uint32_t slot = it % SL::NSTAGE, par = (it / SL::NSTAGE) & 1;
-            if (!dead) {
-                const uint64_t tw0 = prof ? global_timer_ns() : 0;
-                bool got = mbar_wait_bounded(&misc->full_w[slot], par, &misc->abort_flag, P.wait_limit_ns);
-                const uint64_t tw1 = prof ? global_timer_ns() : 0;
-                got = got && mbar_wait_bounded(&misc->full_a[slot], par, &misc->abort_flag, P.wait_limit_ns);
-                if (prof && warp == 0 && lane == 0) {
-                    const uint64_t tw2 = global_timer_ns();
-                    wait_w += tw1 - tw0;
-                    wait_a += tw2 - tw1;
-                }
-                if (!__all_sync(0xffffffffu, got)) dead = true;
-            }
+        const uint32_t buf = pos.q & 1u;
+        const long long tq0 = clock64();
+        if (!dead && !mbar_wait_bounded(&misc->tmem_empty[buf], ((pos.q >> 1) & 1u) ^ 1u, &misc->abort_flag, wait_limit))
+            dead = true;
+        pos.w_acc += (uint32_t)(clock64() - tq0);
+        const uint32_t d_tmem = tmem0 + buf * 32u;
+        const uint32_t lbo_a = (uint32_t)(2 * pcount) * 128u;
+        const uint64_t astep = (uint64_t)((2u * lbo_a) >> 4);
+        const uint64_t adesc0 = umma_smem_desc(ring0, lbo_a, 128u);
+        uint64_t bdesc = bdesc0;
+        int kleft = nk;
+        for (int st = 0; st < nst; ++st, kleft -= SK) {
+            const uint32_t slot = pos.slot, par = pos.par;
+            if (++pos.slot == nstage) { pos.slot = 0; pos.par ^= 1u; }
+            const int nks = min(SK, kleft);
             if (dead) continue;
-            if (prof && p == 0 && st == 0 && warp == 0 && lane == 0) prof[2] = global_timer_ns();
-            const long long c0 = prof ? clock64() : 0;
-            const int kcnt = min(KW, pt.nchunks - st * KW);
-            if (rw < pcount && kw < kcnt) {
-                const uint32_t wbase =
-                    smem_u32(smem + SL::W_OFF + slot * kStageWeightBytes + (kw * pcount + rw) * kTileBytes);
-                const uint32_t abase = smem_u32(smem + SL::A_OFF + slot * SL::A_STAGE + kw * SL::A_CHUNK);
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    uint32_t a0, a1, a2, a3;
-                    ldsm_x4(wbase + swz_unit(lane & 15, ks * 2 + (lane >> 4)), a0, a1, a2, a3);
-#pragma unroll
-                    for (int np = 0; np < NT / 2; ++np) {
-                        uint32_t b0, b1, b2, b3;
-                        const int row = np * 16 + (lane & 7) + ((lane >> 4) << 3);
-                        ldsm_x4(abase + swz_unit(row, ks * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
-                        mma_bf16_16816(acc[2 * np], a0, a1, a2, a3, b0, b1);
-                        mma_bf16_16816(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
-                    }
-                    if (NT & 1) {
-                        uint32_t b0, b1;
-                        const int row = (NT - 1) * 8 + (lane & 7);
-                        ldsm_x2(abase + swz_unit(row, ks * 2 + ((lane >> 3) & 1)), b0, b1);
-                        mma_bf16_16816(acc[NT - 1], a0, a1, a2, a3, b0, b1);
-                    }
+            const long long tw0 = clock64();
+            if (!mbar_wait_bounded(&misc->full[slot], par, &misc->abort_flag, wait_limit)) {
+                dead = true;
+                continue;
+            }
+            pos.w_full += (uint32_t)(clock64() - tw0);
+            tc_fence_after();
+            uint64_t adesc = adesc0 + (uint64_t)((slot * (uint32_t)kStageBytes) >> 4);
+            if (elect_one()) {
+                if (st == 0) umma_bf16_first(d_tmem, adesc, bdesc, idesc);
+                else umma_bf16_acc(d_tmem, adesc, bdesc, idesc);
+#pragma unroll 7
+                for (int ks = 1; ks < nks; ++ks) {
+                    adesc += astep;
+                    bdesc += bstep;
+                    umma_bf16_acc(d_tmem, adesc, bdesc, idesc);
                 }
+                bdesc += bstep;
+                umma_commit(&misc->empty[slot]);  // the slot is free once these instructions have read it
+            } else {
+                bdesc += (uint64_t)nks * bstep;
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&misc->empty[slot]);
-            if (prof) { mma_cycles += (uint64_t)(clock64() - c0); ++mma_stages; }
         }
+        if (!dead && elect_one()) umma_commit(&misc->tmem_full[buf]);
+        __syncwarp();
+    }
+}
 
-        if (prof && p == npass - 1 && warp == 0 && lane == 0) prof[3] = global_timer_ns();
-        if (need_rstd && !have_rstd && !dead) {
-            const bool got = mbar_wait_bounded(&misc->rstd_bar, norm_uses & 1, &misc->abort_flag, P.wait_limit_ns);
-            if (!__all_sync(0xffffffffu, got)) dead = true;
-        }
-        if (need_rstd && !have_rstd && !dead) {
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int n = nt * 8 + q2 + e;
-                    float s = 0.f;
-#pragma unroll
-                    for (int w = 0; w < kLoaderWarps; ++w) s += misc->ss_part[w][n];
-                    rstd[nt][e] = rsqrtf(s / (float)P.d + P.eps);
-                }
-            have_rstd = true;
-        }
+// ------------------------------------------------------------------------------------------
+// Epilogues (warps 0..3).  Thread t = 32 * warp + lane owns accumulator row t of the pass, i.e.
+// weight row 16 * tile_base + t, for all token columns.
+struct ArgBest {
+    float v[kMaxRows];
+    int i[kMaxRows];
+};
 
-        // ---------------- epilogues
-        if (staged) {
-            // partial tiles meet in shared memory: the KW column splits are summed there and each
-            // thread then owns 4 adjacent output rows of one token (one 16-byte global operation)
+template <int NBT>  // token columns read: 16 or 32
+__device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op, int layer, const Part& pt, uint8_t* act, Misc* misc,
+                                            PipePos& pos, bool& dead, int warp, int lane, float (&bv)[NBT], int (&bi)[NBT]) {
+    const int M = P.M;
+    const int t = warp * 32 + lane;
+    float rstd[NBT];
+    if (op == OP_GU || op == OP_LM) {
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
+        for (int n = 0; n < NBT; ++n) rstd[n] = (n < M) ? rsqrtf(misc->sumsq[n] / (float)P.d + P.eps) : 0.f;
+    }
+    for (int p = 0; p < pt.npass; ++p, ++pos.q) {
+        const int pcount = pass_count(pt, p), pstart = pass_start(pt, p);
+        const uint32_t buf = pos.q & 1u;
+        if (!dead && !mbar_wait_bounded(&misc->tmem_full[buf], (pos.q >> 1) & 1u, &misc->abort_flag, P.wait_limit_ns)) dead = true;
+        dead = __any_sync(0xffffffffu, dead);
+        if (dead) continue;
+        tc_fence_after();
+        float v[NBT];
+        {
+            const uint32_t taddr = misc->tmem_base + ((uint32_t)(warp * 32) << 16) + buf * 32u;
+            float lo[16];
+            tmem_ld16(taddr, lo);
 #pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int n = nt * 8 + q2 + e;
-                    red[(warp * MP + n) * 16 + g] = acc[nt][e];
-                    red[(warp * MP + n) * 16 + g + 8] = acc[nt][2 + e];
-                }
-            named_bar_sync(2, kConsumerWarps * 32);
-            if (!dead) {
-                float* out;
-                int stride;
-                if (kind == PH_QKV) { out = P.qkv_acc; stride = P.n_qkv; }
-                else if (kind == PH_RAW) { out = P.raw_out; stride = P.raw_N; }
-                else { out = P.h; stride = P.d; }
-                const int M = P.M, ngroups = pcount * 4 * M;
-                for (int idx = warp * 32 + lane; idx < ngroups; idx += kConsumerWarps * 32) {
-                    const int rwi = idx / (4 * M), rem = idx % (4 * M), n = rem >> 2, r4 = rem & 3;
-                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int kwi = 0; kwi < KW; ++kwi) {
-                        const float4 t =
-                            *reinterpret_cast<const float4*>(red + ((kwi * RW + rwi) * MP + n) * 16 + r4 * 4);
-                        v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
-                    }
-                    float* dst = out + (size_t)n * stride + (tile_base + rwi) * 16 + r4 * 4;
-                    if (od.P_k > 1) {
-                        red_add_v4_f32(dst, v);
-                    } else if (kind == PH_QKV || kind == PH_RAW) {
-                        __stcg(reinterpret_cast<float4*>(dst), v);  // sole owner of a zeroed buffer
-                    } else {
-                        const float4 o = ldcg_f4(dst);  // sole owner: residual add in place
-                        __stcg(reinterpret_cast<float4*>(dst), make_float4(o.x + v.x, o.y + v.y, o.z + v.z, o.w + v.w));
-                    }
+            for (int n = 0; n < 16; ++n) v[n] = lo[n];
+            if (NBT == 32) {
+                float hi[16];
+                tmem_ld16(taddr + 16u, hi);
+#pragma unroll
+                for (int n = 0; n < 16; ++n) v[(NBT == 32 ? 16 : 0) + n] = hi[n];
+            }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&misc->tmem_empty[buf]);  // the accumulator may be overwritten
+        const bool valid = t < 16 * pcount;
+        const int row = (pt.tile0 + pstart) * 16 + t;  // weight row = output feature
+        if (op == OP_GU) {
+            // rows 0..7 of a tile are gate rows, 8..15 the matching up rows: 8 lanes apart
+#pragma unroll
+            for (int n = 0; n < NBT; ++n) {
+                const float up = __shfl_xor_sync(0xffffffffu, v[n], 8);
+                if (valid && (t & 8) == 0 && n < M) {
+                    const float x = v[n] * rstd[n], y = up * rstd[n];
+                    const float a = x / (1.f + expf(-x)) * y;
+                    const int col = (pstart + (t >> 4)) * 8 + (t & 7);  // SwiGLU column within this block's slice
+                    *reinterpret_cast<__nv_bfloat16*>(act + operand_off(col >> 3, n, M) + (col & 7) * 2) = __float2bfloat16(a);
                 }
             }
-            named_bar_sync(2, kConsumerWarps * 32);
-            continue;
-        }
-        if (warp >= pcount || dead) continue;  // RW = 8 here: one tile per warp
-
-        if (kind == PH_GU) {
-            const int fi = tile * 8 + g;  // rows 0..7 of the tile are gate rows, 8..15 the matching up rows
-            uint8_t* dst = P.act + (size_t)(fi >> 6) * SL::A_CHUNK;
+        } else if (op == OP_LM) {
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int n = nt * 8 + q2 + e;
-                    float v = 0.f;
-                    if (n < P.M) {
-                        const float x = acc[nt][e] * rstd[nt][e], y = acc[nt][2 + e] * rstd[nt][e];
-                        v = x / (1.f + expf(-x)) * y;
-                    }
-                    *reinterpret_cast<__nv_bfloat16*>(dst + swz_off(n, fi & 63)) = __float2bfloat16(v);
-                }
-        } else if (kind == PH_LM) {
-            const int r0 = tile * 16 + g;
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int n = nt * 8 + q2 + e;
-                    const float v0 = acc[nt][e] * rstd[nt][e], v1 = acc[nt][2 + e] * rstd[nt][e];
-                    if (P.store_logits && n < P.M) {
-                        __stcg(P.logits + (size_t)n * P.V + r0, v0);
-                        __stcg(P.logits + (size_t)n * P.V + r0 + 8, v1);
-                    }
+            for (int n = 0; n < NBT; ++n) {
+                if (valid && n < M) {
+                    const float x = v[n] * rstd[n];
+                    if (P.store_logits) __stcg(P.logits + (size_t)n * P.V + row, x);
                     // rows come in ascending order per thread, so ">" keeps the lowest id among equals
-                    if (v0 > bv[nt][e]) { bv[nt][e] = v0; bi[nt][e] = r0; }
-                    if (v1 > bv[nt][e]) { bv[nt][e] = v1; bi[nt][e] = r0 + 8; }
+                    if (x > bv[n]) { bv[n] = x; bi[n] = row; }
                 }
+            }
+        } else {
+            float* out;
+            int stride;
+            bool add;
+            if (op == OP_QKV) { out = P.qkv_acc; stride = P.n_qkv; add = P.op[OP_QKV].P_k > 1; }
+            else if (op == OP_RAW) { out = P.raw_out; stride = P.raw_N; add = P.op[OP_RAW].P_k > 1; }
+            else { out = P.h; stride = P.d; add = true; }  // residual add (O, down)
+            if (valid) {
+#pragma unroll
+                for (int n = 0; n < NBT; ++n) {
+                    if (n < M) {
+                        float* dst = out + (size_t)n * stride + row;
+                        if (add) red_add_f32(dst, v[n]);
+                        else __stcg(dst, v[n]);
+                    }
+                }
+            }
         }
     }
-    if (prof && warp == 0 && lane == 0) {
-        prof[4] = global_timer_ns();
-        prof[8] = wait_w;
-        prof[9] = wait_a;
-        prof[10] = mma_cycles;  // SM clock cycles between the waits' end and the slot's release, all stages
-        prof[11] = mma_stages;
+    if (op == OP_GU) {
+        // this warp's SwiGLU columns are written: hand them to the tensor-core thread
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&misc->act_ready);
     }
+}
 
-    if (kind == PH_LM) {
-        // best over the 8 row groups of the warp, then over the 8 warps
+// Best logit per token row over the block: lanes, then the four epilogue warps.
+template <int NBT>
+__device__ __forceinline__ void argmax_finish(const FwdParams& P, Misc* misc, int warp, int lane, float (&bv)[NBT], int (&bi)[NBT],
+                                              bool dead) {
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+    for (int n = 0; n < NBT; ++n) {
+        float v = bv[n];
+        int i = bi[n];
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                float v = bv[nt][e];
-                int i = bi[nt][e];
-#pragma unroll
-                for (int off = 4; off <= 16; off <<= 1) {
-                    const float ov = __shfl_xor_sync(0xffffffffu, v, off);
-                    const int oi = __shfl_xor_sync(0xffffffffu, i, off);
-                    if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
-                }
-                if (g == 0) {
-                    misc->best_v[warp][nt * 8 + q2 + e] = v;
-                    misc->best_i[warp][nt * 8 + q2 + e] = i;
-                }
-            }
-        named_bar_sync(2, kConsumerWarps * 32);
-        const int t = warp * 32 + lane;
-        if (t < MP && !dead) {
-            float v = misc->best_v[0][t];
-            int i = misc->best_i[0][t];
-            for (int w = 1; w < kConsumerWarps; ++w) {
-                const float ov = misc->best_v[w][t];
-                const int oi = misc->best_i[w][t];
-                if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
-            }
-            P.cand_val[(size_t)blockIdx.x * kMaxRows + t] = v;
-            P.cand_idx[(size_t)blockIdx.x * kMaxRows + t] = i;
+        for (int off = 1; off <= 16; off <<= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, v, off);
+            const int oi = __shfl_xor_sync(0xffffffffu, i, off);
+            if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+        }
+        if (lane == 0) {
+            misc->best_v[warp][n] = v;
+            misc->best_i[warp][n] = i;
         }
     }
+    named_bar_sync(2, kEpilogueWarps * 32);
+    const int t = warp * 32 + lane;
+    if (t < NBT && t < P.M && !dead) {
+        float v = misc->best_v[0][t];
+        int i = misc->best_i[0][t];
+        for (int w = 1; w < kEpilogueWarps; ++w) {
+            const float ov = misc->best_v[w][t];
+            const int oi = misc->best_i[w][t];
+            if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+        }
+        P.cand_val[(size_t)blockIdx.x * kMaxRows + t] = v;
+        P.cand_idx[(size_t)blockIdx.x * kMaxRows + t] = i;
+    }
+}
+
+template <int NBT>
+__device__ __noinline__ void epilogue_phase(const FwdParams& P, int kind, int layer, uint8_t* act, Misc* misc, PipePos& pos,
+                                            bool& dead, int warp, int lane) {
+    float bv[NBT];
+    int bi[NBT];
+#pragma unroll
+    for (int n = 0; n < NBT; ++n) { bv[n] = -CUDART_INF_F; bi[n] = 0x7fffffff; }
+    int ops[2];
+    const int nops = phase_ops(kind, ops);
+    for (int oi = 0; oi < nops; ++oi) {
+        const Part& pt = misc->part[ops[oi]];
+        if (pt.ntiles == 0 || pt.nk == 0) continue;
+        epilogue_op<NBT>(P, kind, ops[oi], layer, pt, act, misc, pos, dead, warp, lane, bv, bi);
+    }
+    if (kind == PH_LM) argmax_finish<NBT>(P, misc, warp, lane, bv, bi, dead);
 }
 
 // ------------------------------------------------------------------------------------------
 // Split-KV attention.  The committed cache [0, L) is cut into S key ranges of kps keys (a multiple
-// of 64, as many ranges as there are blocks to take them); unit (kv head, s < S) attends all
-// query rows of the head group to range s; unit (kv head, S) covers the M new rows: it finishes
-// their K/V projection (norm scale, bias, rotary), appends them to the cache and attends to them
-// under the causal mask (row j sees new keys 0..j).  Partial results are merged afterwards.
+// of 64, as many ranges as there are blocks to take them, at most kMaxSplits); unit (kv head,
+// s < S) attends all query rows of the head group to range s; unit (kv head, S) covers the M new
+// rows: it finishes their K/V projection (norm scale, bias, rotary), appends them to the cache and
+// attends to them under the causal mask (row j sees new keys 0..j).  Every unit leaves an
+// un-normalised partial result with its running maximum and sum; the output projection merges them
+// while it builds its operand.
 //
-// Inside a unit the R = (query heads per KV head) x M rows form MT tiles of 16 rows and the keys
-// come in blocks of KB (64 while the row tile leaves room, else 32).  A block takes three short
-// steps, each spread over all 11 worker warps as independent tasks so that no warp runs a long
-// dependent chain:
-//   A  scores: task (row tile, 16 keys) = Q K^T on tensor cores, scaled and masked, kept in
-//      registers; per-row maxima of the 16 keys go to shared memory;
-//   B  same tasks: block maximum per row from the partial maxima, probabilities exp2(s - m),
-//      written as bf16 over the K block (no longer needed), partial row sums to shared memory;
-//   C  output: task (row tile, 16 head columns) = rescale the running output, add P V.
-// Running maximum, sum and rescale factor per row live in shared memory.
+// Inside a unit the R = (query heads per KV head) x M rows form MT tiles of 16 rows.  Keys come in
+// blocks of 32, copied asynchronously into a ring of NBUF shared-memory buffers by all worker
+// warps.  Warp (row tile, key group) owns one row tile and every KG-th group of 16 keys: scores
+// (Q K^T on tensor cores), online softmax with quad shuffles in the log2 domain and P V all stay in
+// its registers; with two key groups the two halves meet in shared memory at the end.
 __device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps) {
     if (P.L <= 0) { S = 0; kps = 0; return; }
     int cap = P.G / P.n_kv - 1;
@@ -584,34 +512,28 @@ __device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps)
     S = (P.L + kps - 1) / kps;
 }
 
-constexpr int kAttnStatsOff = 49152;  // row statistics behind the Q | K | V tiles
-
-template <int HD, bool BIG>  // BIG: more than 64 query rows (4 row tiles)
+template <int HD, bool BIG>  // BIG: more than 64 query rows (up to 8 row tiles)
 __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int S, int kps, uint8_t* att, int wtid,
                                             unsigned long long* prof) {
     constexpr int HD2 = HD / 2;
     constexpr int KSTEPS = HD / 16;
-    constexpr int UNITS = HD / 8;   // 16-byte units per K/V row
-    constexpr int CG = HD / 16;     // 16-column groups of the output
-    constexpr int NWARPS = kWorkerThreads / 32;
-    constexpr int TA_MAX = 2;                                // score tasks per warp (at most 16 tasks)
-    constexpr int TC_MAX = ((BIG ? 8 : 4) * CG + NWARPS - 1) / NWARPS;  // output tasks per warp
-    constexpr int KB = BIG ? 32 : 64, lng = BIG ? 1 : 2, NG = 1 << lng;  // keys per block; 16-key groups
+    constexpr int UNITS = HD / 8;    // 16-byte units per K/V row
+    constexpr int NT_O = HD / 8;     // 8-column tiles of the output
+    constexpr int KB = 32;           // keys per block
+    constexpr int NBUF = BIG ? 2 : 3;
+    constexpr int QBYTES = (BIG ? 128 : 64) * HD * 2;
+    constexpr int KVBYTES = KB * HD * 2;  // one K (or V) block
+    static_assert(QBYTES + NBUF * 2 * KVBYTES <= kAttnSmemBytes, "attention tiles");
+    static_assert(BIG || 4 * NT_O * 32 * 16 + 4 * 32 * 16 <= NBUF * 2 * KVBYTES, "exchange area of the key-group merge");
     const int warp = wtid >> 5, lane = wtid & 31;
     const int M = P.M, L = P.L, R = P.g * M;
     const int MT = (R + 15) >> 4, RP = MT * 16;
+    const int KG = (MT <= 4) ? 2 : 1;
+    const bool active = warp < MT * KG;
+    const int mt = active ? warp % MT : 0, kgp = active ? warp / MT : 0;
     const bool is_new = (s == S);
     uint8_t* Qs = att;
-    uint8_t* Ks = att + RP * HD * 2;
-    uint8_t* Vs = Ks + KB * HD * 2;
-    // probabilities: over the keys once the scores are done (head_dim 128, where the tiles fill the
-    // region), else in the free space behind the tiles
-    uint8_t* Pb = (HD == 128) ? Ks : att + 32768;
-    float* st_m = reinterpret_cast<float*>(att + kAttnStatsOff);  // [2][128] running maximum, by block parity
-    float* st_l = st_m + 256;                                     // [128] running sum
-    float* st_corr = st_l + 128;                                  // [128] rescale factor of this block
-    float* st_pmax = st_corr + 128;                               // [RP][NG] per-task maxima
-    float* st_psum = st_pmax + 256;                               // [RP][NG] per-task sums
+    uint8_t* KVs = att + QBYTES;
     const float* sumsq = P.sumsq + (layer & 1) * kMaxRows;
     const float* bias = P.bias ? P.bias + (size_t)layer * P.n_qkv : nullptr;
     const int Nq = P.n_q * HD, Nkv = P.n_kv * HD;
@@ -627,32 +549,36 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
 
     // cached keys and values of one block: 16-byte asynchronous copies, rows past the range zero-filled
     auto load_block = [&](int blk) {
-        for (int u = wtid; u < KB * UNITS; u += kWorkerThreads) {
-            const int key = u / UNITS, q16 = u % UNITS, kk = blk * KB + key;
-            const bool valid = kk < nkeys;
-            const size_t off = (cache_row0 + t_begin + (valid ? kk : 0)) * HD + q16 * 8;
-            const uint32_t so = (q16 >> 3) * (KB * 128) + swz_unit(key, q16 & 7);
-            cp_async_16_zfill(Ks + so, P.kcache + off, valid);
-            cp_async_16_zfill(Vs + so, P.vcache + off, valid);
+        if (blk < nblk) {
+            uint8_t* Ks = KVs + (blk % NBUF) * 2 * KVBYTES;
+            uint8_t* Vs = Ks + KVBYTES;
+            for (int u = wtid; u < KB * UNITS; u += kWorkerThreads) {
+                const int key = u / UNITS, q16 = u % UNITS, kk = blk * KB + key;
+                const bool valid = kk < nkeys;
+                const size_t off = (cache_row0 + t_begin + (valid ? kk : 0)) * HD + q16 * 8;
+                const uint32_t so = (q16 >> 3) * (KB * 128) + swz_unit(key, q16 & 7);
+                cp_async_16_zfill(Ks + so, P.kcache + off, valid);
+                cp_async_16_zfill(Vs + so, P.vcache + off, valid);
+            }
         }
-        cp_async_commit();
+        cp_async_commit();  // possibly empty: keeps the group count uniform
     };
     if (prof && wtid == 0) prof[2] = global_timer_ns();
-    if (!is_new && nblk > 0) load_block(0);
-    if (wtid < 128) {
-        st_m[wtid] = -CUDART_INF_F;
-        st_l[wtid] = 0.f;
+    if (!is_new) {
+#pragma unroll
+        for (int b = 0; b < NBUF; ++b) load_block(b);
     }
 
     // ---- query tile: normalise, add bias, rotate, round to bf16; 4 rotary pairs per item
     {
+        constexpr int QI = 3;  // items per thread and batch: all loads are issued before the first use
         const int items = RP * (HD2 / 4);
-        for (int base = wtid; base < items; base += 2 * kWorkerThreads) {
-            float4 qa[2], qb[2], c0[2], c1[2];
-            float ssq[2];
-            int rr[2], ii[2];
+        for (int base = wtid; base < items; base += QI * kWorkerThreads) {
+            float4 qa[QI], qb[QI], c0[QI], c1[QI];
+            float ssq[QI];
+            int rr[QI], ii[QI];
 #pragma unroll
-            for (int t = 0; t < 2; ++t) {
+            for (int t = 0; t < QI; ++t) {
                 const int idx = base + t * kWorkerThreads;
                 rr[t] = idx / (HD2 / 4);
                 ii[t] = (idx % (HD2 / 4)) * 4;
@@ -661,15 +587,15 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
                 if (idx < items && rr[t] < R) {
                     const int hl = rr[t] / M, j = rr[t] % M, col = (hk * P.g + hl) * HD + ii[t];
                     ssq[t] = __ldcg(sumsq + j);
-                    qa[t] = ldcg_f4(P.qkv_acc + (size_t)j * P.n_qkv + col);
-                    qb[t] = ldcg_f4(P.qkv_acc + (size_t)j * P.n_qkv + col + HD2);
+                    qa[t] = ld_cg_f4_inorder(P.qkv_acc + (size_t)j * P.n_qkv + col);
+                    qb[t] = ld_cg_f4_inorder(P.qkv_acc + (size_t)j * P.n_qkv + col + HD2);
                     const float4* rp = reinterpret_cast<const float4*>(P.rope + (size_t)(L + j) * HD2 + ii[t]);
-                    c0[t] = __ldg(rp);
-                    c1[t] = __ldg(rp + 1);
+                    c0[t] = ld_nc_f4_inorder(rp);
+                    c1[t] = ld_nc_f4_inorder(rp + 1);
                 }
             }
 #pragma unroll
-            for (int t = 0; t < 2; ++t) {
+            for (int t = 0; t < QI; ++t) {
                 const int idx = base + t * kWorkerThreads;
                 if (idx >= items) continue;
                 const int r = rr[t], i = ii[t];
@@ -696,8 +622,10 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
             }
         }
     }
-    // the new rows' own keys and values fit one block (M <= 32 <= KB)
+    // the new rows' own keys and values fit one block (M <= 32 = KB)
     if (is_new) {
+        uint8_t* Ks = KVs;
+        uint8_t* Vs = Ks + KVBYTES;
         // K and V rows of the new tokens: finish the projection, rotate K, append to the cache
         for (int u = wtid; u < KB * UNITS; u += kWorkerThreads) {
             const int key = u / UNITS, q16 = u % UNITS, kk = key;
@@ -744,169 +672,140 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
     if (prof && wtid == 0) prof[3] = global_timer_ns();
 
     const int g = lane >> 2, q2 = (lane & 3) * 2;
-    const int ntaskA = MT << lng, ntaskC = MT * CG;
-    // byte offset of 16-byte unit `unit` of row r in the probability tile (swizzled against bank conflicts)
-    auto p_unit = [&](uint32_t r, uint32_t unit) -> uint32_t {
-        return KB == 64 ? swz_unit(r, unit) : r * 64u + (((unit ^ (r >> 1)) & 3u) << 4);
-    };
-    float o[TC_MAX][2][4];
+    const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
+    const int j_lo = r_lo % M, j_hi = r_hi % M;
+    float o[NT_O][4];
 #pragma unroll
-    for (int t = 0; t < TC_MAX; ++t)
-#pragma unroll
-        for (int n = 0; n < 2; ++n) o[t][n][0] = o[t][n][1] = o[t][n][2] = o[t][n][3] = 0.f;
+    for (int n = 0; n < NT_O; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+    float m_lo = -CUDART_INF_F, m_hi = -CUDART_INF_F, l_lo = 0.f, l_hi = 0.f;
+    const uint32_t qb = smem_u32(Qs);
 
     for (int blk = 0; blk < nblk; ++blk) {
-        const int par = blk & 1;
-        if (!is_new) {
-            if (blk > 0) load_block(blk);
-            cp_async_wait<0>();
-        }
-        named_bar_sync(1, kWorkerThreads);  // K/V block (and, first time, the Q tile and the row statistics) are in place
+        if (!is_new) cp_async_wait<NBUF - 1>();
+        named_bar_sync(1, kWorkerThreads);  // the block (and, first time, the Q tile) is in place
         if (prof && wtid == 0 && blk == 0) prof[4] = global_timer_ns();
-
-        // ---- A: scores of (row tile, 16 keys), kept in registers
-        float sc[TA_MAX][2][4];
-        const uint32_t qb = smem_u32(Qs), kb = smem_u32(Ks), vb = smem_u32(Vs), pb = smem_u32(Pb);
+        if (active) {
+            const uint32_t kb = smem_u32(KVs + (blk % NBUF) * 2 * KVBYTES), vb = kb + KVBYTES;
+            for (int c = kgp; c < KB / 16; c += KG) {
+                if (blk * KB + c * 16 >= nkeys) break;
+                // ---- scores of 16 rows x 16 keys
+                float sc[2][4];
 #pragma unroll
-        for (int ti = 0; ti < TA_MAX; ++ti) {
-            const int task = warp + ti * NWARPS;
-            if (task >= ntaskA) continue;
-            const int mt = task >> lng, kg = task & (NG - 1);
+                for (int n = 0; n < 2; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
 #pragma unroll
-            for (int n = 0; n < 2; ++n) sc[ti][n][0] = sc[ti][n][1] = sc[ti][n][2] = sc[ti][n][3] = 0.f;
-#pragma unroll
-            for (int ks = 0; ks < KSTEPS; ++ks) {
-                uint32_t a0, a1, a2, a3, b0, b1, b2, b3;
-                ldsm_x4(qb + (ks >> 2) * (RP * 128) + swz_unit(mt * 16 + (lane & 15), (ks & 3) * 2 + (lane >> 4)), a0, a1, a2,
-                        a3);
-                const int row = kg * 16 + (lane & 7) + ((lane >> 4) << 3);
-                ldsm_x4(kb + (ks >> 2) * (KB * 128) + swz_unit(row, (ks & 3) * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
-                mma_bf16_16816(sc[ti][0], a0, a1, a2, a3, b0, b1);
-                mma_bf16_16816(sc[ti][1], a0, a1, a2, a3, b2, b3);
-            }
-            const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
-            const int j_lo = r_lo % M, j_hi = r_hi % M;
-            float mx_lo = -CUDART_INF_F, mx_hi = -CUDART_INF_F;
-#pragma unroll
-            for (int n = 0; n < 2; ++n)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int key = blk * KB + kg * 16 + n * 8 + q2 + (e & 1);
-                    const bool hi = e >= 2;
-                    const int row = hi ? r_hi : r_lo, j = hi ? j_hi : j_lo;
-                    const bool ok = key < nkeys && row < R && (!is_new || key <= j);
-                    const float v = ok ? sc[ti][n][e] * P.scale_log2e : -CUDART_INF_F;
-                    sc[ti][n][e] = v;
-                    if (hi) mx_hi = fmaxf(mx_hi, v); else mx_lo = fmaxf(mx_lo, v);
+                for (int ks = 0; ks < KSTEPS; ++ks) {
+                    uint32_t a0, a1, a2, a3, b0, b1, b2, b3;
+                    ldsm_x4(qb + (ks >> 2) * (RP * 128) + swz_unit(mt * 16 + (lane & 15), (ks & 3) * 2 + (lane >> 4)), a0, a1, a2, a3);
+                    const int row = c * 16 + (lane & 7) + ((lane >> 4) << 3);
+                    ldsm_x4(kb + (ks >> 2) * (KB * 128) + swz_unit(row, (ks & 3) * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
+                    mma_bf16_16816(sc[0], a0, a1, a2, a3, b0, b1);
+                    mma_bf16_16816(sc[1], a0, a1, a2, a3, b2, b3);
                 }
-            mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
-            mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
-            mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
-            mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
-            if ((lane & 3) == 0) {
-                st_pmax[(r_lo << lng) + kg] = mx_lo;
-                st_pmax[(r_hi << lng) + kg] = mx_hi;
+                float mx_lo = -CUDART_INF_F, mx_hi = -CUDART_INF_F;
+#pragma unroll
+                for (int n = 0; n < 2; ++n)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int key = blk * KB + c * 16 + n * 8 + q2 + (e & 1);
+                        const bool hi = e >= 2;
+                        const int row = hi ? r_hi : r_lo, j = hi ? j_hi : j_lo;
+                        const bool ok = key < nkeys && row < R && (!is_new || key <= j);
+                        const float v = ok ? sc[n][e] * P.scale_log2e : -CUDART_INF_F;
+                        sc[n][e] = v;
+                        if (hi) mx_hi = fmaxf(mx_hi, v); else mx_lo = fmaxf(mx_lo, v);
+                    }
+                mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+                mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+                mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+                mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+                // ---- online softmax: new maximum, rescale, probabilities
+                const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+                const float use_lo = (mn_lo == -CUDART_INF_F) ? 0.f : mn_lo, use_hi = (mn_hi == -CUDART_INF_F) ? 0.f : mn_hi;
+                const float c_lo = exp2f(m_lo - use_lo), c_hi = exp2f(m_hi - use_hi);
+                m_lo = mn_lo;
+                m_hi = mn_hi;
+                float p[2][4];
+#pragma unroll
+                for (int n = 0; n < 2; ++n) {
+                    p[n][0] = exp2f(sc[n][0] - use_lo);
+                    p[n][1] = exp2f(sc[n][1] - use_lo);
+                    p[n][2] = exp2f(sc[n][2] - use_hi);
+                    p[n][3] = exp2f(sc[n][3] - use_hi);
+                }
+                l_lo = l_lo * c_lo + p[0][0] + p[0][1] + p[1][0] + p[1][1];
+                l_hi = l_hi * c_hi + p[0][2] + p[0][3] + p[1][2] + p[1][3];
+#pragma unroll
+                for (int n = 0; n < NT_O; ++n) { o[n][0] *= c_lo; o[n][1] *= c_lo; o[n][2] *= c_hi; o[n][3] *= c_hi; }
+                // ---- O += P V: the score accumulators are, pairwise packed, the A operand of the next product
+                const uint32_t a0 = pack_bf16(p[0][0], p[0][1]), a1 = pack_bf16(p[0][2], p[0][3]);
+                const uint32_t a2 = pack_bf16(p[1][0], p[1][1]), a3 = pack_bf16(p[1][2], p[1][3]);
+#pragma unroll
+                for (int cg = 0; cg < NT_O / 2; ++cg) {
+                    uint32_t b0, b1, b2, b3;
+                    const int key = c * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+                    const int cu = cg * 2 + (lane >> 4);
+                    ldsm_x4_trans(vb + (cu >> 3) * (KB * 128) + swz_unit(key, cu & 7), b0, b1, b2, b3);
+                    mma_bf16_16816(o[2 * cg], a0, a1, a2, a3, b0, b1);
+                    mma_bf16_16816(o[2 * cg + 1], a0, a1, a2, a3, b2, b3);
+                }
             }
         }
-        named_bar_sync(1, kWorkerThreads);  // partial maxima are visible; the K block has been read
+        named_bar_sync(1, kWorkerThreads);  // the block has been consumed
+        if (!is_new) load_block(blk + NBUF);
+    }
+    if (!is_new) cp_async_wait<0>();
+    if (prof && wtid == 0) prof[5] = global_timer_ns();
 
-        // ---- B: probabilities
+    // ---- row sums over the quad; the two key groups of a row tile meet in shared memory
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+    if (KG == 2) {
+        float4* ex_o = reinterpret_cast<float4*>(KVs);                      // [row tile][output tile][lane]
+        float4* ex_ml = ex_o + 4 * NT_O * 32;                               // [row tile][lane]
+        if (active && kgp == 1) {
 #pragma unroll
-        for (int ti = 0; ti < TA_MAX; ++ti) {
-            const int task = warp + ti * NWARPS;
-            if (task >= ntaskA) continue;
-            const int mt = task >> lng, kg = task & (NG - 1);
-            const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
-            float mb_lo = st_pmax[r_lo << lng], mb_hi = st_pmax[r_hi << lng];
-            for (int i = 1; i < NG; ++i) {
-                mb_lo = fmaxf(mb_lo, st_pmax[(r_lo << lng) + i]);
-                mb_hi = fmaxf(mb_hi, st_pmax[(r_hi << lng) + i]);
-            }
-            const float mo_lo = st_m[par * 128 + r_lo], mo_hi = st_m[par * 128 + r_hi];
-            const float mn_lo = fmaxf(mo_lo, mb_lo), mn_hi = fmaxf(mo_hi, mb_hi);
+            for (int n = 0; n < NT_O; ++n) ex_o[(mt * NT_O + n) * 32 + lane] = make_float4(o[n][0], o[n][1], o[n][2], o[n][3]);
+            ex_ml[mt * 32 + lane] = make_float4(m_lo, m_hi, l_lo, l_hi);
+        }
+        named_bar_sync(1, kWorkerThreads);
+        if (active && kgp == 0) {
+            const float4 ml = ex_ml[mt * 32 + lane];
+            const float mn_lo = fmaxf(m_lo, ml.x), mn_hi = fmaxf(m_hi, ml.y);
             const float use_lo = (mn_lo == -CUDART_INF_F) ? 0.f : mn_lo, use_hi = (mn_hi == -CUDART_INF_F) ? 0.f : mn_hi;
-            float sum_lo = 0.f, sum_hi = 0.f;
+            const float e0_lo = exp2f(m_lo - use_lo), e1_lo = exp2f(ml.x - use_lo);
+            const float e0_hi = exp2f(m_hi - use_hi), e1_hi = exp2f(ml.y - use_hi);
+            m_lo = mn_lo;
+            m_hi = mn_hi;
+            l_lo = l_lo * e0_lo + ml.z * e1_lo;
+            l_hi = l_hi * e0_hi + ml.w * e1_hi;
 #pragma unroll
-            for (int n = 0; n < 2; ++n) {
-                const float p0 = exp2f(sc[ti][n][0] - use_lo), p1 = exp2f(sc[ti][n][1] - use_lo);
-                const float p2 = exp2f(sc[ti][n][2] - use_hi), p3 = exp2f(sc[ti][n][3] - use_hi);
-                sum_lo += p0 + p1;
-                sum_hi += p2 + p3;
-                const uint32_t unit = (uint32_t)(kg * 2 + n);
-                *reinterpret_cast<uint32_t*>(Pb + p_unit(r_lo, unit) + q2 * 2) = pack_bf16(p0, p1);
-                *reinterpret_cast<uint32_t*>(Pb + p_unit(r_hi, unit) + q2 * 2) = pack_bf16(p2, p3);
-            }
-            sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 1);
-            sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 2);
-            sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 1);
-            sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 2);
-            if ((lane & 3) == 0) {
-                st_psum[(r_lo << lng) + kg] = sum_lo;
-                st_psum[(r_hi << lng) + kg] = sum_hi;
-                if (kg == 0) {
-                    st_corr[r_lo] = exp2f(mo_lo - use_lo);
-                    st_corr[r_hi] = exp2f(mo_hi - use_hi);
-                    st_m[(par ^ 1) * 128 + r_lo] = mn_lo;
-                    st_m[(par ^ 1) * 128 + r_hi] = mn_hi;
-                }
+            for (int n = 0; n < NT_O; ++n) {
+                const float4 t = ex_o[(mt * NT_O + n) * 32 + lane];
+                o[n][0] = o[n][0] * e0_lo + t.x * e1_lo;
+                o[n][1] = o[n][1] * e0_lo + t.y * e1_lo;
+                o[n][2] = o[n][2] * e0_hi + t.z * e1_hi;
+                o[n][3] = o[n][3] * e0_hi + t.w * e1_hi;
             }
         }
-        named_bar_sync(1, kWorkerThreads);  // probabilities, sums and rescale factors are visible
-
-        // ---- C: O = O * corr + P V for (row tile, 16 columns)
-#pragma unroll
-        for (int tj = 0; tj < TC_MAX; ++tj) {
-            const int task = warp + tj * NWARPS;
-            if (task >= ntaskC) continue;
-            const int mt = task / CG, cg = task % CG;
-            const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
-            const float c_lo = st_corr[r_lo], c_hi = st_corr[r_hi];
-#pragma unroll
-            for (int n = 0; n < 2; ++n) { o[tj][n][0] *= c_lo; o[tj][n][1] *= c_lo; o[tj][n][2] *= c_hi; o[tj][n][3] *= c_hi; }
-            for (int k2 = 0; k2 < NG; ++k2) {
-                uint32_t a0, a1, a2, a3, b0, b1, b2, b3;
-                ldsm_x4(pb + p_unit(mt * 16 + (lane & 15), k2 * 2 + (lane >> 4)), a0, a1, a2, a3);
-                const int key = k2 * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
-                const int cu = cg * 2 + (lane >> 4);
-                ldsm_x4_trans(vb + (cu >> 3) * (KB * 128) + swz_unit(key, cu & 7), b0, b1, b2, b3);
-                mma_bf16_16816(o[tj][0], a0, a1, a2, a3, b0, b1);
-                mma_bf16_16816(o[tj][1], a0, a1, a2, a3, b2, b3);
-            }
-            if (cg == 0 && (lane & 3) == 0) {
-                float s_lo = 0.f, s_hi = 0.f;
-                for (int i = 0; i < NG; ++i) {
-                    s_lo += st_psum[(r_lo << lng) + i];
-                    s_hi += st_psum[(r_hi << lng) + i];
-                }
-                st_l[r_lo] = st_l[r_lo] * c_lo + s_lo;
-                st_l[r_hi] = st_l[r_hi] * c_hi + s_hi;
-            }
-        }
-        named_bar_sync(1, kWorkerThreads);  // the block has been consumed; row statistics are up to date
     }
 
     // ---- un-normalised partial result of this key range
-    if (prof && wtid == 0) prof[5] = global_timer_ns();
-#pragma unroll
-    for (int tj = 0; tj < TC_MAX; ++tj) {
-        const int task = warp + tj * NWARPS;
-        if (task >= ntaskC) continue;
-        const int mt = task / CG, cg = task % CG;
+    if (active && kgp == 0) {
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
-            const int r = mt * 16 + g + half * 8;
+            const int r = half ? r_hi : r_lo;
             if (r >= R) continue;
             const int hq = hk * P.g + r / M, j = r % M;
             const size_t row = ((size_t)hq * (kMaxSplits + 1) + s) * kMaxRows + j;
-            float* po = P.part_o + row * HD + cg * 16 + q2;
-            __stcg(reinterpret_cast<float2*>(po), make_float2(o[tj][0][half * 2], o[tj][0][half * 2 + 1]));
-            __stcg(reinterpret_cast<float2*>(po + 8), make_float2(o[tj][1][half * 2], o[tj][1][half * 2 + 1]));
+            float* po = P.part_o + row * HD + q2;
+#pragma unroll
+            for (int n = 0; n < NT_O; ++n)
+                __stcg(reinterpret_cast<float2*>(po + n * 8), make_float2(o[n][half * 2], o[n][half * 2 + 1]));
+            if ((lane & 3) == 0)
+                __stcg(reinterpret_cast<float2*>(P.part_ml + row * 2), make_float2(half ? m_hi : m_lo, half ? l_hi : l_lo));
         }
-    }
-    if (wtid < R) {
-        const int hq = hk * P.g + wtid / M, j = wtid % M;
-        const size_t row = ((size_t)hq * (kMaxSplits + 1) + s) * kMaxRows + j;
-        __stcg(reinterpret_cast<float2*>(P.part_ml + row * 2), make_float2(st_m[(nblk & 1) * 128 + wtid], st_l[wtid]));
     }
 }
 
@@ -929,59 +828,6 @@ __device__ void attention_phase(const FwdParams& P, int layer, uint8_t* att, int
         if (prof && wtid == 0) { prof[6] = global_timer_ns(); prof[7] = (unsigned long long)(s == S); }
     }
 }
-
-// Merge of the split-KV partial results into the output projection's bf16 operand.  One warp per
-// (query head, row, 8 columns); lanes run over the splits.
-template <int NT>
-__device__ __noinline__ void combine_phase(const FwdParams& P, int wtid) {
-    constexpr int A_CHUNK = SmemLayout<NT>::A_CHUNK;
-    int S, kps;
-    attn_split(P, S, kps);
-    const int S1 = S + 1;
-    const int warp = wtid >> 5, lane = wtid & 31;
-    const int U8 = P.hd / 8, nwarps = kWorkerThreads / 32;
-    const int items = P.n_q * P.M * U8;
-    for (int item = blockIdx.x * nwarps + warp; item < items; item += P.G * nwarps) {
-        const int hq = item / (P.M * U8), j = (item / U8) % P.M, c8 = item % U8;
-        const size_t base = ((size_t)hq * (kMaxSplits + 1)) * kMaxRows + j;
-        float m[2], l[2];
-        float4 a[2], b[2];
-#pragma unroll
-        for (int t = 0; t < 2; ++t) {
-            const int s = lane + 32 * t;
-            m[t] = -CUDART_INF_F; l[t] = 0.f;
-            a[t] = b[t] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (s < S1) {
-                const size_t row = base + (size_t)s * kMaxRows;
-                const float2 ml = __ldcg(reinterpret_cast<const float2*>(P.part_ml + row * 2));
-                m[t] = ml.x; l[t] = ml.y;
-                const float* op = P.part_o + row * P.hd + c8 * 8;
-                a[t] = ldcg_f4(op);
-                b[t] = ldcg_f4(op + 4);
-            }
-        }
-        float mmax = fmaxf(m[0], m[1]);
-#pragma unroll
-        for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
-        const float w0 = exp2f(m[0] - mmax), w1 = exp2f(m[1] - mmax);  // 0 for splits that saw no key
-        float v[9];
-        v[0] = w0 * a[0].x + w1 * a[1].x; v[1] = w0 * a[0].y + w1 * a[1].y; v[2] = w0 * a[0].z + w1 * a[1].z;
-        v[3] = w0 * a[0].w + w1 * a[1].w; v[4] = w0 * b[0].x + w1 * b[1].x; v[5] = w0 * b[0].y + w1 * b[1].y;
-        v[6] = w0 * b[0].z + w1 * b[1].z; v[7] = w0 * b[0].w + w1 * b[1].w; v[8] = w0 * l[0] + w1 * l[1];
-#pragma unroll
-        for (int e = 0; e < 9; ++e)
-#pragma unroll
-            for (int off = 16; off; off >>= 1) v[e] += __shfl_xor_sync(0xffffffffu, v[e], off);
-        if (lane == 0) {
-            const float inv = 1.f / v[8];
-            const int col = hq * P.hd + c8 * 8;
-            const uint4 out = make_uint4(pack_bf16(v[0] * inv, v[1] * inv), pack_bf16(v[2] * inv, v[3] * inv),
-                                         pack_bf16(v[4] * inv, v[5] * inv), pack_bf16(v[6] * inv, v[7] * inv));
-            *reinterpret_cast<uint4*>(P.attn_op + (size_t)(col >> 6) * A_CHUNK + swz_unit(j, (col & 63) >> 3)) = out;
-        }
-    }
-}
-
 // ------------------------------------------------------------------------------------------
 __device__ void embed_phase(const FwdParams& P, int wtid) {
     // residual rows from the embedding table; rows beyond M are cleared
@@ -1014,16 +860,91 @@ __device__ void zero_qkv_acc(const FwdParams& P, int sumsq_buf, int wtid) {
     if (blockIdx.x == 0 && wtid < kMaxRows) __stcg(P.sumsq + sumsq_buf * kMaxRows + wtid, 0.f);
 }
 
+
 // ------------------------------------------------------------------------------------------
-template <int NT>
+// One GEMM phase as seen by the worker warps: build the token operand, then the tensor-core
+// thread walks the block's stages while the epilogue warps drain the accumulators.
+__device__ __forceinline__ void advance_pos(PipePos& pos, const Part& pt, uint32_t nstage) {
+    const uint32_t at = pos.slot + (uint32_t)(pt.npass * pt.nst);
+    pos.slot = at % nstage;
+    pos.par ^= (at / nstage) & 1u;
+    pos.q += (uint32_t)pt.npass;
+}
+
+__device__ __noinline__ void gemm_phase(const FwdParams& P, int kind, int layer, uint8_t* smem, Misc* misc, PipePos& pos, int wtid,
+                                        unsigned long long* prof) {
+    const int warp = wtid >> 5, lane = wtid & 31;
+    uint8_t* U = smem + P.u_off;
+    uint8_t* act = smem + P.act_off;
+    int ops[2];
+    const int nops = phase_ops(kind, ops);
+    const Part& p0 = misc->part[ops[0]];
+    const bool have0 = p0.ntiles > 0 && p0.nk > 0;
+    bool dead = *(volatile int*)&misc->abort_flag != 0;
+
+    if (have0 && !dead) {
+        if (kind == PH_O) build_merged_operand(P, p0, U, wtid);
+        else build_norm_operand(P, kind, layer, p0, U, misc, wtid);
+        fence_proxy_async_smem();
+    }
+    if (kind == PH_O) {
+        // clear the accumulators the next QKV projection adds into (idle warps)
+        const int n4 = kMaxRows * P.n_qkv / 4, nth = (kWorkerWarps - kEpilogueWarps) * 32;
+        if (warp >= kEpilogueWarps) {
+            for (int i = blockIdx.x * nth + (wtid - kEpilogueWarps * 32); i < n4; i += P.G * nth)
+                __stcg(reinterpret_cast<float4*>(P.qkv_acc) + i, make_float4(0.f, 0.f, 0.f, 0.f));
+            if (blockIdx.x == 0 && wtid >= kEpilogueWarps * 32 && wtid < kEpilogueWarps * 32 + kMaxRows)
+                __stcg(P.sumsq + ((layer + 1) & 1) * kMaxRows + (wtid - kEpilogueWarps * 32), 0.f);
+        }
+    }
+    named_bar_sync(1, kWorkerThreads);  // the operand is complete and visible to the tensor core
+    if (prof && wtid == 0) prof[2] = global_timer_ns();
+
+    if (warp == kMmaWarp) {
+        PipePos mp = pos;
+        mp.w_full = mp.w_acc = 0;
+        const long long tc0 = clock64();
+        tc_fence_after();
+        for (int oi = 0; oi < nops; ++oi) {
+            const Part& pt = misc->part[ops[oi]];
+            if (pt.ntiles == 0 || pt.nk == 0) continue;
+            if (ops[oi] == OP_DOWN) {
+                if (prof && lane == 0) prof[5] = global_timer_ns();
+                if (!dead && !mbar_wait_bounded(&misc->act_ready, mp.act_uses & 1u, &misc->abort_flag, P.wait_limit_ns))
+                    dead = true;
+                dead = __any_sync(0xffffffffu, dead);
+                tc_fence_after();
+                if (prof && lane == 0) prof[6] = global_timer_ns();
+            }
+            mma_op(P, pt, smem, ops[oi] == OP_DOWN ? act : U, misc, mp, dead);
+        }
+        if (prof && lane == 0) {
+            prof[3] = global_timer_ns();
+            prof[7] = mp.w_full;
+            prof[8] = mp.w_acc;
+            prof[9] = (unsigned long long)(clock64() - tc0);  // cycles of the whole issue loop
+        }
+    } else if (warp < kEpilogueWarps) {
+        PipePos ep = pos;
+        if (P.NB == 32) epilogue_phase<32>(P, kind, layer, act, misc, ep, dead, warp, lane);
+        else epilogue_phase<16>(P, kind, layer, act, misc, ep, dead, warp, lane);
+        if (prof && wtid == 0) prof[4] = global_timer_ns();
+    }
+    // pipeline positions advance identically for every role
+    for (int oi = 0; oi < nops; ++oi) {
+        const Part& pt = misc->part[ops[oi]];
+        if (pt.ntiles == 0 || pt.nk == 0) continue;
+        advance_pos(pos, pt, (uint32_t)P.nstage);
+        if (ops[oi] == OP_GU) ++pos.act_uses;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_constant__ FwdParams Pg) {
-    using SL = SmemLayout<NT>;
-    static_assert(SL::NSTAGE >= 4 && SL::NSTAGE <= 16, "ring depth");
-    static_assert(kConsumerWarps * SL::MP * 16 * 4 <= kRedBytes, "staged epilogue buffer");
     static_assert(sizeof(FwdParams) % 4 == 0, "parameter block is copied word by word");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    Misc* misc = reinterpret_cast<Misc*>(smem + SL::MISC_OFF);
+    Misc* misc = reinterpret_cast<Misc*>(smem + Pg.misc_off);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     {
         const int* src = reinterpret_cast<const int*>(&Pg);
@@ -1031,73 +952,77 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
         for (int i = tid; i < (int)(sizeof(FwdParams) / 4); i += kThreads) dst[i] = src[i];
     }
     const FwdParams& P = misc->P;
-    if (tid >= 32 && tid < 32 + OP_COUNT) misc->part[tid - 32] = get_part(Pg.op[tid - 32], blockIdx.x, Pg.G);
+    if (tid >= 32 && tid < 32 + OP_COUNT) misc->part[tid - 32] = get_part(Pg.op[tid - 32], Pg.op[OP_GU], blockIdx.x, Pg.G);
 
     if (tid == 0) {
-        for (int s = 0; s < SL::NSTAGE; ++s) {
-            mbar_init(&misc->full_w[s], 1);
-            mbar_init(&misc->full_a[s], kMaxKW);
-            mbar_init(&misc->empty[s], kConsumerWarps);
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(&misc->full[s], 1);
+            mbar_init(&misc->empty[s], 1);
         }
-        mbar_init(&misc->rstd_bar, kLoaderWarps);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&misc->tmem_full[b], 1);
+            mbar_init(&misc->tmem_empty[b], kEpilogueWarps);
+        }
+        mbar_init(&misc->act_ready, kEpilogueWarps);
+        mbar_init(&misc->done_bar, 1);
         misc->abort_flag = 0;
         misc->skip = 0;
         mbar_fence_init();
     }
+    if (warp == kMmaWarp) tmem_alloc(&misc->tmem_base, kTmemCols);
+    tc_fence_before();
     __syncthreads();
+    tc_fence_after();
 
-    if (warp == kConsumerWarps + kLoaderWarps) {
-        if (lane == 0) producer_loop<NT>(P, smem, misc);
+    if (warp == kProducerWarp) {
+        if (lane == 0) producer_loop(P, smem, misc);
         return;
     }
 
     const int wtid = tid;  // 0 .. kWorkerThreads-1
-    uint32_t it = 0, ci = 0, norm_uses = 0;
+    PipePos pos;
+    pos.slot = pos.par = pos.q = pos.act_uses = pos.w_full = pos.w_acc = 0;
     int nbar = 0;
     bool skip = false;
     for (int ph = P.ph_begin; ph < P.ph_end; ++ph) {
         int layer;
         const int kind = decode_phase(ph, P.n_layers, layer);
-        if (P.prof && wtid == 0) P.prof[((size_t)(ph - P.ph_begin) * P.G + blockIdx.x) * kProfWords] = global_timer_ns();
+        unsigned long long* pp = P.prof ? P.prof + ((size_t)(ph - P.ph_begin) * P.G + blockIdx.x) * kProfWords : nullptr;
+        if (pp && wtid == 0) pp[0] = global_timer_ns();
         // after an abandoned wait the remaining phases do no work but still meet at every barrier
         if (skip) {
         } else if (kind == PH_EMBED) {
             embed_phase(P, wtid);
             zero_qkv_acc(P, 0, wtid);
         } else if (kind == PH_ATTN) {
-            attention_phase(P, layer, smem + SL::ATT_OFF, wtid,
-                            P.prof ? P.prof + ((size_t)(ph - P.ph_begin) * P.G + blockIdx.x) * kProfWords : nullptr);
-        } else if (kind == PH_COMB) {
-            combine_phase<NT>(P, wtid);
+            attention_phase(P, layer, smem + P.u_off, wtid, pp);
         } else {
-            if (kind == PH_O) zero_qkv_acc(P, (layer + 1) & 1, wtid);
-            const OpDesc& od = P.op[phase_op(kind)];
-            const Part& pt = misc->part[phase_op(kind)];
-            if (pt.ntiles > 0) {
-                unsigned long long* pp =
-                    P.prof ? P.prof + ((size_t)(ph - P.ph_begin) * P.G + blockIdx.x) * kProfWords : nullptr;
-                if (warp < kConsumerWarps) {
-                    consumer_phase<NT>(P, kind, layer, od, pt, smem, misc, it, norm_uses, warp, lane, pp);
-                } else {
-                    const bool norm = (kind == PH_QKV || kind == PH_GU || kind == PH_LM);
-                    if (norm) loader_norm<NT>(P, kind, layer, od, pt, smem, misc, it, ci, warp - kConsumerWarps, lane, pp);
-                    else loader_copy<NT>(P, kind, od, pt, smem, misc, it, ci, warp - kConsumerWarps, lane, pp);
-                }
-                // pipeline positions advance identically for every role
-                it += (uint32_t)(pt.npass * pt.nst);
-                ci += (uint32_t)(pt.npass * pt.nchunks);
-                if (kind == PH_GU || kind == PH_LM) ++norm_uses;
-            }
+            gemm_phase(P, kind, layer, smem, misc, pos, wtid, pp);
         }
-        if (P.prof) {
+        if (pp) {
             named_bar_sync(1, kWorkerThreads);
-            if (wtid == 0) P.prof[((size_t)(ph - P.ph_begin) * P.G + blockIdx.x) * kProfWords + 1] = global_timer_ns();
+            if (wtid == 0) pp[1] = global_timer_ns();
         }
         if (ph + 1 < P.ph_end) {
             ++nbar;
             skip = grid_barrier(P, P.bar_base + nbar * P.G, misc, wtid);
         }
     }
+    // all tensor-core work must have completed before tensor memory is returned
+    if (warp == kMmaWarp && lane == 0) {
+        umma_commit(&misc->done_bar);
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(&misc->done_bar, 0)) {
+            if (global_timer_ns() - t0 > P.wait_limit_ns) {
+                *(volatile int*)&misc->abort_flag = 1;
+                break;
+            }
+        }
+    }
+    tc_fence_before();
+    named_bar_sync(1, kWorkerThreads);
+    tc_fence_after();
+    if (warp == kMmaWarp) tmem_dealloc(misc->tmem_base, kTmemCols);
     if (*(volatile int*)&misc->abort_flag) {
         if (wtid == 0) atomicExch(P.state + ST_ERR, 1);
     }

@@ -1,54 +1,63 @@
 // Shapes, buffer pointers and the static work partition shared by host code and kernels.
 //
-// Weight streaming layout.  Every linear layer W[N][K] (bf16) is cut into tiles of 16 rows x 64
-// columns (2 KB, 128-byte rows with XOR-swizzled 16-byte units).  An operation's tile grid
-// (T = N/16 row tiles, C = K/64 column chunks) is split into P_row x P_k rectangular
-// partitions, one per thread block.  The block's 8 MMA warps form an RW x KW grid (RW * KW = 8):
-// it walks its partition in passes of at most RW row tiles and, inside a pass, in stages of KW
-// consecutive chunks, so one stage is RW x KW tiles (<= 16 KB), one per warp.  Tiles are stored
-// pass by pass, chunk by chunk, tile by tile: every stage is one contiguous bulk copy and a
-// block's whole share of an operation is one contiguous byte range.
+// Weight streaming layout.  Every linear layer W[N][K] (bf16) is seen as a grid of T = N/16 row
+// tiles by K16 = K/16 column steps (one step = the 16 input features of one tensor-core
+// instruction).  The grid is split into P_row x P_k rectangular partitions, one per thread
+// block.  A block walks its partition in passes of at most RW row tiles (RW <= 8: one pass is
+// one 128-row accumulator in tensor memory, rows past the pass are don't-care) and, inside a
+// pass, in stages of at most SK column steps (RW * SK <= 64, i.e. <= 32 KB).  A stage is stored
+// as the shared-memory image the tensor core reads: column step by column step, the two
+// 8-column halves of a step one after the other, each a run of 8-row x 16-byte core matrices
+//     [step][half][8-row group][row][8 bf16]
+// with no padding.  Stages follow each other pass by pass, so every stage is one contiguous
+// bulk copy and a block's whole share of an operation is one contiguous byte range.
 #pragma once
 #include <cuda_bf16.h>
 #include <stdint.h>
 
 namespace sdv {
 
-constexpr int kConsumerWarps = 8;
-constexpr int kLoaderWarps = 3;
-constexpr int kWorkerThreads = (kConsumerWarps + kLoaderWarps) * 32;  // 352: every warp but the producer
-constexpr int kThreads = kWorkerThreads + 32;                        // 384 with the weight-streaming warp
-constexpr int kTileBytes = 2048;                                     // 16 rows x 64 cols bf16
-constexpr int kStageWeightBytes = kConsumerWarps * kTileBytes;       // 16 KB
-constexpr int kMaxRows = 32;                                         // token rows a buffer is sized for
-constexpr int kMaxSplits = 40;                                       // KV splits per head (+1 unit for new rows)
-constexpr int kMaxKW = 4;                                             // chunks per stage at most
-constexpr int kSmemBudget = 232448;                                  // 227 KB
-constexpr int kAttnSmemBytes = 49152 + 4096;                         // Q tile + K and V blocks (48 KB), row statistics
+constexpr int kWorkerWarps = 11;                       // every warp but the weight streamer
+constexpr int kWorkerThreads = kWorkerWarps * 32;      // 352
+constexpr int kThreads = kWorkerThreads + 32;          // 384 with the weight-streaming warp
+constexpr int kEpilogueWarps = 4;                      // warps 0..3 read the accumulator (tensor-memory lanes 32w..32w+31)
+constexpr int kMmaWarp = 10;                           // its lane 0 issues the tensor-core instructions
+constexpr int kProducerWarp = 11;
+constexpr int kStepBytes = 512;                        // one row tile x one column step: 16 x 16 bf16
+constexpr int kStageBytes = 32768;                     // ring slot
+constexpr int kMaxStages = 8;                          // ring slots at most
+constexpr int kMaxRows = 32;                           // token rows a buffer is sized for
+constexpr int kMaxSplits = 19;                         // KV key ranges per head (+1 partial result for the new rows)
+constexpr int kSmemBudget = 232448;                    // 227 KB
+constexpr int kAttnSmemBytes = 65536;                  // Q tile (16 or 32 KB) + ring of K|V blocks (48 or 32 KB)
+constexpr int kActSmemMax = 32768;                     // SwiGLU output of this block (operand of its down-projection slice) at most
 constexpr int kMiscSmemBytes = 4096;
 constexpr int kMaxDraftWords = 32;
-constexpr int kProfWords = 12;                                       // timestamps per (phase, block)
+constexpr int kProfWords = 12;                         // timestamps per (phase, block)
+constexpr int kTmemCols = 64;                          // two accumulators of up to 32 fp32 columns
 
 enum OpIndex { OP_QKV = 0, OP_O = 1, OP_GU = 2, OP_DOWN = 3, OP_LM = 4, OP_RAW = 5, OP_COUNT = 6 };
 
 struct OpDesc {
     int T;       // row tiles (16 weight rows each)
-    int C;       // column chunks (64 input features each)
+    int K16;     // column steps (16 input features each)
     int P_row;   // partitions along rows
-    int P_k;     // partitions along columns (> 1: partial sums meet by atomic adds)
+    int P_k;     // partitions along columns (> 1: partial sums meet by reductions in L2)
     int rot;     // block index that owns partition 0 (spreads idle blocks over operations)
-    int RW;      // row tiles per pass (8, 4 or 2); KW = 8 / RW chunks per stage
+    int RW;      // row tiles per pass at most (8, 4, 2 or 1)
+    int SK;      // column steps per stage at most (RW * SK <= 64)
+    int unit;    // row partitions are multiples of this many tiles (2 for gate|up: 16 SwiGLU columns)
+    int follow;  // 1: one row partition; block i takes the columns that partition i of `gate|up` produces
+    int pad;
     unsigned long long w_off;  // byte offset of the operation inside its weight region
 };
 
 struct Part {
-    int tile0, ntiles, chunk0, nchunks, pr, pk;
+    int tile0, ntiles, k0, nk, pr, pk;
     unsigned long long off;  // byte offset of this partition from the operation's base
-    // derived once per launch so that the per-stage code needs no integer division
-    int npass, nst;          // passes over the row tiles; stages (groups of KW chunks) per pass
+    int npass, nst;          // passes over the row tiles; stages per pass
     int pbase, prem;         // tiles per pass: pbase + (p < prem)
-    int lkw;                 // log2(KW)
-    int pad;
+    int SK, pad;
 };
 __host__ __device__ inline int pass_count(const Part& p, int i) { return p.pbase + (i < p.prem ? 1 : 0); }
 __host__ __device__ inline int pass_start(const Part& p, int i) { return i * p.pbase + (i < p.prem ? i : p.prem); }
@@ -67,47 +76,76 @@ __host__ __device__ inline int even_find(int total, int parts, int x) {
     return r + (x - r * (b + 1)) / b;
 }
 
-__host__ __device__ inline Part get_part(const OpDesc& o, int cta, int G) {
+__host__ __device__ inline void finish_part(Part& p, const OpDesc& o) {
+    p.off = (unsigned long long)kStepBytes *
+            ((unsigned long long)p.tile0 * o.K16 + (unsigned long long)p.ntiles * p.k0);
+    p.SK = o.SK;
+    p.npass = (p.ntiles + o.RW - 1) / o.RW;
+    p.nst = (p.nk + o.SK - 1) / o.SK;
+    p.pbase = p.npass ? p.ntiles / p.npass : 0;
+    p.prem = p.npass ? p.ntiles % p.npass : 0;
+}
+
+// Partition (pr, pk) of an operation; `gu` is the gate|up operation (used when o.follow).
+__host__ __device__ inline Part make_part(const OpDesc& o, const OpDesc& gu, int pr, int pk) {
     Part p;
-    int idx = cta - o.rot;
+    p.pr = pr;
+    p.pk = pk;
+    p.pad = 0;
+    if (o.follow) {
+        p.tile0 = 0;
+        p.ntiles = o.T;
+        p.k0 = even_start(gu.T / gu.unit, gu.P_row, pk);
+        p.nk = even_count(gu.T / gu.unit, gu.P_row, pk);
+    } else {
+        p.tile0 = o.unit * even_start(o.T / o.unit, o.P_row, pr);
+        p.ntiles = o.unit * even_count(o.T / o.unit, o.P_row, pr);
+        p.k0 = even_start(o.K16, o.P_k, pk);
+        p.nk = even_count(o.K16, o.P_k, pk);
+    }
+    finish_part(p, o);
+    return p;
+}
+
+__host__ __device__ inline Part get_part(const OpDesc& o, const OpDesc& gu, int cta, int G) {
+    const int rot = o.follow ? gu.rot : o.rot;
+    const int nparts = o.follow ? gu.P_row : o.P_row * o.P_k;
+    int idx = cta - rot;
     if (idx < 0) idx += G;
-    p.npass = p.nst = p.pbase = p.prem = p.lkw = p.pad = 0;
-    if (idx >= o.P_row * o.P_k) {
-        p.tile0 = p.ntiles = p.chunk0 = p.nchunks = p.pr = p.pk = 0;
+    if (idx >= nparts) {
+        Part p;
+        p.tile0 = p.ntiles = p.k0 = p.nk = p.pr = p.pk = p.npass = p.nst = p.pbase = p.prem = p.pad = 0;
+        p.SK = o.SK;
         p.off = 0;
         return p;
     }
-    p.pr = idx / o.P_k;
-    p.pk = idx % o.P_k;
-    p.tile0 = even_start(o.T, o.P_row, p.pr);
-    p.ntiles = even_count(o.T, o.P_row, p.pr);
-    p.chunk0 = even_start(o.C, o.P_k, p.pk);
-    p.nchunks = even_count(o.C, o.P_k, p.pk);
-    p.off = (unsigned long long)kTileBytes *
-            ((unsigned long long)p.tile0 * o.C + (unsigned long long)p.ntiles * p.chunk0);
-    const int KW = kConsumerWarps / o.RW;
-    p.lkw = KW == 4 ? 2 : (KW == 2 ? 1 : 0);
-    p.npass = (p.ntiles + o.RW - 1) / o.RW;
-    p.nst = (p.nchunks + KW - 1) / KW;
-    p.pbase = p.ntiles / p.npass;
-    p.prem = p.ntiles % p.npass;
-    return p;
+    if (o.follow) return make_part(o, gu, 0, idx);
+    return make_part(o, gu, idx / o.P_k, idx % o.P_k);
 }
-__host__ __device__ inline int part_passes(const Part& p, int RW) { return (p.ntiles + RW - 1) / RW; }
 
-// Byte offset (from the operation's base) of tile t, chunk c: the inverse view used when packing.
-__host__ __device__ inline unsigned long long tile_offset(const OpDesc& o, int t, int c) {
-    const int pr = even_find(o.T, o.P_row, t), pk = even_find(o.C, o.P_k, c);
-    const int tile0 = even_start(o.T, o.P_row, pr), ntiles = even_count(o.T, o.P_row, pr);
-    const int chunk0 = even_start(o.C, o.P_k, pk), nchunks = even_count(o.C, o.P_k, pk);
-    const int npass = (ntiles + o.RW - 1) / o.RW;
-    const int lt = t - tile0;
-    const int p = even_find(ntiles, npass, lt);
-    const int start = even_start(ntiles, npass, p), cnt = even_count(ntiles, npass, p);
-    const unsigned long long tiles_before = (unsigned long long)tile0 * o.C + (unsigned long long)ntiles * chunk0 +
-                                            (unsigned long long)start * nchunks +
-                                            (unsigned long long)cnt * (c - chunk0) + (lt - start);
-    return tiles_before * kTileBytes;
+// Byte offset (from the operation's base) of the 16-byte unit holding columns 8*k8 .. 8*k8+7 of
+// weight row `row`: the inverse view used when packing.
+__host__ __device__ inline unsigned long long weight_offset(const OpDesc& o, const OpDesc& gu, int row, int k8) {
+    const int t = row >> 4, ks = k8 >> 1, half = k8 & 1;
+    int pr, pk;
+    if (o.follow) {
+        pr = 0;
+        pk = even_find(gu.T / gu.unit, gu.P_row, ks);
+    } else {
+        pr = even_find(o.T / o.unit, o.P_row, t / o.unit);
+        pk = even_find(o.K16, o.P_k, ks);
+    }
+    const Part p = make_part(o, gu, pr, pk);
+    const int lt = t - p.tile0;
+    const int pass = even_find(p.ntiles, p.npass, lt);
+    const int start = pass_start(p, pass), pcount = pass_count(p, pass);
+    const int tip = lt - start, lk = ks - p.k0;
+    const int st = lk / p.SK, kin = lk % p.SK;
+    const unsigned long long stage_base =
+        p.off + (unsigned long long)kStepBytes * ((unsigned long long)start * p.nk + (unsigned long long)pcount * st * p.SK);
+    const unsigned long long in_stage =
+        ((unsigned long long)(kin * 2 + half) * (2 * pcount) + (tip * 2 + ((row & 15) >> 3))) * 128 + (row & 7) * 16;
+    return stage_base + in_stage;
 }
 
 // Device state block (int32 words).
@@ -141,27 +179,31 @@ struct FwdParams {
     float* h;          // [kMaxRows][d] residual stream
     float* qkv_acc;    // [kMaxRows][n_qkv] un-normalised q|k|v sums
     float* sumsq;      // [2][kMaxRows] sum of squares of h rows for the attention-side norm
-    uint8_t* act;      // bf16 [f/64][rows][64] swizzled: SwiGLU output, the down projection's operand
-    uint8_t* attn_op;  // bf16 [n_q*hd/64][rows][64] swizzled: attention output, the o projection's operand
     float* part_o;     // [n_q][kMaxSplits+1][kMaxRows][hd] un-normalised split outputs
     float* part_ml;    // [n_q][kMaxSplits+1][kMaxRows][2]  (running max in log2 units, sum)
     float* cand_val;   // [G][kMaxRows] per-block best logit
     int* cand_idx;     // [G][kMaxRows] and its token id
     float* logits;     // [kMaxRows][V]
+    const float* raw_x;  // [M][raw_K] operand of the stand-alone GEMM
     float* raw_out;    // [kMaxRows][raw_N] output of the stand-alone GEMM
-    int raw_N;
+    int raw_N, raw_K;
     int* state;
     const int* hist;
     int* bar;          // grid barrier counter
     unsigned long long* prof;  // optional [phase][block][kProfWords] timestamps (ns)
     // per launch
     int L;             // committed KV length = position of row 0
-    int M;             // rows computed (1..8*NT)
+    int M;             // rows computed (1..kMaxRows)
+    int NB;            // N of the tensor-core instruction: 16, or 32 when M > 16
     int mode;          // 0: rows are [pending, draft...]; 1: rows are hist[L..L+M)
     int ph_begin, ph_end;
     int bar_base;      // barrier counter value before this launch
     int store_logits;
-    int ahead;         // weight stages the streamer may run ahead of the MMA warps (<= ring size)
+    // shared-memory plan of this launch (bytes from the 1024-aligned base)
+    int nstage;        // ring slots of kStageBytes, at offset 0
+    int u_off;         // operand region (token operand of the running GEMM; attention tiles)
+    int act_off;       // SwiGLU output operand
+    int misc_off;
     unsigned long long wait_limit_ns;
 };
 

@@ -22,9 +22,9 @@ namespace {
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Regions {
-    size_t state, bar, never, hist, rope, norm_w, bias, wlayers, wlm, emb, kcache, vcache, h, qkv_acc, sumsq, act,
-        attn_op, part_o, part_ml, cand_val, cand_idx, logits, raw_out, staging, wraw, xstage, prof, total;
-    size_t layer_stride, staging_bytes, act_k;
+    size_t state, bar, never, hist, rope, norm_w, bias, wlayers, wlm, emb, kcache, vcache, h, qkv_acc, sumsq, part_o,
+        part_ml, cand_val, cand_idx, logits, raw_out, staging, wraw, xstage, prof, total;
+    size_t layer_stride, staging_bytes, raw_kmax;
 };
 
 constexpr int kMaxGrid = 256;  // per-block candidate arrays are sized for this many blocks
@@ -73,12 +73,10 @@ Regions carve(const sdv_config* c) {
     r.h = take((size_t)kMaxRows * d * 4);
     r.qkv_acc = take((size_t)kMaxRows * nqkv * 4);
     r.sumsq = take(2 * kMaxRows * 4);
-    size_t act_k = f;  // the stand-alone GEMM stages operands of any K up to max(f, d, nq)
-    if (d > act_k) act_k = d;
-    if (nq > act_k) act_k = nq;
-    r.act_k = act_k;
-    r.act = take(act_k / 64 * kMaxRows * 128);
-    r.attn_op = take(nq / 64 * kMaxRows * 128);
+    size_t raw_kmax = f;  // the stand-alone GEMM takes operands of any K up to max(f, d, nq)
+    if (d > raw_kmax) raw_kmax = d;
+    if (nq > raw_kmax) raw_kmax = nq;
+    r.raw_kmax = raw_kmax;
     r.part_o = take((size_t)c->n_q_heads * (kMaxSplits + 1) * kMaxRows * hd * 4);
     r.part_ml = take((size_t)c->n_q_heads * (kMaxSplits + 1) * kMaxRows * 2 * 4);
     r.cand_val = take((size_t)kMaxGrid * kMaxRows * 4);
@@ -92,46 +90,133 @@ Regions carve(const sdv_config* c) {
     r.staging = take(st);
     r.wraw = take(st);
     r.raw_out = take((size_t)kMaxRows * (st / 128) * 4);  // N <= staging / (2 bytes * 64 columns)
-    r.xstage = take((size_t)kMaxRows * act_k * 4);
+    r.xstage = take((size_t)kMaxRows * raw_kmax * 4);
     r.prof = take((size_t)(3 + kPhasesPerLayer * c->n_layers) * kMaxGrid * kProfWords * 8);
     r.total = off;
     return r;
 }
 
-// Chooses how an operation's tile grid is cut among the blocks and how a block's 8 MMA warps are
-// arranged (RW row tiles x KW column chunks per stage).  Model of a block's time in microseconds:
-// the larger of streaming its share (at a fair share of HBM bandwidth) and walking its pipeline
-// stages or loading its operand chunks (costlier when the RMSNorm scale is applied on the way),
-// plus a charge per column partition for the atomic adds that merge partial sums.
-// Operations whose epilogue needs complete sums (full_k) keep all columns in one block.
-void choose_partition(OpDesc& o, int G, bool full_k, bool norm_operand) {
+// Chooses how an operation's grid of row tiles x column steps is cut among the blocks and how a
+// block walks its share (RW row tiles per pass, SK column steps per stage).  Model of a block's
+// time in microseconds: streaming its share at a fair share of HBM bandwidth or walking its
+// stages and passes, whichever is longer, plus building its token operand (the bytes it reads from
+// L2: residual rows, or split-KV partial results when `merge`) and, when partial sums meet in L2
+// (column partitions, or the residual add), the reductions of all blocks.
+void choose_partition(OpDesc& o, int G, int rows, bool merge, bool always_add) {
     double best_t = -1.0;
-    o.RW = kConsumerWarps;
+    o.RW = 8;
+    o.SK = kStageBytes / kStepBytes / 8;
     o.P_row = 1;
     o.P_k = 1;
-    const int rw_first = kConsumerWarps, rw_last = full_k ? kConsumerWarps : kConsumerWarps / kMaxKW;
-    for (int RW = rw_first; RW >= rw_last; RW /= 2) {
-        const int KW = kConsumerWarps / RW;
+    o.unit = 1;
+    o.follow = 0;
+    for (int RW = 8; RW >= 1; RW /= 2) {
+        const int SK = kStageBytes / kStepBytes / RW;
         for (int pr = 1; pr <= o.T && pr <= G; ++pr) {
-            const int pk_max = full_k ? 1 : (G / pr < o.C ? G / pr : o.C);
+            const int pk_max = G / pr < o.K16 ? G / pr : o.K16;
             for (int pk = 1; pk <= pk_max; ++pk) {
-                const int tiles = (o.T + pr - 1) / pr, chunks = (o.C + pk - 1) / pk;
+                const int tiles = (o.T + pr - 1) / pr, ks = (o.K16 + pk - 1) / pk;
                 const int passes = (tiles + RW - 1) / RW;
-                const int stages = passes * ((chunks + KW - 1) / KW);
-                const double stream = (double)tiles * chunks * kTileBytes / 44000.0;
-                const double walk = 0.24 * stages;  // an MMA warp needs about 450 cycles per stage
-                const double load = (double)passes * chunks * (norm_operand ? 0.28 : 0.05);  // operand chunk visits
-                double t = stream > walk ? stream : walk;
-                if (load > t) t = load;
-                if (pk > 1) t += 0.3 + 0.05 * pk;
+                const int stages = passes * ((ks + SK - 1) / SK);
+                const double stream = (double)tiles * ks * kStepBytes / 44000.0;
+                const double walk = 0.06 * stages + 0.25 * passes;
+                const double operand_bytes =
+                    merge ? (double)rows * ks * 2 * (kMaxSplits + 1) * 40.0 : (double)rows * ks * 16 * 4.0;
+                double t = (stream > walk ? stream : walk) + 0.8 + operand_bytes / 60000.0;
+                if (pk > 1 || always_add) t += 0.7 + 0.016 * pk * (rows / 9.0);
                 if (best_t < 0 || t < best_t - 1e-9) {
                     best_t = t;
                     o.RW = RW;
+                    o.SK = SK;
                     o.P_row = pr;
                     o.P_k = pk;
                 }
             }
         }
+    }
+}
+// Operations whose epilogue needs complete sums: all columns in one block, rows spread evenly.
+void full_k_partition(OpDesc& o, int G, int unit) {
+    o.RW = 8;
+    o.SK = kStageBytes / kStepBytes / 8;
+    o.unit = unit;
+    o.follow = 0;
+    o.P_k = 1;
+    o.P_row = o.T / unit < G ? o.T / unit : G;
+}
+
+// Shared-memory plan of a launch over `rows` token rows: ring of weight stages | operand region |
+// SwiGLU operand | bookkeeping.  The operand region holds the token operand of the widest GEMM
+// share (or the attention tiles); the ring takes what is left.
+struct SmemPlan {
+    int NG, NB, nstage, u_off, act_off, misc_off, total;
+    bool ok;
+};
+SmemPlan plan_smem(const FwdParams& P, int rows, bool raw_only) {
+    SmemPlan s;
+    s.NG = (rows + 7) / 8;
+    s.NB = rows > 16 ? 32 : 16;
+    const int step_bytes = 32 * rows;  // token operand bytes per column step: 16 columns x rows x bf16
+    int max_ks = 0;
+    for (int i = 0; i < OP_COUNT; ++i) {
+        const OpDesc& o = P.op[i];
+        if (o.T == 0 || o.follow || (raw_only != (i == OP_RAW))) continue;
+        const int ks = (o.K16 + o.P_k - 1) / o.P_k;
+        if (ks > max_ks) max_ks = ks;
+    }
+    int u = max_ks * step_bytes;
+    if (!raw_only && u < kAttnSmemBytes) u = kAttnSmemBytes;
+    u = (u + 1023) / 1024 * 1024;
+    s.ok = true;
+    int act = 1024;
+    if (!raw_only) {
+        const OpDesc& gu = P.op[OP_GU];
+        const int units = (gu.T / gu.unit + gu.P_row - 1) / gu.P_row;  // SwiGLU column steps per block at most
+        act = (units * step_bytes + 1023) / 1024 * 1024;
+        if (act > kActSmemMax) s.ok = false;
+    }
+    const int ring = kSmemBudget - 1024 - kMiscSmemBytes - act - u;
+    s.nstage = ring / kStageBytes;
+    if (s.nstage > kMaxStages) s.nstage = kMaxStages;
+    if (s.nstage < 2) s.ok = false;
+    s.u_off = s.nstage * kStageBytes;
+    s.act_off = s.u_off + u;
+    s.misc_off = s.act_off + act;
+    s.total = s.misc_off + kMiscSmemBytes + 1024;  // + slack for 1024-byte alignment
+    return s;
+}
+
+// The operations of one layer, in streaming order, and the LM head: shapes, partitions, offsets.
+void setup_ops(FwdParams& P, const sdv_config* cfg, int G) {
+    const int d = cfg->d_model, f = cfg->d_ffn, hd = cfg->head_dim;
+    const int nq = cfg->n_q_heads * hd, nkv = cfg->n_kv_heads * hd, nqkv = nq + 2 * nkv;
+    struct { int idx, N, K; } ops[5] = {{OP_QKV, nqkv, d}, {OP_O, d, nq}, {OP_GU, 2 * f, d}, {OP_DOWN, d, f},
+                                        {OP_LM, cfg->vocab, d}};
+    unsigned long long woff = 0;
+    int rot = 0;
+    const int rows_max = cfg->k_max + 1;
+    for (int i = 0; i < 5; ++i) {
+        OpDesc& o = P.op[ops[i].idx];
+        memset(&o, 0, sizeof(o));
+        o.T = ops[i].N / 16;
+        o.K16 = ops[i].K / 16;
+        switch (ops[i].idx) {
+            case OP_QKV: choose_partition(o, G, rows_max, false, false); break;
+            case OP_O: choose_partition(o, G, rows_max, true, true); break;
+            case OP_GU: full_k_partition(o, G, 2); break;   // pairs of tiles: 16 SwiGLU columns = one column step of down
+            case OP_LM: full_k_partition(o, G, 1); break;
+            default:  // down: every block multiplies the SwiGLU columns it produced
+                o.RW = 8; o.SK = kStageBytes / kStepBytes / 8; o.unit = 1; o.follow = 1; o.P_row = 1; o.P_k = P.op[OP_GU].P_row;
+                break;
+        }
+        if (ops[i].idx == OP_DOWN) {
+            o.rot = P.op[OP_GU].rot;
+        } else {
+            o.rot = rot % G;
+            rot += o.P_row * o.P_k;
+        }
+        o.w_off = (ops[i].idx == OP_LM) ? 0 : woff;
+        if (ops[i].idx != OP_LM) woff += (unsigned long long)ops[i].N * ops[i].K * 2;
     }
 }
 
@@ -155,7 +240,6 @@ struct sdv_ctx {
     int bar_base;
     int parity;
     int profile;
-    int ahead;
     int last_cuda;
     long long launches;
     bool have_verify_time;
@@ -174,43 +258,46 @@ int cuda_fail(sdv_ctx* ctx, cudaError_t e) {
         if (e_ != cudaSuccess) return cuda_fail(ctx, e_); \
     } while (0)
 
-template <int NT>
-cudaError_t launch_forward_nt(sdv_ctx* ctx, const FwdParams& P) {
-    using SL = SmemLayout<NT>;
-    cudaError_t e = cudaFuncSetAttribute(sdv_forward_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::TOTAL);
+cudaError_t launch_kernel(const FwdParams& P, int smem_bytes, cudaStream_t stream) {
+    cudaError_t e = cudaFuncSetAttribute(sdv_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     if (e != cudaSuccess) return e;
     void* args[] = {(void*)&P};
     // phases meet at grid barriers, so more than one phase needs all blocks co-resident
     if (P.ph_end - P.ph_begin > 1)
-        return cudaLaunchCooperativeKernel((const void*)sdv_forward_kernel<NT>, dim3(P.G), dim3(kThreads), args, SL::TOTAL,
-                                           ctx->stream);
-    return cudaLaunchKernel((const void*)sdv_forward_kernel<NT>, dim3(P.G), dim3(kThreads), args, SL::TOTAL, ctx->stream);
+        return cudaLaunchCooperativeKernel((const void*)sdv_forward_kernel, dim3(P.G), dim3(kThreads), args, smem_bytes, stream);
+    return cudaLaunchKernel((const void*)sdv_forward_kernel, dim3(P.G), dim3(kThreads), args, smem_bytes, stream);
+}
+
+bool apply_plan(FwdParams& P, int rows, bool raw_only, int* smem_bytes) {
+    const SmemPlan sp = plan_smem(P, rows, raw_only);
+    if (!sp.ok) return false;
+    P.M = rows;
+    P.NB = sp.NB;
+    P.nstage = sp.nstage;
+    P.u_off = sp.u_off;
+    P.act_off = sp.act_off;
+    P.misc_off = sp.misc_off;
+    *smem_bytes = sp.total;
+    return true;
 }
 
 // Runs phases [ph_begin, ph_end) over `rows` token rows at position L.
 int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph_end, bool timed) {
     FwdParams P = ctx->P;
+    int smem_bytes = 0;
+    const bool raw_only = (ph_begin == 2 + kPhasesPerLayer * ctx->cfg.n_layers);
+    if (!apply_plan(P, rows, raw_only, &smem_bytes)) return SDV_EINVAL;
     P.L = L;
-    P.M = rows;
     P.mode = mode;
     P.ph_begin = ph_begin;
     P.ph_end = ph_end;
     P.bar_base = ctx->bar_base;
     P.store_logits = ctx->parity;
-    P.ahead = ctx->ahead;
     P.prof = ctx->profile ? (unsigned long long*)(ctx->ws + ctx->r.prof) : nullptr;
     const int nbar = ph_end - ph_begin - 1;
     ctx->bar_base += nbar * ctx->G;
-    const int NT = (rows + 7) / 8;
     if (timed) CK(cudaEventRecord(ctx->ev0, ctx->stream));
-    cudaError_t e;
-    switch (NT) {
-        case 1: e = launch_forward_nt<1>(ctx, P); break;
-        case 2: e = launch_forward_nt<2>(ctx, P); break;
-        case 3: e = launch_forward_nt<3>(ctx, P); break;
-        case 4: e = launch_forward_nt<4>(ctx, P); break;
-        default: return SDV_EINVAL;
-    }
+    cudaError_t e = launch_kernel(P, smem_bytes, ctx->stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches++;
     if (timed) {
@@ -232,11 +319,11 @@ int read_state(sdv_ctx* ctx) {
 
 int pack_op(sdv_ctx* ctx, const OpDesc& o, uint8_t* dst_base, const uint16_t* s0, int rows0, const uint16_t* s1,
             int rows1, const uint16_t* s2, int K, int mode, int t_begin, int t_end, int row_base) {
-    const long long total = (long long)(t_end - t_begin) * o.C * 128;
+    const long long total = (long long)(t_end - t_begin) * 16 * (K / 8);
     int blocks = (int)((total + 255) / 256);
     if (blocks > 148 * 16) blocks = 148 * 16;
-    pack_weights_kernel<<<blocks, 256, 0, ctx->stream>>>(o, dst_base, s0, rows0, s1, rows1, s2, K, mode, t_begin, t_end,
-                                                       row_base);
+    pack_weights_kernel<<<blocks, 256, 0, ctx->stream>>>(o, ctx->P.op[OP_GU], dst_base, s0, rows0, s1, rows1, s2, K, mode,
+                                                       t_begin, t_end, row_base);
     ctx->launches++;
     CK(cudaGetLastError());
     return SDV_OK;
@@ -318,10 +405,6 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
     if (sms > kMaxGrid) sms = kMaxGrid;
     ctx->G = sms;  // one persistent block per SM
     ctx->r = carve(cfg);
-    {
-        const char* e_ahead = getenv("SDV_AHEAD");
-        ctx->ahead = e_ahead ? atoi(e_ahead) : 0;
-    }
     e = cudaHostAlloc((void**)&ctx->pinned, 4096, cudaHostAllocDefault);
     if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev0);
     if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev1);
@@ -338,22 +421,8 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
     P.eps = cfg->rms_eps;
     P.scale_log2e = (float)((1.0 / sqrt((double)hd)) * 1.4426950408889634);
     P.G = ctx->G;
-    // operations of one layer, in streaming order, and the LM head
-    struct { int idx, N, K; bool full_k; } ops[5] = {
-        {OP_QKV, nqkv, d, false}, {OP_O, d, nq, false}, {OP_GU, 2 * f, d, true}, {OP_DOWN, d, f, false},
-        {OP_LM, cfg->vocab, d, true}};
-    unsigned long long woff = 0;
-    int rot = 0;
-    for (int i = 0; i < 5; ++i) {
-        OpDesc& o = P.op[ops[i].idx];
-        o.T = ops[i].N / 16;
-        o.C = ops[i].K / 64;
-        choose_partition(o, ctx->G, ops[i].full_k, ops[i].idx != OP_O && ops[i].idx != OP_DOWN);
-        o.rot = rot % ctx->G;
-        rot += o.P_row * o.P_k;
-        o.w_off = (ops[i].idx == OP_LM) ? 0 : woff;
-        if (ops[i].idx != OP_LM) woff += (unsigned long long)ops[i].N * ops[i].K * 2;
-    }
+    setup_ops(P, cfg, ctx->G);
+    const int rows_max = cfg->k_max + 1;
     P.layer_stride = ctx->r.layer_stride;
     uint8_t* ws = ctx->ws;
     P.wlayers = ws + ctx->r.wlayers;
@@ -368,19 +437,29 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
     P.h = (float*)(ws + ctx->r.h);
     P.qkv_acc = (float*)(ws + ctx->r.qkv_acc);
     P.sumsq = (float*)(ws + ctx->r.sumsq);
-    P.act = ws + ctx->r.act;
-    P.attn_op = ws + ctx->r.attn_op;
     P.part_o = (float*)(ws + ctx->r.part_o);
     P.part_ml = (float*)(ws + ctx->r.part_ml);
     P.cand_val = (float*)(ws + ctx->r.cand_val);
     P.cand_idx = (int*)(ws + ctx->r.cand_idx);
     P.logits = (float*)(ws + ctx->r.logits);
     P.raw_out = (float*)(ws + ctx->r.raw_out);
+    P.raw_x = (const float*)(ws + ctx->r.xstage);
     P.raw_N = 0;
+    P.raw_K = 0;
     P.state = (int*)(ws + ctx->r.state);
     P.hist = (const int*)(ws + ctx->r.hist);
     P.bar = (int*)(ws + ctx->r.bar);
     P.wait_limit_ns = 2000000000ull;
+    {
+        // the widest verify step must fit the shared-memory plan
+        FwdParams probe = P;
+        int smem_bytes = 0;
+        if (!apply_plan(probe, rows_max, false, &smem_bytes)) {
+            cudaFreeHost(ctx->pinned);
+            delete ctx;
+            return SDV_EINVAL;
+        }
+    }
 
     // rotary table in double, rounded once to fp32
     {
@@ -525,6 +604,12 @@ int sdv_prefill_chunk(sdv_ctx* ctx, const int32_t* host_tokens, int n, int is_la
     if (tile > 24) tile = 24;
     tile = tile / 8 * 8;
     if (tile < 8) tile = 8;
+    {
+        // wide models: fewer rows per launch so that the token operand leaves room for the weight ring
+        FwdParams probe = ctx->P;
+        int smem_bytes = 0;
+        while (tile > 8 && (!apply_plan(probe, tile, false, &smem_bytes) || probe.nstage < 4)) tile -= 8;
+    }
     const int n_ph = 1 + kPhasesPerLayer * c.n_layers;
     int done = 0;
     while (done < n) {
@@ -748,7 +833,7 @@ int sdv_debug_gemm(sdv_ctx* ctx, const float* host_x, const uint16_t* host_w, fl
     if (!ctx || !host_x || !host_w || !host_y) return SDV_EINVAL;
     if (ctx->poisoned) return SDV_ETIMEOUT;
     if (M < 1 || M > kMaxRows || N < 16 || N % 16 || K < 64 || K % 64) return SDV_EINVAL;
-    if ((size_t)K > ctx->r.act_k || (size_t)N * K * 2 > ctx->r.staging_bytes || (size_t)N > ctx->r.staging_bytes / 128)
+    if ((size_t)K > ctx->r.raw_kmax || (size_t)N * K * 2 > ctx->r.staging_bytes || (size_t)N > ctx->r.staging_bytes / 128)
         return SDV_EINVAL;
     const sdv_config& c = ctx->cfg;
     uint8_t* ws = ctx->ws;
@@ -756,26 +841,24 @@ int sdv_debug_gemm(sdv_ctx* ctx, const float* host_x, const uint16_t* host_w, fl
     OpDesc o;
     memset(&o, 0, sizeof(o));
     o.T = N / 16;
-    o.C = K / 64;
-    choose_partition(o, ctx->G, false, false);
-    const int NT = (M + 7) / 8;
+    o.K16 = K / 16;
+    choose_partition(o, ctx->G, M, false, false);
     CK(cudaMemcpyAsync(ws + ctx->r.staging, host_w, (size_t)N * K * 2, cudaMemcpyDefault, s));
     int rc = pack_op(ctx, o, ws + ctx->r.wraw, (const uint16_t*)(ws + ctx->r.staging), N, nullptr, 0, nullptr, K, 0, 0,
                      o.T, 0);
     if (rc) return rc;
     CK(cudaMemcpyAsync(ws + ctx->r.xstage, host_x, (size_t)M * K * 4, cudaMemcpyDefault, s));
-    stage_operand_kernel<<<64, 256, 0, s>>>((const float*)(ws + ctx->r.xstage), ws + ctx->r.act, M, K, 8 * NT);
-    ctx->launches++;
-    CK(cudaGetLastError());
     CK(cudaMemsetAsync(ws + ctx->r.raw_out, 0, (size_t)kMaxRows * N * 4, s));
     const OpDesc saved = ctx->P.op[OP_RAW];
-    const int saved_N = ctx->P.raw_N;
+    const int saved_N = ctx->P.raw_N, saved_K = ctx->P.raw_K;
     ctx->P.op[OP_RAW] = o;
     ctx->P.raw_N = N;
+    ctx->P.raw_K = K;
     const int ph = 2 + kPhasesPerLayer * c.n_layers;
     rc = launch_forward(ctx, M, 0, 1, ph, ph + 1, true);
     ctx->P.op[OP_RAW] = saved;
     ctx->P.raw_N = saved_N;
+    ctx->P.raw_K = saved_K;
     if (rc) return rc;
     CK(cudaMemcpyAsync(host_y, ws + ctx->r.raw_out, (size_t)M * N * 4, cudaMemcpyDeviceToHost, s));
     rc = read_state(ctx);
@@ -797,6 +880,76 @@ int sdv_debug_profile(sdv_ctx* ctx, int on, unsigned long long* host_out, int n_
                            (size_t)(3 + kPhasesPerLayer * ctx->cfg.n_layers) * kMaxGrid * kProfWords * 8, ctx->stream));
     ctx->profile = on ? 1 : 0;
     return ctx->G;
+}
+
+// Host-only self-check of the streaming layout: walks every block's share of an operation the way
+// the weight streamer and the tensor-core thread do (pass by pass, stage by stage, the addresses the
+// shared-memory descriptors generate) and checks that each 16-byte unit of the matrix is met exactly
+// once, at the offset the packing function gives.  desc = {T, K16, P_row, P_k, RW, SK, unit, follow};
+// gu_desc likewise (only read when follow is set).  Returns 0, or a negative code.
+int sdv_debug_layout_check(const int* desc, const int* gu_desc, int G) {
+    if (!desc || !gu_desc || G < 1) return SDV_EINVAL;
+    OpDesc o, gu;
+    memset(&o, 0, sizeof(o));
+    memset(&gu, 0, sizeof(gu));
+    o.T = desc[0]; o.K16 = desc[1]; o.P_row = desc[2]; o.P_k = desc[3]; o.RW = desc[4]; o.SK = desc[5]; o.unit = desc[6];
+    o.follow = desc[7];
+    gu.T = gu_desc[0]; gu.K16 = gu_desc[1]; gu.P_row = gu_desc[2]; gu.P_k = gu_desc[3]; gu.RW = gu_desc[4]; gu.SK = gu_desc[5];
+    gu.unit = gu_desc[6];
+    if (o.T < 1 || o.K16 < 1 || o.RW < 1 || o.SK < 1 || o.RW * o.SK * kStepBytes > kStageBytes || o.unit < 1 || o.T % o.unit) return SDV_EINVAL;
+    const size_t units = (size_t)o.T * 16 * o.K16 * 2;  // 16-byte units of the matrix
+    std::vector<unsigned char> seen(units, 0);
+    for (int cta = 0; cta < G; ++cta) {
+        const Part pt = get_part(o, gu, cta, G);
+        if (pt.ntiles == 0 || pt.nk == 0) continue;
+        unsigned long long src = pt.off;  // the streamer's running offset
+        for (int p = 0; p < pt.npass; ++p) {
+            const int pcount = pass_count(pt, p), pstart = pass_start(pt, p);
+            if (pcount < 1 || pcount > 8) return -100;
+            for (int st = 0; st < pt.nst; ++st) {
+                const int nks = (pt.SK < pt.nk - st * pt.SK) ? pt.SK : pt.nk - st * pt.SK;
+                const unsigned long long bytes = (unsigned long long)pcount * nks * kStepBytes;
+                if (bytes > (unsigned long long)kStageBytes) return -101;
+                const unsigned lbo = 2u * pcount * 128u, astep = 2u * lbo;
+                for (int ks = 0; ks < nks; ++ks)
+                    for (int half = 0; half < 2; ++half)
+                        for (int r = 0; r < 16 * pcount; ++r) {
+                            const unsigned long long in_slot = (unsigned long long)ks * astep + half * lbo + (r >> 3) * 128 + (r & 7) * 16;
+                            if (in_slot + 16 > bytes) return -102;
+                            const int row = (pt.tile0 + pstart) * 16 + r;
+                            const int k8 = (pt.k0 + st * pt.SK + ks) * 2 + half;
+                            const unsigned long long want = weight_offset(o, gu, row, k8);
+                            if (want != src + in_slot) return -103;
+                            const size_t u = want / 16;
+                            if (u >= units || seen[u]) return -104;
+                            seen[u] = 1;
+                        }
+                src += bytes;
+            }
+        }
+    }
+    for (size_t u = 0; u < units; ++u)
+        if (!seen[u]) return -105;
+    return 0;
+}
+
+// Host-only: the work partition and shared-memory plan a context of this configuration would use
+// with G thread blocks and `rows` token rows.  out[op * 8 + {0..7}] = {T, K16, P_row, P_k, RW, SK,
+// unit, follow} for the five operations (QKV, O, gate|up, down, LM head), then out[40..45] =
+// {NG, NB, ring slots, operand region bytes, total dynamic shared memory, plan ok}.
+int sdv_debug_plan(const sdv_config* cfg, int G, int rows, int* out) {
+    if (!config_ok(cfg) || !out || G < 1 || G > kMaxGrid || rows < 1 || rows > kMaxRows) return SDV_EINVAL;
+    FwdParams P;
+    memset(&P, 0, sizeof(P));
+    setup_ops(P, cfg, G);
+    for (int i = 0; i < 5; ++i) {
+        const OpDesc& o = P.op[i];
+        const int v[8] = {o.T, o.K16, o.P_row, o.P_k, o.RW, o.SK, o.unit, o.follow};
+        for (int j = 0; j < 8; ++j) out[i * 8 + j] = v[j];
+    }
+    const SmemPlan sp = plan_smem(P, rows, false);
+    out[40] = sp.NG; out[41] = sp.NB; out[42] = sp.nstage; out[43] = sp.act_off - sp.u_off; out[44] = sp.total; out[45] = sp.ok ? 1 : 0;
+    return SDV_OK;
 }
 
 int sdv_debug_timeout_probe(sdv_ctx* ctx) {
@@ -825,9 +978,7 @@ int sdv_debug_timeout_probe(sdv_ctx* ctx) {
 namespace {
 constexpr size_t kNaWeightBytes = (size_t)2 << 20;              // packed weights: N * K * 2 <= 2 MiB
 constexpr int kNaMaxK = 4096, kNaMaxN = 4096;
-constexpr size_t kNaActOff = kNaWeightBytes;                    // operand chunks: K/64 * 32 rows * 128 B
-constexpr size_t kNaActBytes = (size_t)kNaMaxK / 64 * kMaxRows * 128;
-constexpr size_t kNaOutOff = kNaActOff + kNaActBytes;           // fp32 accumulators [32][N]
+constexpr size_t kNaOutOff = kNaWeightBytes;                    // fp32 accumulators [32][N]
 constexpr size_t kNaOutBytes = (size_t)kMaxRows * kNaMaxN * 4;
 constexpr size_t kNaStateOff = kNaOutOff + kNaOutBytes;         // state words (error flag)
 constexpr size_t kNaTotal = kNaStateOff + 1024;
@@ -835,18 +986,7 @@ constexpr int kNaMaxDevices = 64;
 uint8_t* g_na_ptr[kNaMaxDevices];  // device address of the scratch array, per device (0 = not looked up yet)
 }  // namespace
 
-static __device__ __align__(256) uint8_t g_na_scratch[kNaTotal];  // ~2.8 MB per GPU that loads the library
-
-namespace {
-template <int NT>
-cudaError_t launch_raw_nt(const FwdParams& P, cudaStream_t stream) {
-    using SL = SmemLayout<NT>;
-    cudaError_t e = cudaFuncSetAttribute(sdv_forward_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::TOTAL);
-    if (e != cudaSuccess) return e;
-    void* args[] = {(void*)&P};
-    return cudaLaunchKernel((const void*)sdv_forward_kernel<NT>, dim3(P.G), dim3(kThreads), args, SL::TOTAL, stream);
-}
-}  // namespace
+static __device__ __align__(256) uint8_t g_na_scratch[kNaTotal];  // ~2.5 MB per GPU that loads the library
 
 extern "C" {
 
@@ -872,38 +1012,31 @@ int sdv_gemm_noalloc(const float* dev_x, const uint16_t* dev_w, float* dev_y, in
     P.G = sms;
     OpDesc& o = P.op[OP_RAW];
     o.T = N / 16;
-    o.C = K / 64;
-    choose_partition(o, sms, false, false);
+    o.K16 = K / 16;
+    choose_partition(o, sms, M, false, false);
     P.wraw = sc;
-    P.act = sc + kNaActOff;
+    P.raw_x = dev_x;  // the caller's rows are read in place
     P.raw_out = (float*)(sc + kNaOutOff);
     P.raw_N = N;
+    P.raw_K = K;
     P.state = (int*)(sc + kNaStateOff);
     P.bar = P.state + 200;  // unused by a one-phase launch, kept inside the cleared words
-    P.M = M;
     P.mode = 1;
     P.ph_begin = 2;  // with n_layers = 0 phase 2 is the stand-alone GEMM
     P.ph_end = 3;
     P.wait_limit_ns = 2000000000ull;
-    const int NT = (M + 7) / 8;
+    int smem_bytes = 0;
+    if (!apply_plan(P, M, true, &smem_bytes)) return SDV_EINVAL;
 
     // the array keeps the previous call's contents: clear what must start at zero
     if (cudaMemsetAsync(sc + kNaOutOff, 0, (size_t)kMaxRows * N * 4, s) != cudaSuccess) return SDV_ECUDA;
     if (cudaMemsetAsync(sc + kNaStateOff, 0, 1024, s) != cudaSuccess) return SDV_ECUDA;
-    const long long total = (long long)o.T * o.C * 128;
+    const long long total = (long long)o.T * 16 * (K / 8);
     int blocks = (int)((total + 255) / 256);
     if (blocks > 148 * 16) blocks = 148 * 16;
-    pack_weights_kernel<<<blocks, 256, 0, s>>>(o, sc, dev_w, N, nullptr, 0, nullptr, K, 0, 0, o.T, 0);
-    stage_operand_kernel<<<64, 256, 0, s>>>(dev_x, sc + kNaActOff, M, K, 8 * NT);
+    pack_weights_kernel<<<blocks, 256, 0, s>>>(o, o, sc, dev_w, N, nullptr, 0, nullptr, K, 0, 0, o.T, 0);
     if (cudaGetLastError() != cudaSuccess) return SDV_ECUDA;
-    cudaError_t e;
-    switch (NT) {
-        case 1: e = launch_raw_nt<1>(P, s); break;
-        case 2: e = launch_raw_nt<2>(P, s); break;
-        case 3: e = launch_raw_nt<3>(P, s); break;
-        default: e = launch_raw_nt<4>(P, s); break;
-    }
-    if (e != cudaSuccess) return SDV_ECUDA;
+    if (launch_kernel(P, smem_bytes, s) != cudaSuccess) return SDV_ECUDA;
     if (cudaMemcpyAsync(dev_y, sc + kNaOutOff, (size_t)M * N * 4, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
         return SDV_ECUDA;
     int err = 0;

@@ -1,5 +1,5 @@
 // The integer kernels of the path (n-gram drafter, accept scan, commit) and set-up helpers
-// (weight re-layout, operand staging for the stand-alone GEMM, fills).
+// (weight re-layout, fills).
 #pragma once
 #include <math_constants.h>
 
@@ -9,44 +9,32 @@
 namespace sdv {
 
 // ------------------------------------------------------------------------------------------
-// Weight re-layout: row-major bf16 [rows][K] -> streaming tile order (see layout.cuh).
+// Weight re-layout: row-major bf16 [rows][K] -> streaming order (see layout.cuh).  One thread per
+// 16-byte unit (8 columns of one row).
 // mode 0: the operation's rows are src0 | src1 | src2 stacked (the sources hold the rows from
 // row_base on); mode 1: every 16-row tile holds 8 rows of src0 (gate) followed by the 8 matching
 // rows of src1 (up).  Only tiles [t_begin, t_end) are written.
-__global__ void pack_weights_kernel(OpDesc o, uint8_t* dst_base, const uint16_t* src0, int rows0,
+__global__ void pack_weights_kernel(OpDesc o, OpDesc gu, uint8_t* dst_base, const uint16_t* src0, int rows0,
                                     const uint16_t* src1, int rows1, const uint16_t* src2, int K, int mode,
                                     int t_begin, int t_end, int row_base) {
-    const long long total = (long long)(t_end - t_begin) * o.C * 128;
+    const int K8 = K / 8;
+    const long long total = (long long)(t_end - t_begin) * 16 * K8;
     for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < total;
          u += (long long)gridDim.x * blockDim.x) {
-        const int q = (int)(u & 7), r = (int)((u >> 3) & 15);
-        const long long tc = u >> 7;
-        const int c = (int)(tc % o.C), t = t_begin + (int)(tc / o.C);
+        const int k8 = (int)(u % K8);
+        const int row = t_begin * 16 + (int)(u / K8);  // row of the operation
+        const int t = row >> 4, r = row & 15;
         const uint16_t* src;
         if (mode == 1) {
             src = (r < 8) ? src0 + (size_t)(8 * t + r) * K : src1 + (size_t)(8 * t + r - 8) * K;
         } else {
-            const int row = 16 * t + r - row_base;
-            if (row < rows0) src = src0 + (size_t)row * K;
-            else if (row < rows0 + rows1) src = src1 + (size_t)(row - rows0) * K;
-            else src = src2 + (size_t)(row - rows0 - rows1) * K;
+            const int lr = row - row_base;
+            if (lr < rows0) src = src0 + (size_t)lr * K;
+            else if (lr < rows0 + rows1) src = src1 + (size_t)(lr - rows0) * K;
+            else src = src2 + (size_t)(lr - rows0 - rows1) * K;
         }
-        const uint4 v = *reinterpret_cast<const uint4*>(src + c * 64 + q * 8);
-        *reinterpret_cast<uint4*>(dst_base + tile_offset(o, t, c) + swz_unit(r, q)) = v;
-    }
-}
-
-// fp32 [M][K] -> the bf16 chunked operand layout [K/64][rows][64] (swizzled), rows >= M zero.
-__global__ void stage_operand_kernel(const float* x, uint8_t* act, int M, int K, int rows) {
-    const int total = (K / 64) * rows * 8;
-    for (int u = blockIdx.x * blockDim.x + threadIdx.x; u < total; u += gridDim.x * blockDim.x) {
-        const int q = u & 7, tok = (u >> 3) % rows, c = (u >> 3) / rows;
-        uint4 out = make_uint4(0, 0, 0, 0);
-        if (tok < M) {
-            const float* p = x + (size_t)tok * K + c * 64 + q * 8;
-            out = make_uint4(pack_bf16(p[0], p[1]), pack_bf16(p[2], p[3]), pack_bf16(p[4], p[5]), pack_bf16(p[6], p[7]));
-        }
-        *reinterpret_cast<uint4*>(act + (size_t)c * rows * 128 + swz_unit(tok, q)) = out;
+        const uint4 v = *reinterpret_cast<const uint4*>(src + k8 * 8);
+        *reinterpret_cast<uint4*>(dst_base + weight_offset(o, gu, row, k8)) = v;
     }
 }
 
