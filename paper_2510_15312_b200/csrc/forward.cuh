@@ -174,7 +174,7 @@ __device__ __noinline__ void build_norm_operand(const FwdParams& P, int kind, in
     const float* xbase = raw ? P.raw_x : P.h;
     const float* wn = raw ? nullptr
                           : P.norm_w + (size_t)(kind == PH_QKV ? layer * 2 : (kind == PH_GUD ? layer * 2 + 1 : P.n_layers * 2)) * P.d;
-    for (int row = warp; row < M; row += kWorkerWarps) {
+    for (int row = warp; row < M; row += kBuilderWarps) {
         const float4* src = reinterpret_cast<const float4*>(xbase + (size_t)row * stride) + k4_0;
         const float4* wsrc = wn ? reinterpret_cast<const float4*>(wn) + k4_0 : nullptr;
         float ss = 0.f;
@@ -222,7 +222,7 @@ __device__ __noinline__ void build_merged_operand(const FwdParams& P, const Part
     const int M = P.M, hd = P.hd;
     const int k8_0 = pt.k0 * 2, nk8 = pt.nk * 2;
     const int nitems = M * nk8, sub = wtid & 3;
-    for (int it0 = 0; it0 < nitems; it0 += kWorkerThreads / 4) {
+    for (int it0 = 0; it0 < nitems; it0 += kBuilderWarps * 32 / 4) {
         const int item = it0 + (wtid >> 2);
         const bool live = item < nitems;
         const int j = live ? item / nk8 : 0, k8l = live ? item % nk8 : 0;
@@ -288,7 +288,7 @@ struct PipePos {
 };
 
 __device__ __forceinline__ void mma_op(const FwdParams& P, const Part& pt, uint8_t* smem, const uint8_t* B, Misc* misc,
-                                       PipePos& pos, bool& dead) {
+                                       PipePos& pos, bool& dead, bool& synced) {
     const uint32_t nstage = (uint32_t)P.nstage;
     const uint32_t idesc = umma_idesc_bf16_m128((uint32_t)P.NB);
     const uint64_t wait_limit = P.wait_limit_ns;
@@ -305,7 +305,8 @@ __device__ __forceinline__ void mma_op(const FwdParams& P, const Part& pt, uint8
         if (!dead && !mbar_wait_bounded(&misc->tmem_empty[buf], ((pos.q >> 1) & 1u) ^ 1u, &misc->abort_flag, wait_limit))
             dead = true;
         pos.w_acc += (uint32_t)(clock64() - tq0);
-        const uint32_t d_tmem = tmem0 + buf * 32u;
+        const uint32_t d_tmem = tmem0 + buf * 64u;
+        const bool two = pcount > 8;  // rows 128.. of the pass go to the buffer's second accumulator
         const uint32_t lbo_a = (uint32_t)(2 * pcount) * 128u;
         const uint64_t astep = (uint64_t)((2u * lbo_a) >> 4);
         const uint64_t adesc0 = umma_smem_desc(ring0, lbo_a, 128u);
@@ -315,6 +316,11 @@ __device__ __forceinline__ void mma_op(const FwdParams& P, const Part& pt, uint8
             const uint32_t slot = pos.slot, par = pos.par;
             if (++pos.slot == nstage) { pos.slot = 0; pos.par ^= 1u; }
             const int nks = min(SK, kleft);
+            if (!synced) {
+                // everything above ran while the other warps were still building the token operand
+                named_bar_sync(1, kWorkerThreads);
+                synced = true;
+            }
             if (dead) continue;
             const long long tw0 = clock64();
             if (!mbar_wait_bounded(&misc->full[slot], par, &misc->abort_flag, wait_limit)) {
@@ -325,13 +331,19 @@ __device__ __forceinline__ void mma_op(const FwdParams& P, const Part& pt, uint8
             tc_fence_after();
             uint64_t adesc = adesc0 + (uint64_t)((slot * (uint32_t)kStageBytes) >> 4);
             if (elect_one()) {
-                if (st == 0) umma_bf16_first(d_tmem, adesc, bdesc, idesc);
-                else umma_bf16_acc(d_tmem, adesc, bdesc, idesc);
-#pragma unroll 7
+                if (st == 0) {
+                    umma_bf16_first(d_tmem, adesc, bdesc, idesc);
+                    if (two) umma_bf16_first(d_tmem + 32u, adesc + 128u, bdesc, idesc);
+                } else {
+                    umma_bf16_acc(d_tmem, adesc, bdesc, idesc);
+                    if (two) umma_bf16_acc(d_tmem + 32u, adesc + 128u, bdesc, idesc);
+                }
+#pragma unroll 3
                 for (int ks = 1; ks < nks; ++ks) {
                     adesc += astep;
                     bdesc += bstep;
                     umma_bf16_acc(d_tmem, adesc, bdesc, idesc);
+                    if (two) umma_bf16_acc(d_tmem + 32u, adesc + 128u, bdesc, idesc);
                 }
                 bdesc += bstep;
                 umma_commit(&misc->empty[slot]);  // the slot is free once these instructions have read it
@@ -358,73 +370,84 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
                                             PipePos& pos, bool& dead, int warp, int lane, float (&bv)[NBT], int (&bi)[NBT]) {
     const int M = P.M;
     const int t = warp * 32 + lane;
+    const uint64_t wait_limit = P.wait_limit_ns;
+    const uint32_t tmem_lane = misc->tmem_base + ((uint32_t)(warp * 32) << 16);
+    const int npass = pt.npass, tile0 = pt.tile0;
     float rstd[NBT];
     if (op == OP_GU || op == OP_LM) {
+        const float inv_d = 1.f / (float)P.d, eps = P.eps;
 #pragma unroll
-        for (int n = 0; n < NBT; ++n) rstd[n] = (n < M) ? rsqrtf(misc->sumsq[n] / (float)P.d + P.eps) : 0.f;
+        for (int n = 0; n < NBT; ++n) rstd[n] = (n < M) ? rsqrtf(misc->sumsq[n] * inv_d + eps) : 0.f;
     }
-    for (int p = 0; p < pt.npass; ++p, ++pos.q) {
+    float* out = P.h;
+    int stride = P.d;
+    bool add = true;  // residual add (O, down)
+    if (op == OP_QKV) { out = P.qkv_acc; stride = P.n_qkv; add = P.op[OP_QKV].P_k > 1; }
+    else if (op == OP_RAW) { out = P.raw_out; stride = P.raw_N; add = P.op[OP_RAW].P_k > 1; }
+    const int store_logits = P.store_logits;
+    for (int p = 0; p < npass; ++p, ++pos.q) {
         const int pcount = pass_count(pt, p), pstart = pass_start(pt, p);
         const uint32_t buf = pos.q & 1u;
-        if (!dead && !mbar_wait_bounded(&misc->tmem_full[buf], (pos.q >> 1) & 1u, &misc->abort_flag, P.wait_limit_ns)) dead = true;
+        if (!dead && !mbar_wait_bounded(&misc->tmem_full[buf], (pos.q >> 1) & 1u, &misc->abort_flag, wait_limit)) dead = true;
         dead = __any_sync(0xffffffffu, dead);
         if (dead) continue;
         tc_fence_after();
-        float v[NBT];
-        {
-            const uint32_t taddr = misc->tmem_base + ((uint32_t)(warp * 32) << 16) + buf * 32u;
-            float lo[16];
-            tmem_ld16(taddr, lo);
+        const int nhalf = pcount > 8 ? 2 : 1;  // a pass of more than 8 tiles fills both 128-row accumulators of the buffer
+        for (int half = 0; half < nhalf; ++half) {
+            float v[NBT];
+            {
+                const uint32_t taddr = tmem_lane + buf * 64u + (uint32_t)half * 32u;
+                float lo[16];
+                tmem_ld16(taddr, lo);
 #pragma unroll
-            for (int n = 0; n < 16; ++n) v[n] = lo[n];
-            if (NBT == 32) {
-                float hi[16];
-                tmem_ld16(taddr + 16u, hi);
+                for (int n = 0; n < 16; ++n) v[n] = lo[n];
+                if (NBT == 32) {
+                    float hi[16];
+                    tmem_ld16(taddr + 16u, hi);
 #pragma unroll
-                for (int n = 0; n < 16; ++n) v[(NBT == 32 ? 16 : 0) + n] = hi[n];
-            }
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&misc->tmem_empty[buf]);  // the accumulator may be overwritten
-        const bool valid = t < 16 * pcount;
-        const int row = (pt.tile0 + pstart) * 16 + t;  // weight row = output feature
-        if (op == OP_GU) {
-            // rows 0..7 of a tile are gate rows, 8..15 the matching up rows: 8 lanes apart
-#pragma unroll
-            for (int n = 0; n < NBT; ++n) {
-                const float up = __shfl_xor_sync(0xffffffffu, v[n], 8);
-                if (valid && (t & 8) == 0 && n < M) {
-                    const float x = v[n] * rstd[n], y = up * rstd[n];
-                    const float a = x / (1.f + expf(-x)) * y;
-                    const int col = (pstart + (t >> 4)) * 8 + (t & 7);  // SwiGLU column within this block's slice
-                    *reinterpret_cast<__nv_bfloat16*>(act + operand_off(col >> 3, n, M) + (col & 7) * 2) = __float2bfloat16(a);
+                    for (int n = 0; n < 16; ++n) v[(NBT == 32 ? 16 : 0) + n] = hi[n];
                 }
             }
-        } else if (op == OP_LM) {
-#pragma unroll
-            for (int n = 0; n < NBT; ++n) {
-                if (valid && n < M) {
-                    const float x = v[n] * rstd[n];
-                    if (P.store_logits) __stcg(P.logits + (size_t)n * P.V + row, x);
-                    // rows come in ascending order per thread, so ">" keeps the lowest id among equals
-                    if (x > bv[n]) { bv[n] = x; bi[n] = row; }
-                }
+            if (half == nhalf - 1) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&misc->tmem_empty[buf]);  // the accumulators may be overwritten
             }
-        } else {
-            float* out;
-            int stride;
-            bool add;
-            if (op == OP_QKV) { out = P.qkv_acc; stride = P.n_qkv; add = P.op[OP_QKV].P_k > 1; }
-            else if (op == OP_RAW) { out = P.raw_out; stride = P.raw_N; add = P.op[OP_RAW].P_k > 1; }
-            else { out = P.h; stride = P.d; add = true; }  // residual add (O, down)
-            if (valid) {
+            const int tt = half * 128 + t;         // row within the pass
+            const bool valid = tt < 16 * pcount;
+            const int row = (tile0 + pstart) * 16 + tt;  // weight row = output feature
+            if (op == OP_GU) {
+                // rows 0..7 of a tile are gate rows, 8..15 the matching up rows, 8 lanes apart: the gate
+                // lane evaluates the even token columns, the up lane the odd ones
+                const bool is_up = (t & 8) != 0;
+                const int col = (pstart + (tt >> 4)) * 8 + (tt & 7);  // SwiGLU column within this block's slice
+                uint8_t* dst = act + operand_off(col >> 3, 0, M) + (col & 7) * 2;
+#pragma unroll
+                for (int n = 0; n < NBT; ++n) {
+                    const float other = __shfl_xor_sync(0xffffffffu, v[n], 8);
+                    if (valid && n < M && ((n & 1) != 0) == is_up) {
+                        const float x = (is_up ? other : v[n]) * rstd[n], y = (is_up ? v[n] : other) * rstd[n];
+                        const float a = __fdividef(x, 1.f + __expf(-x)) * y;
+                        *reinterpret_cast<__nv_bfloat16*>(dst + n * 16) = __float2bfloat16(a);
+                    }
+                }
+            } else if (op == OP_LM) {
+#pragma unroll
+                for (int n = 0; n < NBT; ++n) {
+                    if (valid && n < M) {
+                        const float x = v[n] * rstd[n];
+                        if (store_logits) __stcg(P.logits + (size_t)n * P.V + row, x);
+                        // rows come in ascending order per thread, so ">" keeps the lowest id among equals
+                        if (x > bv[n]) { bv[n] = x; bi[n] = row; }
+                    }
+                }
+            } else if (valid) {
 #pragma unroll
                 for (int n = 0; n < NBT; ++n) {
                     if (n < M) {
-                        float* dst = out + (size_t)n * stride + row;
-                        if (add) red_add_f32(dst, v[n]);
-                        else __stcg(dst, v[n]);
+                        float* d2 = out + (size_t)n * stride + row;
+                        if (add) red_add_f32(d2, v[n]);
+                        else __stcg(d2, v[n]);
                     }
                 }
             }
@@ -882,29 +905,13 @@ __device__ __noinline__ void gemm_phase(const FwdParams& P, int kind, int layer,
     const bool have0 = p0.ntiles > 0 && p0.nk > 0;
     bool dead = *(volatile int*)&misc->abort_flag != 0;
 
-    if (have0 && !dead) {
-        if (kind == PH_O) build_merged_operand(P, p0, U, wtid);
-        else build_norm_operand(P, kind, layer, p0, U, misc, wtid);
-        fence_proxy_async_smem();
-    }
-    if (kind == PH_O) {
-        // clear the accumulators the next QKV projection adds into (idle warps)
-        const int n4 = kMaxRows * P.n_qkv / 4, nth = (kWorkerWarps - kEpilogueWarps) * 32;
-        if (warp >= kEpilogueWarps) {
-            for (int i = blockIdx.x * nth + (wtid - kEpilogueWarps * 32); i < n4; i += P.G * nth)
-                __stcg(reinterpret_cast<float4*>(P.qkv_acc) + i, make_float4(0.f, 0.f, 0.f, 0.f));
-            if (blockIdx.x == 0 && wtid >= kEpilogueWarps * 32 && wtid < kEpilogueWarps * 32 + kMaxRows)
-                __stcg(P.sumsq + ((layer + 1) & 1) * kMaxRows + (wtid - kEpilogueWarps * 32), 0.f);
-        }
-    }
-    named_bar_sync(1, kWorkerThreads);  // the operand is complete and visible to the tensor core
-    if (prof && wtid == 0) prof[2] = global_timer_ns();
-
     if (warp == kMmaWarp) {
+        // the tensor-core warp builds nothing: it prepares its descriptors and meets the others at the
+        // operand barrier just before its first instruction
         PipePos mp = pos;
         mp.w_full = mp.w_acc = 0;
         const long long tc0 = clock64();
-        tc_fence_after();
+        bool synced = false;
         for (int oi = 0; oi < nops; ++oi) {
             const Part& pt = misc->part[ops[oi]];
             if (pt.ntiles == 0 || pt.nk == 0) continue;
@@ -916,15 +923,33 @@ __device__ __noinline__ void gemm_phase(const FwdParams& P, int kind, int layer,
                 tc_fence_after();
                 if (prof && lane == 0) prof[6] = global_timer_ns();
             }
-            mma_op(P, pt, smem, ops[oi] == OP_DOWN ? act : U, misc, mp, dead);
+            mma_op(P, pt, smem, ops[oi] == OP_DOWN ? act : U, misc, mp, dead, synced);
         }
+        if (!synced) named_bar_sync(1, kWorkerThreads);
         if (prof && lane == 0) {
             prof[3] = global_timer_ns();
             prof[7] = mp.w_full;
             prof[8] = mp.w_acc;
             prof[9] = (unsigned long long)(clock64() - tc0);  // cycles of the whole issue loop
         }
-    } else if (warp < kEpilogueWarps) {
+    } else {
+        if (have0 && !dead) {
+            if (kind == PH_O) build_merged_operand(P, p0, U, wtid);
+            else build_norm_operand(P, kind, layer, p0, U, misc, wtid);
+            fence_proxy_async_smem();
+        }
+        if (kind == PH_O && warp >= kEpilogueWarps) {
+            // clear the accumulators the next QKV projection adds into (idle warps)
+            const int n4 = kMaxRows * P.n_qkv / 4, nth = (kBuilderWarps - kEpilogueWarps) * 32;
+            for (int i = blockIdx.x * nth + (wtid - kEpilogueWarps * 32); i < n4; i += P.G * nth)
+                __stcg(reinterpret_cast<float4*>(P.qkv_acc) + i, make_float4(0.f, 0.f, 0.f, 0.f));
+            if (blockIdx.x == 0 && wtid < kEpilogueWarps * 32 + kMaxRows)
+                __stcg(P.sumsq + ((layer + 1) & 1) * kMaxRows + (wtid - kEpilogueWarps * 32), 0.f);
+        }
+        named_bar_sync(1, kWorkerThreads);  // the operand is complete and visible to the tensor core
+        if (prof && wtid == 0) prof[2] = global_timer_ns();
+    }
+    if (warp < kEpilogueWarps) {
         PipePos ep = pos;
         if (P.NB == 32) epilogue_phase<32>(P, kind, layer, act, misc, ep, dead, warp, lane);
         else epilogue_phase<16>(P, kind, layer, act, misc, ep, dead, warp, lane);

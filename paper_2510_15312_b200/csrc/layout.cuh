@@ -3,8 +3,8 @@
 // Weight streaming layout.  Every linear layer W[N][K] (bf16) is seen as a grid of T = N/16 row
 // tiles by K16 = K/16 column steps (one step = the 16 input features of one tensor-core
 // instruction).  The grid is split into P_row x P_k rectangular partitions, one per thread
-// block.  A block walks its partition in passes of at most RW row tiles (RW <= 8: one pass is
-// one 128-row accumulator in tensor memory, rows past the pass are don't-care) and, inside a
+// block.  A block walks its partition in passes of at most RW row tiles (RW <= 16: one pass is
+// one or two 128-row accumulators in tensor memory, rows past the pass are don't-care) and, inside a
 // pass, in stages of at most SK column steps (RW * SK <= 64, i.e. <= 32 KB).  A stage is stored
 // as the shared-memory image the tensor core reads: column step by column step, the two
 // 8-column halves of a step one after the other, each a run of 8-row x 16-byte core matrices
@@ -20,6 +20,7 @@ namespace sdv {
 constexpr int kWorkerWarps = 11;                       // every warp but the weight streamer
 constexpr int kWorkerThreads = kWorkerWarps * 32;      // 352
 constexpr int kThreads = kWorkerThreads + 32;          // 384 with the weight-streaming warp
+constexpr int kBuilderWarps = 10;                      // warps 0..9 build the token operand of a GEMM
 constexpr int kEpilogueWarps = 4;                      // warps 0..3 read the accumulator (tensor-memory lanes 32w..32w+31)
 constexpr int kMmaWarp = 10;                           // its lane 0 issues the tensor-core instructions
 constexpr int kProducerWarp = 11;
@@ -34,7 +35,7 @@ constexpr int kActSmemMax = 32768;                     // SwiGLU output of this 
 constexpr int kMiscSmemBytes = 4096;
 constexpr int kMaxDraftWords = 32;
 constexpr int kProfWords = 12;                         // timestamps per (phase, block)
-constexpr int kTmemCols = 64;                          // two accumulators of up to 32 fp32 columns
+constexpr int kTmemCols = 128;                         // two buffers of two 128-row accumulators of up to 32 fp32 columns
 
 enum OpIndex { OP_QKV = 0, OP_O = 1, OP_GU = 2, OP_DOWN = 3, OP_LM = 4, OP_RAW = 5, OP_COUNT = 6 };
 
@@ -44,7 +45,7 @@ struct OpDesc {
     int P_row;   // partitions along rows
     int P_k;     // partitions along columns (> 1: partial sums meet by reductions in L2)
     int rot;     // block index that owns partition 0 (spreads idle blocks over operations)
-    int RW;      // row tiles per pass at most (8, 4, 2 or 1)
+    int RW;      // row tiles per pass at most (16, 8, 4, 2 or 1)
     int SK;      // column steps per stage at most (RW * SK <= 64)
     int unit;    // row partitions are multiples of this many tiles (2 for gate|up: 16 SwiGLU columns)
     int follow;  // 1: one row partition; block i takes the columns that partition i of `gate|up` produces

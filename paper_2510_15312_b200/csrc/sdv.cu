@@ -104,13 +104,13 @@ Regions carve(const sdv_config* c) {
 // (column partitions, or the residual add), the reductions of all blocks.
 void choose_partition(OpDesc& o, int G, int rows, bool merge, bool always_add) {
     double best_t = -1.0;
-    o.RW = 8;
-    o.SK = kStageBytes / kStepBytes / 8;
+    o.RW = 16;
+    o.SK = kStageBytes / kStepBytes / 16;
     o.P_row = 1;
     o.P_k = 1;
     o.unit = 1;
     o.follow = 0;
-    for (int RW = 8; RW >= 1; RW /= 2) {
+    for (int RW = 16; RW >= 1; RW /= 2) {
         const int SK = kStageBytes / kStepBytes / RW;
         for (int pr = 1; pr <= o.T && pr <= G; ++pr) {
             const int pk_max = G / pr < o.K16 ? G / pr : o.K16;
@@ -137,8 +137,8 @@ void choose_partition(OpDesc& o, int G, int rows, bool merge, bool always_add) {
 }
 // Operations whose epilogue needs complete sums: all columns in one block, rows spread evenly.
 void full_k_partition(OpDesc& o, int G, int unit) {
-    o.RW = 8;
-    o.SK = kStageBytes / kStepBytes / 8;
+    o.RW = 16;
+    o.SK = kStageBytes / kStepBytes / 16;
     o.unit = unit;
     o.follow = 0;
     o.P_k = 1;
@@ -206,7 +206,7 @@ void setup_ops(FwdParams& P, const sdv_config* cfg, int G) {
             case OP_GU: full_k_partition(o, G, 2); break;   // pairs of tiles: 16 SwiGLU columns = one column step of down
             case OP_LM: full_k_partition(o, G, 1); break;
             default:  // down: every block multiplies the SwiGLU columns it produced
-                o.RW = 8; o.SK = kStageBytes / kStepBytes / 8; o.unit = 1; o.follow = 1; o.P_row = 1; o.P_k = P.op[OP_GU].P_row;
+                o.RW = 16; o.SK = kStageBytes / kStepBytes / 16; o.unit = 1; o.follow = 1; o.P_row = 1; o.P_k = P.op[OP_GU].P_row;
                 break;
         }
         if (ops[i].idx == OP_DOWN) {
@@ -905,7 +905,7 @@ int sdv_debug_layout_check(const int* desc, const int* gu_desc, int G) {
         unsigned long long src = pt.off;  // the streamer's running offset
         for (int p = 0; p < pt.npass; ++p) {
             const int pcount = pass_count(pt, p), pstart = pass_start(pt, p);
-            if (pcount < 1 || pcount > 8) return -100;
+            if (pcount < 1 || pcount > 16) return -100;
             for (int st = 0; st < pt.nst; ++st) {
                 const int nks = (pt.SK < pt.nk - st * pt.SK) ? pt.SK : pt.nk - st * pt.SK;
                 const unsigned long long bytes = (unsigned long long)pcount * nks * kStepBytes;

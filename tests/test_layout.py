@@ -30,7 +30,7 @@ def test_partitions_of_every_configuration_cover_each_matrix_once(name):
 def test_random_partitions_and_ragged_shapes():
     rng = np.random.default_rng(0)
     for _ in range(300):
-        RW = int(rng.choice([1, 2, 4, 8]))
+        RW = int(rng.choice([1, 2, 4, 8, 16]))
         SK = int(rng.integers(1, 64 // RW + 1))
         unit = int(rng.choice([1, 2]))
         T = unit * int(rng.integers(1, 40))
@@ -44,8 +44,8 @@ def test_random_partitions_and_ragged_shapes():
     for _ in range(100):
         G = int(rng.integers(1, 20))
         units = int(rng.integers(1, 60))
-        gu = [2 * units, int(rng.integers(1, 20)), min(G, units), 1, 8, 8, 2, 0]
-        down = [int(rng.integers(1, 30)), units, 1, gu[2], 8, int(rng.integers(1, 9)), 1, 1]
+        gu = [2 * units, int(rng.integers(1, 20)), min(G, units), 1, 16, 4, 2, 0]
+        down = [int(rng.integers(1, 30)), units, 1, gu[2], 16, int(rng.integers(1, 5)), 1, 1]
         assert layout_check(gu, gu, G) == OK
         assert layout_check(down, gu, G) == OK, (down, gu)
 
