@@ -62,6 +62,7 @@ struct Misc {
     uint64_t act_ready;   // the SwiGLU operand of this block is complete (one arrival per epilogue warp)
     uint64_t done_bar;    // last tensor-core instruction of the launch has completed
     uint32_t tmem_base;
+    unsigned long long* prof_ptr;  // this block's profile words of the running phase (or null)
     int abort_flag;
     int skip;  // block-uniform copy of abort_flag, refreshed inside every grid barrier
     float sumsq[kMaxRows];  // sums of squares of the residual rows (this block's operand columns)
@@ -392,6 +393,7 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
         dead = __any_sync(0xffffffffu, dead);
         if (dead) continue;
         tc_fence_after();
+        if (misc->prof_ptr && t == 0 && p == npass - 1) misc->prof_ptr[10] = global_timer_ns();
         const int nhalf = pcount > 8 ? 2 : 1;  // a pass of more than 8 tiles fills both 128-row accumulators of the buffer
         for (int half = 0; half < nhalf; ++half) {
             float v[NBT];
@@ -408,6 +410,7 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
                     for (int n = 0; n < 16; ++n) v[(NBT == 32 ? 16 : 0) + n] = hi[n];
                 }
             }
+            if (misc->prof_ptr && t == 0 && p == npass - 1 && half == nhalf - 1) misc->prof_ptr[11] = global_timer_ns();
             if (half == nhalf - 1) {
                 tc_fence_before();
                 __syncwarp();
@@ -514,46 +517,53 @@ __device__ __noinline__ void epilogue_phase(const FwdParams& P, int kind, int la
 
 // ------------------------------------------------------------------------------------------
 // Split-KV attention.  The committed cache [0, L) is cut into S key ranges of kps keys (a multiple
-// of 64, as many ranges as there are blocks to take them, at most kMaxSplits); unit (kv head,
-// s < S) attends all query rows of the head group to range s; unit (kv head, S) covers the M new
-// rows: it finishes their K/V projection (norm scale, bias, rotary), appends them to the cache and
-// attends to them under the causal mask (row j sees new keys 0..j).  Every unit leaves an
-// un-normalised partial result with its running maximum and sum; the output projection merges them
-// while it builds its operand.
+// of 64, as many ranges as there are blocks to take them, at most kMaxSplits); the query heads of a
+// KV head are cut into QG groups small enough that a group's rows (heads x M) fit two 16-row tiles.
+// Unit (kv head, head group, s < S) attends the group's rows to range s; unit (kv head, head group,
+// S) covers the M new rows: it finishes their K/V projection (norm scale, bias, rotary), appends
+// them to the cache (group 0 only) and attends to them under the causal mask (row j sees new keys
+// 0..j).  Every unit leaves an un-normalised partial result with its running maximum and sum; the
+// output projection merges them while it builds its operand.
 //
-// Inside a unit the R = (query heads per KV head) x M rows form MT tiles of 16 rows.  Keys come in
-// blocks of 32, copied asynchronously into a ring of NBUF shared-memory buffers by all worker
-// warps.  Warp (row tile, key group) owns one row tile and every KG-th group of 16 keys: scores
-// (Q K^T on tensor cores), online softmax with quad shuffles in the log2 domain and P V all stay in
-// its registers; with two key groups the two halves meet in shared memory at the end.
+// Keys come in blocks of 64, copied asynchronously into two shared-memory buffers by all worker
+// warps.  Warp (row tile, key group) owns one row tile and every KG-th group of 16 keys of a block
+// (KG = 4 with up to two row tiles): scores (Q K^T on tensor cores), online softmax with quad
+// shuffles in the log2 domain and P V all stay in its registers; the key groups of a row tile meet
+// in shared memory at the end.
+__device__ __forceinline__ int attn_head_groups(const FwdParams& P) {
+    int qg = 1;
+    while (qg < P.g && ((P.g / qg) * P.M > 32 || P.g % qg)) ++qg;
+    return qg;
+}
 __device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps) {
     if (P.L <= 0) { S = 0; kps = 0; return; }
-    int cap = P.G / P.n_kv - 1;
+    int cap = P.G / (P.n_kv * attn_head_groups(P)) - 1;
     if (cap > kMaxSplits) cap = kMaxSplits;
     if (cap < 1) cap = 1;
     kps = ((P.L + cap - 1) / cap + 63) / 64 * 64;
     S = (P.L + kps - 1) / kps;
 }
 
-template <int HD, bool BIG>  // BIG: more than 64 query rows (up to 8 row tiles)
-__device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int hk, int s, int S, int kps, uint8_t* att, int wtid,
-                                            unsigned long long* prof) {
+template <int HD>
+__device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int hk, int qg, int gh, int s, int S, int kps, uint8_t* att,
+                                            int wtid, unsigned long long* prof) {
     constexpr int HD2 = HD / 2;
     constexpr int KSTEPS = HD / 16;
     constexpr int UNITS = HD / 8;    // 16-byte units per K/V row
     constexpr int NT_O = HD / 8;     // 8-column tiles of the output
-    constexpr int KB = 32;           // keys per block
-    constexpr int NBUF = BIG ? 2 : 3;
-    constexpr int QBYTES = (BIG ? 128 : 64) * HD * 2;
+    constexpr int KB = 64;           // keys per block
+    constexpr int NBUF = 2;
+    constexpr int QBYTES = 32 * HD * 2;
     constexpr int KVBYTES = KB * HD * 2;  // one K (or V) block
+    constexpr int KG = 4;            // key groups: 16-key chunks of a block handled side by side
     static_assert(QBYTES + NBUF * 2 * KVBYTES <= kAttnSmemBytes, "attention tiles");
-    static_assert(BIG || 4 * NT_O * 32 * 16 + 4 * 32 * 16 <= NBUF * 2 * KVBYTES, "exchange area of the key-group merge");
+    static_assert((KG - 1) * 2 * (NT_O + 1) * 32 * 16 <= NBUF * 2 * KVBYTES, "exchange area of the key-group merge");
     const int warp = wtid >> 5, lane = wtid & 31;
-    const int M = P.M, L = P.L, R = P.g * M;
+    const int M = P.M, L = P.L, R = gh * M;   // R <= 32
     const int MT = (R + 15) >> 4, RP = MT * 16;
-    const int KG = (MT <= 4) ? 2 : 1;
     const bool active = warp < MT * KG;
     const int mt = active ? warp % MT : 0, kgp = active ? warp / MT : 0;
+    const int head0 = hk * P.g + qg * gh;     // first query head of this unit
     const bool is_new = (s == S);
     uint8_t* Qs = att;
     uint8_t* KVs = att + QBYTES;
@@ -594,7 +604,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
 
     // ---- query tile: normalise, add bias, rotate, round to bf16; 4 rotary pairs per item
     {
-        constexpr int QI = 3;  // items per thread and batch: all loads are issued before the first use
+        constexpr int QI = 2;  // items per thread and batch: all loads are issued before the first use
         const int items = RP * (HD2 / 4);
         for (int base = wtid; base < items; base += QI * kWorkerThreads) {
             float4 qa[QI], qb[QI], c0[QI], c1[QI];
@@ -608,7 +618,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
                 ssq[t] = 0.f;
                 qa[t] = qb[t] = c0[t] = c1[t] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (idx < items && rr[t] < R) {
-                    const int hl = rr[t] / M, j = rr[t] % M, col = (hk * P.g + hl) * HD + ii[t];
+                    const int hl = rr[t] / M, j = rr[t] % M, col = (head0 + hl) * HD + ii[t];
                     ssq[t] = __ldcg(sumsq + j);
                     qa[t] = ld_cg_f4_inorder(P.qkv_acc + (size_t)j * P.n_qkv + col);
                     qb[t] = ld_cg_f4_inorder(P.qkv_acc + (size_t)j * P.n_qkv + col + HD2);
@@ -628,7 +638,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
                     float a[4] = {qa[t].x * rs, qa[t].y * rs, qa[t].z * rs, qa[t].w * rs};
                     float b[4] = {qb[t].x * rs, qb[t].y * rs, qb[t].z * rs, qb[t].w * rs};
                     if (bias) {
-                        const int col = (hk * P.g + r / M) * HD + i;
+                        const int col = (head0 + r / M) * HD + i;
 #pragma unroll
                         for (int e = 0; e < 4; ++e) { a[e] += bias[col + e]; b[e] += bias[col + HD2 + e]; }
                     }
@@ -645,7 +655,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
             }
         }
     }
-    // the new rows' own keys and values fit one block (M <= 32 = KB)
+    // the new rows' own keys and values fit one block (M <= 32 <= KB)
     if (is_new) {
         uint8_t* Ks = KVs;
         uint8_t* Vs = Ks + KVBYTES;
@@ -683,9 +693,11 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
                                  pack_bf16(kvals[4], kvals[5]), pack_bf16(kvals[6], kvals[7]));
                 vv4 = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]),
                                  pack_bf16(v[6], v[7]));
-                const size_t off = (cache_row0 + L + kk) * HD + q16 * 8;
-                *reinterpret_cast<uint4*>(P.kcache + off) = kv4;
-                *reinterpret_cast<uint4*>(P.vcache + off) = vv4;
+                if (qg == 0) {  // every head group computes the rows, one appends them
+                    const size_t off = (cache_row0 + L + kk) * HD + q16 * 8;
+                    *reinterpret_cast<uint4*>(P.kcache + off) = kv4;
+                    *reinterpret_cast<uint4*>(P.vcache + off) = vv4;
+                }
             }
             const uint32_t so = (q16 >> 3) * (KB * 128) + swz_unit(key, q16 & 7);
             *reinterpret_cast<uint4*>(Ks + so) = kv4;
@@ -779,37 +791,41 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
     if (!is_new) cp_async_wait<0>();
     if (prof && wtid == 0) prof[5] = global_timer_ns();
 
-    // ---- row sums over the quad; the two key groups of a row tile meet in shared memory
+    // ---- row sums over the quad; the key groups of a row tile meet in shared memory
     l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
     l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-    if (KG == 2) {
-        float4* ex_o = reinterpret_cast<float4*>(KVs);                      // [row tile][output tile][lane]
-        float4* ex_ml = ex_o + 4 * NT_O * 32;                               // [row tile][lane]
-        if (active && kgp == 1) {
+    {
+        float4* ex_o = reinterpret_cast<float4*>(KVs);          // [key group - 1][row tile][output tile][lane]
+        float4* ex_ml = ex_o + (KG - 1) * 2 * NT_O * 32;        // [key group - 1][row tile][lane]
+        if (active && kgp > 0) {
+            float4* dst = ex_o + ((kgp - 1) * 2 + mt) * NT_O * 32;
 #pragma unroll
-            for (int n = 0; n < NT_O; ++n) ex_o[(mt * NT_O + n) * 32 + lane] = make_float4(o[n][0], o[n][1], o[n][2], o[n][3]);
-            ex_ml[mt * 32 + lane] = make_float4(m_lo, m_hi, l_lo, l_hi);
+            for (int n = 0; n < NT_O; ++n) dst[n * 32 + lane] = make_float4(o[n][0], o[n][1], o[n][2], o[n][3]);
+            ex_ml[((kgp - 1) * 2 + mt) * 32 + lane] = make_float4(m_lo, m_hi, l_lo, l_hi);
         }
         named_bar_sync(1, kWorkerThreads);
         if (active && kgp == 0) {
-            const float4 ml = ex_ml[mt * 32 + lane];
-            const float mn_lo = fmaxf(m_lo, ml.x), mn_hi = fmaxf(m_hi, ml.y);
-            const float use_lo = (mn_lo == -CUDART_INF_F) ? 0.f : mn_lo, use_hi = (mn_hi == -CUDART_INF_F) ? 0.f : mn_hi;
-            const float e0_lo = exp2f(m_lo - use_lo), e1_lo = exp2f(ml.x - use_lo);
-            const float e0_hi = exp2f(m_hi - use_hi), e1_hi = exp2f(ml.y - use_hi);
-            m_lo = mn_lo;
-            m_hi = mn_hi;
-            l_lo = l_lo * e0_lo + ml.z * e1_lo;
-            l_hi = l_hi * e0_hi + ml.w * e1_hi;
+            for (int og = 0; og < KG - 1; ++og) {
+                const float4 ml = ex_ml[(og * 2 + mt) * 32 + lane];
+                const float mn_lo = fmaxf(m_lo, ml.x), mn_hi = fmaxf(m_hi, ml.y);
+                const float use_lo = (mn_lo == -CUDART_INF_F) ? 0.f : mn_lo, use_hi = (mn_hi == -CUDART_INF_F) ? 0.f : mn_hi;
+                const float e0_lo = exp2f(m_lo - use_lo), e1_lo = exp2f(ml.x - use_lo);
+                const float e0_hi = exp2f(m_hi - use_hi), e1_hi = exp2f(ml.y - use_hi);
+                m_lo = mn_lo;
+                m_hi = mn_hi;
+                l_lo = l_lo * e0_lo + ml.z * e1_lo;
+                l_hi = l_hi * e0_hi + ml.w * e1_hi;
+                const float4* src = ex_o + (og * 2 + mt) * NT_O * 32;
 #pragma unroll
-            for (int n = 0; n < NT_O; ++n) {
-                const float4 t = ex_o[(mt * NT_O + n) * 32 + lane];
-                o[n][0] = o[n][0] * e0_lo + t.x * e1_lo;
-                o[n][1] = o[n][1] * e0_lo + t.y * e1_lo;
-                o[n][2] = o[n][2] * e0_hi + t.z * e1_hi;
-                o[n][3] = o[n][3] * e0_hi + t.w * e1_hi;
+                for (int n = 0; n < NT_O; ++n) {
+                    const float4 t = src[n * 32 + lane];
+                    o[n][0] = o[n][0] * e0_lo + t.x * e1_lo;
+                    o[n][1] = o[n][1] * e0_lo + t.y * e1_lo;
+                    o[n][2] = o[n][2] * e0_hi + t.z * e1_hi;
+                    o[n][3] = o[n][3] * e0_hi + t.w * e1_hi;
+                }
             }
         }
     }
@@ -820,7 +836,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
         for (int half = 0; half < 2; ++half) {
             const int r = half ? r_hi : r_lo;
             if (r >= R) continue;
-            const int hq = hk * P.g + r / M, j = r % M;
+            const int hq = head0 + r / M, j = r % M;
             const size_t row = ((size_t)hq * (kMaxSplits + 1) + s) * kMaxRows + j;
             float* po = P.part_o + row * HD + q2;
 #pragma unroll
@@ -836,17 +852,12 @@ __device__ void attention_phase(const FwdParams& P, int layer, uint8_t* att, int
     int S, kps;
     attn_split(P, S, kps);
     const int S1 = S + 1;
-    const int nunits = P.n_kv * S1;
+    const int QG = attn_head_groups(P), gh = P.g / QG;
+    const int nunits = P.n_kv * QG * S1;
     for (int unit = blockIdx.x; unit < nunits; unit += P.G) {
-        const int hk = unit / S1, s = unit % S1;
-        const bool big = P.g * P.M > 64;
-        if (P.hd == 128) {
-            if (big) attention_unit<128, true>(P, layer, hk, s, S, kps, att, wtid, prof);
-            else attention_unit<128, false>(P, layer, hk, s, S, kps, att, wtid, prof);
-        } else {
-            if (big) attention_unit<64, true>(P, layer, hk, s, S, kps, att, wtid, prof);
-            else attention_unit<64, false>(P, layer, hk, s, S, kps, att, wtid, prof);
-        }
+        const int hk = unit / (QG * S1), rem = unit % (QG * S1), qg = rem / S1, s = rem % S1;
+        if (P.hd == 128) attention_unit<128>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof);
+        else attention_unit<64>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof);
         named_bar_sync(1, kWorkerThreads);  // the unit's shared-memory tiles are free again
         if (prof && wtid == 0) { prof[6] = global_timer_ns(); prof[7] = (unsigned long long)(s == S); }
     }
@@ -904,6 +915,7 @@ __device__ __noinline__ void gemm_phase(const FwdParams& P, int kind, int layer,
     const Part& p0 = misc->part[ops[0]];
     const bool have0 = p0.ntiles > 0 && p0.nk > 0;
     bool dead = *(volatile int*)&misc->abort_flag != 0;
+    if (wtid == 0) misc->prof_ptr = prof;
 
     if (warp == kMmaWarp) {
         // the tensor-core warp builds nothing: it prepares its descriptors and meets the others at the

@@ -30,7 +30,7 @@ constexpr int kMaxStages = 8;                          // ring slots at most
 constexpr int kMaxRows = 32;                           // token rows a buffer is sized for
 constexpr int kMaxSplits = 19;                         // KV key ranges per head (+1 partial result for the new rows)
 constexpr int kSmemBudget = 232448;                    // 227 KB
-constexpr int kAttnSmemBytes = 65536;                  // Q tile (16 or 32 KB) + ring of K|V blocks (48 or 32 KB)
+constexpr int kAttnSmemBytes = 73728;                  // Q tile (8 KB) + two K|V blocks of 64 keys (64 KB)
 constexpr int kActSmemMax = 32768;                     // SwiGLU output of this block (operand of its down-projection slice) at most
 constexpr int kMiscSmemBytes = 4096;
 constexpr int kMaxDraftWords = 32;

@@ -38,7 +38,6 @@ bool config_ok(const sdv_config* c) {
     const int g = c->n_q_heads / c->n_kv_heads;
     if (g > 8) return false;
     if (c->k_max < 1 || c->k_max > SDV_K_MAX) return false;
-    if (g * (c->k_max + 1) > 128) return false;  // query tile of the attention step
     if (c->max_seq < c->k_max + 2) return false;
     if (c->ngram_n < 1 || c->ngram_n > 8 || c->ngram_min < 1 || c->ngram_min > c->ngram_n) return false;
     if (!(c->rope_theta > 0.f) || !(c->rms_eps > 0.f)) return false;
@@ -598,12 +597,8 @@ int sdv_prefill_chunk(sdv_ctx* ctx, const int32_t* host_tokens, int n, int is_la
         if (host_tokens[i] < 0 || host_tokens[i] >= c.vocab) return SDV_EINVAL;
     int* hist = (int*)(ctx->ws + ctx->r.hist);
     CK(cudaMemcpyAsync(hist + ctx->hist_len, host_tokens, (size_t)n * 4, cudaMemcpyDefault, ctx->stream));
-    // rows per launch: the attention step's query tile holds (q heads per kv head) x rows <= 128
-    const int g = c.n_q_heads / c.n_kv_heads;
-    int tile = 128 / g;
-    if (tile > 24) tile = 24;
-    tile = tile / 8 * 8;
-    if (tile < 8) tile = 8;
+    // rows per launch
+    int tile = 24;
     {
         // wide models: fewer rows per launch so that the token operand leaves room for the weight ring
         FwdParams probe = ctx->P;
