@@ -35,8 +35,10 @@ def test_host_side_argument_checks():
         c = SdvConfig.from_buffer_copy(good)
         setattr(c, field, bad)
         assert L.sdv_workspace_bytes(ctypes.byref(c)) == 0, field
-    # 8 query heads per KV head with 17 rows would overflow the attention query tile
+    # 8 query heads per KV head with 17 rows: the attention step cuts the heads into groups, so this fits
     c = SdvConfig(2, 512, 8, 1, 64, 1024, 4096, 600, 16, 0, 0, 3, 1, 0, 1e4, 1e-6)
+    assert L.sdv_workspace_bytes(ctypes.byref(c)) > 0
+    c.n_q_heads = 16  # more than 8 query heads per KV head is not supported
     assert L.sdv_workspace_bytes(ctypes.byref(c)) == 0
     assert L.sdv_strerror(pkg.ETIMEOUT).decode().startswith("a bounded")
     assert L.sdv_strerror(-99) == b"unknown error"
