@@ -158,6 +158,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--k", type=int, default=0)
+    ap.add_argument("--sweep-k", default="", help="comma-separated draft lengths: adds verify-step us and GB/s per k "
+                                                 "at the fixed KV length reached after prefill (rolled back after each step)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -182,17 +184,32 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     k = cfg.k
+    sweep = [int(x) for x in args.sweep_k.split(",") if x.strip()]
+    k_max = max([k] + sweep)
     total = args.warmup + args.steps
     max_seq = cfg.n_ctx + 2 * total * (k + 1) + 64          # room for two timed loops at full acceptance
     cores = len(os.sched_getaffinity(0))
     w = make_weights(cfg, threads=max(8, cores // max(1, world)))
     ctx = make_context(cfg)
     stream = torch.cuda.Stream()
-    s = Sdv(config_from(cfg, max_seq=max_seq), stream=stream)
+    s = Sdv(config_from(cfg, k_max=k_max, max_seq=max_seq), stream=stream)
     s.load_weights(w)
     for i in range(0, cfg.n_ctx, cfg.chunk):
         s.prefill_chunk(ctx[i:i + cfg.chunk], is_last=(i + cfg.chunk >= cfg.n_ctx))
     L0 = s.kv_len()
+
+    def sweep_point(kk, n):
+        """n verify steps of kk+1 rows at KV length L0 (nothing committed): mean forward-kernel ms."""
+        draft = [int(t) for t in ctx[:kk]]
+        ms = []
+        for i in range(n + 3):
+            s.verify(draft, fetch=False)
+            s.rollback(L0)
+            if i >= 3:
+                ms.append(s.last_verify_ms())
+        return statistics.mean(ms)
+
+    sweep_ms = {kk: sweep_point(kk, max(10, args.steps // 4)) for kk in sweep}
 
     def barrier():
         if world > 1:
@@ -279,6 +296,13 @@ def main():
             "gpu_launches": launches,
             "clocks": clocks,
         }
+        if sweep:
+            line["k_sweep"] = []
+            for kk in sweep:
+                wb, kb = s.step_bytes(kk + 1, L0)
+                gbs = (wb + kb) / (sweep_ms[kk] * 1e-3) / 1e9
+                line["k_sweep"].append({"k": kk, "kv_len": L0, "verify_kernel_us": sweep_ms[kk] * 1e3, "GB/s": gbs,
+                                        "frac": gbs / peak})
         if world == 1 and not args.no_cpu_baseline:
             n_prefill = min(cfg.chunk, cfg.n_ctx)
             n_steps = 48 if cfg.linear_params() < 1.0e9 else (24 if cfg.linear_params() < 4.0e9 else 8)

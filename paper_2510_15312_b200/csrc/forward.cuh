@@ -517,8 +517,9 @@ __device__ __noinline__ void epilogue_phase(const FwdParams& P, int kind, int la
 
 // ------------------------------------------------------------------------------------------
 // Split-KV attention.  The committed cache [0, L) is cut into S key ranges of kps keys (a multiple
-// of 64, as many ranges as there are blocks to take them, at most kMaxSplits); the query heads of a
-// KV head are cut into QG groups small enough that a group's rows (heads x M) fit two 16-row tiles.
+// of 64, at most kMaxSplits ranges); the query heads of a KV head are cut into QG groups of up to
+// gh heads, a group's rows (heads x M) filling at most four 16-row tiles (the host picks gh so
+// that the longest chain of 16-key steps a warp walks is shortest).
 // Unit (kv head, head group, s < S) attends the group's rows to range s; unit (kv head, head group,
 // S) covers the M new rows: it finishes their K/V projection (norm scale, bias, rotary), appends
 // them to the cache (group 0 only) and attends to them under the causal mask (row j sees new keys
@@ -527,17 +528,15 @@ __device__ __noinline__ void epilogue_phase(const FwdParams& P, int kind, int la
 //
 // Keys come in blocks of 64, copied asynchronously into two shared-memory buffers by all worker
 // warps.  Warp (row tile, key group) owns one row tile and every KG-th group of 16 keys of a block
-// (KG = 4 with up to two row tiles): scores (Q K^T on tensor cores), online softmax with quad
+// (KG = 4 with up to two row tiles, 3 with three, 2 with four): scores (Q K^T on tensor cores), online softmax with quad
 // shuffles in the log2 domain and P V all stay in its registers; the key groups of a row tile meet
 // in shared memory at the end.
-__device__ __forceinline__ int attn_head_groups(const FwdParams& P) {
-    int qg = 1;
-    while (qg < P.g && ((P.g / qg) * P.M > 32 || P.g % qg)) ++qg;
-    return qg;
-}
+// The heads per group are chosen on the host per launch; the key ranges follow from it: as many
+// as there are blocks to take a (KV head, head group, range) unit each, at most kMaxSplits.
 __device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps) {
     if (P.L <= 0) { S = 0; kps = 0; return; }
-    int cap = P.G / (P.n_kv * attn_head_groups(P)) - 1;
+    const int QG = (P.g + P.att_gh - 1) / P.att_gh;
+    int cap = P.G / (P.n_kv * QG) - 1;
     if (cap > kMaxSplits) cap = kMaxSplits;
     if (cap < 1) cap = 1;
     kps = ((P.L + cap - 1) / cap + 63) / 64 * 64;
@@ -553,14 +552,17 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
     constexpr int NT_O = HD / 8;     // 8-column tiles of the output
     constexpr int KB = 64;           // keys per block
     constexpr int NBUF = 2;
-    constexpr int QBYTES = 32 * HD * 2;
+    constexpr int QBYTES = 64 * HD * 2;
     constexpr int KVBYTES = KB * HD * 2;  // one K (or V) block
-    constexpr int KG = 4;            // key groups: 16-key chunks of a block handled side by side
     static_assert(QBYTES + NBUF * 2 * KVBYTES <= kAttnSmemBytes, "attention tiles");
-    static_assert((KG - 1) * 2 * (NT_O + 1) * 32 * 16 <= NBUF * 2 * KVBYTES, "exchange area of the key-group merge");
+    // exchange area of the key-group merge: (KG - 1) * MT <= 6 tiles of (output + statistics)
+    static_assert(6 * (NT_O + 1) * 32 * 16 <= NBUF * 2 * KVBYTES, "exchange area of the key-group merge");
     const int warp = wtid >> 5, lane = wtid & 31;
-    const int M = P.M, L = P.L, R = gh * M;   // R <= 32
+    const int M = P.M, L = P.L;
+    const int nheads = min(gh, P.g - qg * gh);   // the last group may hold fewer heads
+    const int R = nheads * M;                    // R <= 64
     const int MT = (R + 15) >> 4, RP = MT * 16;
+    const int KG = MT <= 2 ? 4 : (MT == 3 ? 3 : 2);  // key groups: 16-key chunks of a block handled side by side
     const bool active = warp < MT * KG;
     const int mt = active ? warp % MT : 0, kgp = active ? warp / MT : 0;
     const int head0 = hk * P.g + qg * gh;     // first query head of this unit
@@ -798,17 +800,17 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
     {
         float4* ex_o = reinterpret_cast<float4*>(KVs);          // [key group - 1][row tile][output tile][lane]
-        float4* ex_ml = ex_o + (KG - 1) * 2 * NT_O * 32;        // [key group - 1][row tile][lane]
+        float4* ex_ml = ex_o + 6 * NT_O * 32;                   // [key group - 1][row tile][lane]
         if (active && kgp > 0) {
-            float4* dst = ex_o + ((kgp - 1) * 2 + mt) * NT_O * 32;
+            float4* dst = ex_o + ((kgp - 1) * MT + mt) * NT_O * 32;
 #pragma unroll
             for (int n = 0; n < NT_O; ++n) dst[n * 32 + lane] = make_float4(o[n][0], o[n][1], o[n][2], o[n][3]);
-            ex_ml[((kgp - 1) * 2 + mt) * 32 + lane] = make_float4(m_lo, m_hi, l_lo, l_hi);
+            ex_ml[((kgp - 1) * MT + mt) * 32 + lane] = make_float4(m_lo, m_hi, l_lo, l_hi);
         }
         named_bar_sync(1, kWorkerThreads);
         if (active && kgp == 0) {
             for (int og = 0; og < KG - 1; ++og) {
-                const float4 ml = ex_ml[(og * 2 + mt) * 32 + lane];
+                const float4 ml = ex_ml[(og * MT + mt) * 32 + lane];
                 const float mn_lo = fmaxf(m_lo, ml.x), mn_hi = fmaxf(m_hi, ml.y);
                 const float use_lo = (mn_lo == -CUDART_INF_F) ? 0.f : mn_lo, use_hi = (mn_hi == -CUDART_INF_F) ? 0.f : mn_hi;
                 const float e0_lo = exp2f(m_lo - use_lo), e1_lo = exp2f(ml.x - use_lo);
@@ -817,7 +819,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
                 m_hi = mn_hi;
                 l_lo = l_lo * e0_lo + ml.z * e1_lo;
                 l_hi = l_hi * e0_hi + ml.w * e1_hi;
-                const float4* src = ex_o + (og * 2 + mt) * NT_O * 32;
+                const float4* src = ex_o + (og * MT + mt) * NT_O * 32;
 #pragma unroll
                 for (int n = 0; n < NT_O; ++n) {
                     const float4 t = src[n * 32 + lane];
@@ -852,7 +854,7 @@ __device__ void attention_phase(const FwdParams& P, int layer, uint8_t* att, int
     int S, kps;
     attn_split(P, S, kps);
     const int S1 = S + 1;
-    const int QG = attn_head_groups(P), gh = P.g / QG;
+    const int gh = P.att_gh, QG = (P.g + gh - 1) / gh;
     const int nunits = P.n_kv * QG * S1;
     for (int unit = blockIdx.x; unit < nunits; unit += P.G) {
         const int hk = unit / (QG * S1), rem = unit % (QG * S1), qg = rem / S1, s = rem % S1;

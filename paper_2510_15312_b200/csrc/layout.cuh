@@ -30,7 +30,7 @@ constexpr int kMaxStages = 8;                          // ring slots at most
 constexpr int kMaxRows = 32;                           // token rows a buffer is sized for
 constexpr int kMaxSplits = 19;                         // KV key ranges per head (+1 partial result for the new rows)
 constexpr int kSmemBudget = 232448;                    // 227 KB
-constexpr int kAttnSmemBytes = 73728;                  // Q tile (8 KB) + two K|V blocks of 64 keys (64 KB)
+constexpr int kAttnSmemBytes = 81920;                  // Q tile (up to 16 KB) + two K|V blocks of 64 keys (64 KB)
 constexpr int kActSmemMax = 32768;                     // SwiGLU output of this block (operand of its down-projection slice) at most
 constexpr int kMiscSmemBytes = 4096;
 constexpr int kMaxDraftWords = 32;
@@ -196,6 +196,7 @@ struct FwdParams {
     int L;             // committed KV length = position of row 0
     int M;             // rows computed (1..kMaxRows)
     int NB;            // N of the tensor-core instruction: 16, or 32 when M > 16
+    int att_gh;        // attention split: query heads per unit (the key ranges follow from it)
     int mode;          // 0: rows are [pending, draft...]; 1: rows are hist[L..L+M)
     int ph_begin, ph_end;
     int bar_base;      // barrier counter value before this launch

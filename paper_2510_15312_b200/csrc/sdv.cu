@@ -280,6 +280,32 @@ bool apply_plan(FwdParams& P, int rows, bool raw_only, int* smem_bytes) {
     return true;
 }
 
+// Attention split of a launch: heads per unit (a unit's rows, heads x M, fill at most four 16-row
+// tiles), number of key ranges and keys per range (a multiple of 64).  Cost of a choice = the
+// 16-key steps a warp walks one after another: blocks of 64 keys per range x steps per block.
+void plan_attention(FwdParams& P, int rows, int L) {
+    P.att_gh = 1;
+    if (P.g < 1) return;
+    int best = -1;
+    for (int gh = 1; gh <= P.g; ++gh) {
+        if (gh * rows > 64 && gh > 1) break;
+        const int MT = (gh * rows + 15) / 16, KG = MT <= 2 ? 4 : (MT == 3 ? 3 : 2);
+        const int QG = (P.g + gh - 1) / gh;
+        int cap = P.G / (P.n_kv * QG) - 1;
+        if (cap > kMaxSplits) cap = kMaxSplits;
+        if (cap < 1) cap = 1;
+        int cost = 1;
+        if (L > 0) {
+            const int kps = ((L + cap - 1) / cap + 63) / 64 * 64;
+            cost = (kps / 64) * ((4 + KG - 1) / KG);
+        }
+        if (best < 0 || cost <= best) {  // ties: more heads per unit (fewer reloads of the keys)
+            best = cost;
+            P.att_gh = gh;
+        }
+    }
+}
+
 // Runs phases [ph_begin, ph_end) over `rows` token rows at position L.
 int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph_end, bool timed) {
     FwdParams P = ctx->P;
@@ -287,6 +313,7 @@ int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph
     const bool raw_only = (ph_begin == 2 + kPhasesPerLayer * ctx->cfg.n_layers);
     if (!apply_plan(P, rows, raw_only, &smem_bytes)) return SDV_EINVAL;
     P.L = L;
+    plan_attention(P, rows, L);
     P.mode = mode;
     P.ph_begin = ph_begin;
     P.ph_end = ph_end;
