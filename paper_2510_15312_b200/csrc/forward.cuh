@@ -81,12 +81,14 @@ __device__ __forceinline__ bool grid_barrier(const FwdParams& P, int target, Mis
     named_bar_sync(1, kWorkerThreads);
     if (wtid == 0) {
         red_release_add_s32(P.bar, 1);  // no return value to wait for: polling starts at once
-        const uint64_t t0 = global_timer_ns();
+        uint64_t t0 = 0;  // the global timer is slow to read: only once the wait has lasted a while
         uint32_t spins = 0;
         while ((int)(ld_acquire_gpu(P.bar) - target) < 0) {
             if ((++spins & 63u) == 0) {
                 if (*(volatile int*)&misc->abort_flag) break;
-                if (global_timer_ns() - t0 > P.wait_limit_ns) {
+                const uint64_t now = global_timer_ns();
+                if (t0 == 0) t0 = now;
+                if (now - t0 > P.wait_limit_ns) {
                     *(volatile int*)&misc->abort_flag = 1;
                     break;
                 }
@@ -370,9 +372,10 @@ template <int NBT>  // token columns read: 16 or 32
 __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op, int layer, const Part& pt, uint8_t* act, Misc* misc,
                                             PipePos& pos, bool& dead, int warp, int lane, float (&bv)[NBT], int (&bi)[NBT]) {
     const int M = P.M;
-    const int t = warp * 32 + lane;
+    const int quarter = warp & 3, myhalf = warp >> 2;  // this warp's 32 accumulator lanes; which of the two accumulators
+    const int t = quarter * 32 + lane;
     const uint64_t wait_limit = P.wait_limit_ns;
-    const uint32_t tmem_lane = misc->tmem_base + ((uint32_t)(warp * 32) << 16);
+    const uint32_t tmem_lane = misc->tmem_base + ((uint32_t)(quarter * 32) << 16);
     const int npass = pt.npass, tile0 = pt.tile0;
     float rstd[NBT];
     if (op == OP_GU || op == OP_LM) {
@@ -395,7 +398,11 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
         tc_fence_after();
         if (misc->prof_ptr && t == 0 && p == npass - 1) misc->prof_ptr[10] = global_timer_ns();
         const int nhalf = pcount > 8 ? 2 : 1;  // a pass of more than 8 tiles fills both 128-row accumulators of the buffer
-        for (int half = 0; half < nhalf; ++half) {
+        // two accumulators: warps 0..3 read the first, 4..7 the second; one accumulator: both groups read
+        // it and share its token columns (pairs of columns alternate between the groups)
+        const int nsel = (nhalf == 2) ? -1 : myhalf;
+        {
+            const int half = (nhalf == 2) ? myhalf : 0;
             float v[NBT];
             {
                 const uint32_t taddr = tmem_lane + buf * 64u + (uint32_t)half * 32u;
@@ -410,12 +417,9 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
                     for (int n = 0; n < 16; ++n) v[(NBT == 32 ? 16 : 0) + n] = hi[n];
                 }
             }
-            if (misc->prof_ptr && t == 0 && p == npass - 1 && half == nhalf - 1) misc->prof_ptr[11] = global_timer_ns();
-            if (half == nhalf - 1) {
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&misc->tmem_empty[buf]);  // the accumulators may be overwritten
-            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&misc->tmem_empty[buf]);  // this warp's part of the accumulators may be overwritten
             const int tt = half * 128 + t;         // row within the pass
             const bool valid = tt < 16 * pcount;
             const int row = (tile0 + pstart) * 16 + tt;  // weight row = output feature
@@ -428,7 +432,7 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
 #pragma unroll
                 for (int n = 0; n < NBT; ++n) {
                     const float other = __shfl_xor_sync(0xffffffffu, v[n], 8);
-                    if (valid && n < M && ((n & 1) != 0) == is_up) {
+                    if (valid && n < M && ((n & 1) != 0) == is_up && (nsel < 0 || ((n >> 1) & 1) == nsel)) {
                         const float x = (is_up ? other : v[n]) * rstd[n], y = (is_up ? v[n] : other) * rstd[n];
                         const float a = __fdividef(x, 1.f + __expf(-x)) * y;
                         *reinterpret_cast<__nv_bfloat16*>(dst + n * 16) = __float2bfloat16(a);
@@ -437,7 +441,7 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
             } else if (op == OP_LM) {
 #pragma unroll
                 for (int n = 0; n < NBT; ++n) {
-                    if (valid && n < M) {
+                    if (valid && n < M && (nsel < 0 || ((n >> 1) & 1) == nsel)) {
                         const float x = v[n] * rstd[n];
                         if (store_logits) __stcg(P.logits + (size_t)n * P.V + row, x);
                         // rows come in ascending order per thread, so ">" keeps the lowest id among equals
@@ -447,7 +451,7 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
             } else if (valid) {
 #pragma unroll
                 for (int n = 0; n < NBT; ++n) {
-                    if (n < M) {
+                    if (n < M && (nsel < 0 || ((n >> 1) & 1) == nsel)) {
                         float* d2 = out + (size_t)n * stride + row;
                         if (add) red_add_f32(d2, v[n]);
                         else __stcg(d2, v[n]);
@@ -952,13 +956,13 @@ __device__ __noinline__ void gemm_phase(const FwdParams& P, int kind, int layer,
             else build_norm_operand(P, kind, layer, p0, U, misc, wtid);
             fence_proxy_async_smem();
         }
-        if (kind == PH_O && warp >= kEpilogueWarps) {
+        if (kind == PH_O && warp >= 4) {
             // clear the accumulators the next QKV projection adds into (idle warps)
-            const int n4 = kMaxRows * P.n_qkv / 4, nth = (kBuilderWarps - kEpilogueWarps) * 32;
-            for (int i = blockIdx.x * nth + (wtid - kEpilogueWarps * 32); i < n4; i += P.G * nth)
+            const int n4 = kMaxRows * P.n_qkv / 4, nth = (kBuilderWarps - 4) * 32;
+            for (int i = blockIdx.x * nth + (wtid - 4 * 32); i < n4; i += P.G * nth)
                 __stcg(reinterpret_cast<float4*>(P.qkv_acc) + i, make_float4(0.f, 0.f, 0.f, 0.f));
-            if (blockIdx.x == 0 && wtid < kEpilogueWarps * 32 + kMaxRows)
-                __stcg(P.sumsq + ((layer + 1) & 1) * kMaxRows + (wtid - kEpilogueWarps * 32), 0.f);
+            if (blockIdx.x == 0 && wtid < 4 * 32 + kMaxRows)
+                __stcg(P.sumsq + ((layer + 1) & 1) * kMaxRows + (wtid - 4 * 32), 0.f);
         }
         named_bar_sync(1, kWorkerThreads);  // the operand is complete and visible to the tensor core
         if (prof && wtid == 0) prof[2] = global_timer_ns();
@@ -1050,13 +1054,7 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
     // all tensor-core work must have completed before tensor memory is returned
     if (warp == kMmaWarp && lane == 0) {
         umma_commit(&misc->done_bar);
-        const uint64_t t0 = global_timer_ns();
-        while (!mbar_try_wait(&misc->done_bar, 0)) {
-            if (global_timer_ns() - t0 > P.wait_limit_ns) {
-                *(volatile int*)&misc->abort_flag = 1;
-                break;
-            }
-        }
+        mbar_wait_bounded(&misc->done_bar, 0, &misc->abort_flag, P.wait_limit_ns);
     }
     tc_fence_before();
     named_bar_sync(1, kWorkerThreads);

@@ -21,7 +21,7 @@ constexpr int kWorkerWarps = 11;                       // every warp but the wei
 constexpr int kWorkerThreads = kWorkerWarps * 32;      // 352
 constexpr int kThreads = kWorkerThreads + 32;          // 384 with the weight-streaming warp
 constexpr int kBuilderWarps = 10;                      // warps 0..9 build the token operand of a GEMM
-constexpr int kEpilogueWarps = 4;                      // warps 0..3 read the accumulator (tensor-memory lanes 32w..32w+31)
+constexpr int kEpilogueWarps = 8;                      // warps 0..7 read the accumulators: warp w lanes 32(w%4)..+31 of accumulator w/4
 constexpr int kMmaWarp = 10;                           // its lane 0 issues the tensor-core instructions
 constexpr int kProducerWarp = 11;
 constexpr int kStepBytes = 512;                        // one row tile x one column step: 16 x 16 bf16
