@@ -188,13 +188,17 @@ int sdv_debug_gemm(sdv_ctx *ctx, const float *host_x, const uint16_t *host_w, fl
  * context stays usable), SDV_OK if the wait wrongly succeeded. */
 int sdv_debug_timeout_probe(sdv_ctx *ctx);
 
-/* Per-phase timing of the forward kernel.  host_out != NULL: copies the timestamps recorded by the
- * last profiled launch, uint64 nanoseconds [n_phases][blocks][12] per thread block: phase work
- * begin, end, token operand built, last tensor-core instruction issued, epilogue done (GEMM
- * phases; the attention phase uses words 2..7 for its own steps; the rest spare) (phase 0 =
- * embedding, then 4 per layer: qkv, attention, o, gate|up + down; last = LM head).  Then switches
- * recording on or off for later launches (it adds a block-wide barrier per phase, so timed runs
- * keep it off).  Returns the number of thread blocks, or an error. */
+/* Per-phase timing of the forward kernel.  host_out != NULL: copies what the last profiled launch
+ * recorded, uint64 [n_phases][blocks][12] per thread block (phase 0 = embedding, then 4 per layer:
+ * qkv, attention, o, gate|up + down; last = LM head).  Words 0, 1: phase work begin and end
+ * (nanoseconds of the global timer).  GEMM phases: 2 token operand built, 3 last tensor-core
+ * instruction issued, 4 epilogue done, 5 / 6 wait for the SwiGLU operand begins / ends (gate|up +
+ * down only), 10 last accumulator seen complete by the epilogue (nanoseconds); 7, 8, 9 cycles the
+ * tensor-core warp waited for weights, waited for a free accumulator, and spent in its loop.
+ * Attention phase: 2 unit begins, 3 query tile built, 4 first key block in place, 5 key loop done,
+ * 6 unit done, 7 whether the unit was a new-rows unit.  Then switches recording on or off for
+ * later launches (it adds a block-wide barrier per phase, so timed runs keep it off).  Returns the
+ * number of thread blocks, or an error. */
 int sdv_debug_profile(sdv_ctx *ctx, int on, unsigned long long *host_out, int n_phases);
 
 /* Host-only self-check of the weight streaming layout (no GPU needed): walks every thread block's
