@@ -125,6 +125,19 @@ def oracle_steps_per_sec(cfg, weights, ctx, n_prefill, n_steps, k):
     return emitted_total / dt, dt / n_steps, emitted_total
 
 
+def aggregate_over_ranks(times_ms, counts, world, device):
+    """Replicas only: the job's time is the slowest rank's (MAX), its work the sum over ranks (SUM).
+    Needs an initialised process group when world > 1 (any backend); returns two lists of floats."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    c = torch.tensor(list(counts), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return t.tolist(), c.tolist()
+
+
 def run_reference(args, cfg):
     from sdv_inputs import make_context, make_weights
     rank = int(os.environ.get("RANK", "0"))
@@ -258,13 +271,8 @@ def main():
     barrier()
     ms_e2e = e0.elapsed_time(e1)
 
-    stats = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
-    counts = torch.tensor([tokens, tokens_e], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
-        dist.all_reduce(counts, op=dist.ReduceOp.SUM)
-    ms_total, ms_e2e = stats.tolist()
-    tokens_all, tokens_e_all = counts.tolist()
+    (ms_total, ms_e2e), (tokens_all, tokens_e_all) = aggregate_over_ranks([ms_total, ms_e2e], [tokens, tokens_e], world,
+                                                                          "cuda")
 
     if rank == 0:
         peak, peak_kind = load_peaks()
