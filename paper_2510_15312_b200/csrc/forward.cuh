@@ -449,13 +449,15 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
                     }
                 }
             } else if (valid) {
+                float* d2 = out + row;
+                if (add) {
 #pragma unroll
-                for (int n = 0; n < NBT; ++n) {
-                    if (n < M && (nsel < 0 || ((n >> 1) & 1) == nsel)) {
-                        float* d2 = out + (size_t)n * stride + row;
-                        if (add) red_add_f32(d2, v[n]);
-                        else __stcg(d2, v[n]);
-                    }
+                    for (int n = 0; n < NBT; ++n, d2 += stride)
+                        if (n < M && (nsel < 0 || ((n >> 1) & 1) == nsel)) red_add_f32(d2, v[n]);
+                } else {
+#pragma unroll
+                    for (int n = 0; n < NBT; ++n, d2 += stride)
+                        if (n < M && (nsel < 0 || ((n >> 1) & 1) == nsel)) __stcg(d2, v[n]);
                 }
             }
         }
