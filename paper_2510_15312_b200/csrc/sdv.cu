@@ -963,6 +963,7 @@ int sdv_debug_plan(const sdv_config* cfg, int G, int rows, int* out) {
     if (!config_ok(cfg) || !out || G < 1 || G > kMaxGrid || rows < 1 || rows > kMaxRows) return SDV_EINVAL;
     FwdParams P;
     memset(&P, 0, sizeof(P));
+    P.d = cfg->d_model;
     setup_ops(P, cfg, G);
     for (int i = 0; i < 5; ++i) {
         const OpDesc& o = P.op[i];
