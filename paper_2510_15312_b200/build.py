@@ -9,13 +9,26 @@ LIB_PATH = os.path.join(_HERE, "libsdv.so")
 _SOURCES = ["sdv.cu", "forward.cuh", "layout.cuh", "ptx.cuh", "small_kernels.cuh"]
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB_PATH):
-        return True
-    t = os.path.getmtime(LIB_PATH)
+HASH_PATH = LIB_PATH + ".srchash"
+
+
+def _source_hash() -> str:
+    """Digest of every source the library is built from (file times do not survive a checkout or a copy)."""
+    import hashlib
+    h = hashlib.sha256()
     deps = [os.path.join(_HERE, "csrc", s) for s in _SOURCES]
     deps.append(os.path.join(os.path.dirname(_HERE), "include", "sdv.h"))
-    return any(os.path.getmtime(d) > t for d in deps)
+    for d in deps:
+        with open(d, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
+def _stale() -> bool:
+    if not os.path.exists(LIB_PATH) or not os.path.exists(HASH_PATH):
+        return True
+    with open(HASH_PATH) as fh:
+        return fh.read().strip() != _source_hash()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -30,6 +43,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         print(" ".join(cmd))
     subprocess.run(cmd, check=True)
     os.replace(LIB_PATH + ".tmp", LIB_PATH)
+    with open(HASH_PATH, "w") as fh:
+        fh.write(_source_hash())
     return LIB_PATH
 
 
