@@ -175,6 +175,72 @@ def accept_len(x: Sequence[int], y: Sequence[int]) -> int:
     return int(lib().orc_accept_len(_p(x), _p(y), len(x)))
 
 
+# ---------------------------------------------------------------- draft extension (Sec. 4.4)
+def reuse_segment(x: Sequence[int], y: Sequence[int], a: int):
+    """Eq. 3: among the drafts beyond the reject point, the longest run on which the draft agrees
+    with the model's own predictions.
+
+    x = x_1..x_n (x[i] is x_{i+1}), y = y_1..y_{n+1}, a = accept length, so the reject position is
+    e = a + 1 (x[a] != y[a]) when a < n.  Every pair (first, last) with a < first <= last < n is
+    tried, as the equation states it; the constraint is x_i = y_i on the whole range.  The paper
+    names no tie rule: the earliest longest run wins.  Returns (first index into x, length),
+    (0, 0) when nothing qualifies (no reject, or no agreement beyond it: the "redundant" pattern
+    of Table 2).
+    """
+    n = len(x)
+    assert len(y) == n + 1 and 0 <= a <= n
+    best_first, best_len = 0, 0
+    for first in range(a + 1, n):
+        for last in range(first, n):
+            if all(x[i] == y[i] for i in range(first, last + 1)) and last - first + 1 > best_len:
+                best_first, best_len = first, last - first + 1
+    return best_first, best_len
+
+
+class DraftExtension:
+    """Reuse of rejected drafts (Sec. 4.4 "Reuse strategy"): one retained segment with a lifetime.
+
+    The paper fixes: the segment is the solution of Eq. 3; it is appended to later drafts; it is
+    kept for at least one decoding step and dropped once its accumulated lifetime or the total
+    draft length exceeds a threshold (32 in Sec. 5.1).  Readings taken where it is silent:
+    * lifetime counts the verify steps the segment was appended to;
+    * a draft that would grow beyond `max_total` with the segment drops the segment instead of
+      cutting it;
+    * a segment into which the accepted prefix reached is spent (its leading tokens were emitted;
+      what still matches behind the new reject point comes back as a new candidate);
+    * a new candidate replaces the retained segment only when strictly longer (length-first), so
+      the retained segment found again in its own appended copy does not renew its lifetime.
+    """
+
+    def __init__(self, max_total: int = 32, max_life: int = 32):
+        self.max_total, self.max_life = int(max_total), int(max_life)
+        self.seg: List[int] = []
+        self.life = 0
+        self.used = False      # the segment is part of the draft under verification
+        self.base_len = 0      # length of that draft before the segment was appended
+
+    def extend(self, draft: Sequence[int]) -> List[int]:
+        draft = [int(t) for t in draft]
+        self.base_len, self.used = len(draft), False
+        if self.seg:
+            if len(draft) + len(self.seg) <= self.max_total:
+                self.used = True
+                return draft + list(self.seg)
+            self.seg, self.life = [], 0
+        return draft
+
+    def update(self, x: Sequence[int], y: Sequence[int], a: int) -> None:
+        """After the verify step of draft x (as returned by extend) with predictions y, accept a."""
+        if self.used:
+            self.life += 1
+        if self.seg and ((self.used and a > self.base_len) or self.life > self.max_life):
+            self.seg, self.life = [], 0
+        first, length = reuse_segment(x, y, a)
+        if length > len(self.seg):
+            self.seg, self.life = [int(t) for t in x[first:first + length]], 0
+        self.used = False
+
+
 # ---------------------------------------------------------------- the model
 class OracleModel:
     """Holds the weight arrays (bf16 bit patterns from sdv_inputs) and an fp32 KV cache."""
@@ -276,10 +342,12 @@ def greedy_decode(model: OracleModel, context, gen: int, chunk: int):
 
 
 def spec_decode(model: OracleModel, context, gen: int, chunk: int, k: int, ngram_n: int, ngram_min: int,
-                drafter=None, search_history: bool = False, keep_logits: bool = False):
+                drafter=None, search_history: bool = False, keep_logits: bool = False,
+                extension: Optional[DraftExtension] = None):
     """Retrieval-based greedy speculative decoding.
 
     `drafter(history, k) -> list` overrides the n-gram drafter (tests use it to force drafts).
+    `extension` appends the retained segment of earlier rejected drafts to every draft (Sec. 4.4).
     The first generated token comes from prefill; each step then verifies [T, x_1..x_dl] at
     positions L..L+dl, accepts a drafts, emits x_1..x_a, y_{a+1} and sets L += a+1.
     Returns (tokens, steps).
@@ -299,10 +367,14 @@ def spec_decode(model: OracleModel, context, gen: int, chunk: int, k: int, ngram
             draft = ngram_draft(hist, hist, ngram_n, ngram_min, k, exclude_from=len(hist) - 1)[0].tolist()
         else:
             draft = ngram_draft(context, hist, ngram_n, ngram_min, k)[0].tolist()
+        if extension is not None:
+            draft = extension.extend(draft)
         dl = len(draft)
         logits = model.forward([T] + draft, L, logits_from=0)
         y = [argmax(logits[j]) for j in range(dl + 1)]
         a = accept_len(draft, y)
+        if extension is not None:
+            extension.update(draft, y, a)
         emitted = draft[:a] + [y[a]]
         room = gen - len(out)
         emitted = emitted[:room]
