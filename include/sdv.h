@@ -41,13 +41,14 @@ enum {
     SDV_ETOOBIG = -7    /* sdv_gemm_noalloc: the problem exceeds its fixed scratch area */
 };
 
-#define SDV_K_MAX 16 /* longest draft per verify step (M = k+1 <= 17 rows) */
+#define SDV_K_MAX 31 /* longest draft per verify step (M = k+1 <= 32 rows) */
 
 typedef struct sdv_ctx sdv_ctx;
 
 /* Model shape and drafter settings.  Supported: head_dim 64 or 128; d_model and d_ffn multiples
  * of 64; vocab a multiple of 16; n_q_heads a multiple of n_kv_heads with at most 8 query heads
- * per KV head and (n_q_heads / n_kv_heads) * (k_max + 1) <= 128; 1 <= k_max <= SDV_K_MAX;
+ * per KV head; 1 <= k_max <= SDV_K_MAX, further limited by shared memory (the k_max + 1 token rows
+ * of d_model columns must fit next to the weight ring: sdv_create returns SDV_EINVAL otherwise);
  * 1 <= ngram_min <= ngram_n <= 8. */
 typedef struct {
     int n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
@@ -121,6 +122,27 @@ int sdv_draft(sdv_ctx *ctx, int k, int32_t *host_draft, int *draft_len);
  * Errors: SDV_ESTATE before prefill has finished, SDV_ECAPACITY, SDV_EINVAL, SDV_ETIMEOUT. */
 int sdv_verify(sdv_ctx *ctx, const int32_t *host_draft, int draft_len, int32_t *host_y, int *accept_len);
 
+/* Draft extension (paper Sec. 4.4 "Reuse strategy", Eq. 3): drafts rejected by one verify step
+ * are kept when they agree with the model's own predictions and are appended to later drafts.
+ *
+ * sdv_extend_draft: call after sdv_draft.  Appends the retained segment to the device draft when
+ * the result has at most max_total tokens (1 <= max_total <= k_max; the paper's threshold is 32
+ * rows); a segment that does not fit is dropped, not cut.  host_draft (max_total ints) and
+ * draft_len may be NULL; if either is given the stream is synchronised and the next sdv_verify
+ * computes exactly draft_len + 1 rows, otherwise it computes max_total + 1 rows (rows past the
+ * draft are padding and never accepted).
+ *
+ * sdv_extension_update: call after sdv_verify, before sdv_commit.  Among the drafts beyond the
+ * reject point e = a + 1 it finds the longest run with x_i == y_i (Eq. 3; the earliest among
+ * equally long runs) and applies the retention rules: a segment that was appended ages by one
+ * step; it is dropped when the accepted prefix reached into it or when its age exceeds max_life
+ * (>= 1); the candidate replaces the retained segment when strictly longer.  host_segment
+ * (k_max ints), segment_len and lifetime may be NULL; if any is given the stream is synchronised.
+ * The segment is cleared by prefill, sdv_rollback and sdv_debug_set_history.
+ * Errors: SDV_ESTATE without a pending draft / verify result, SDV_EINVAL. */
+int sdv_extend_draft(sdv_ctx *ctx, int max_total, int32_t *host_draft, int *draft_len);
+int sdv_extension_update(sdv_ctx *ctx, int max_life, int32_t *host_segment, int *segment_len, int *lifetime);
+
 /* Commit / rollback (paper Sec. 3.2: tokens after the first mismatch are discarded; Sec. 4.4:
  * the accepted prefix is x_1..x_{e-1}, y_e): emits x_1..x_a, y_{a+1} of the last verify, cut to
  * max_emit tokens when max_emit > 0; appends them to the history; L += number emitted; the last
@@ -159,7 +181,11 @@ int sdv_step_bytes(const sdv_ctx *ctx, int rows, int kv_len, double *weight_byte
  * context, without running the model (drafter tests).  L becomes hist_len - 1. */
 int sdv_debug_set_history(sdv_ctx *ctx, const int32_t *host_hist, int hist_len, int n_ctx);
 
-/* Runs the accept scan on host-given predictions y (draft_len+1 ints) against host-given drafts,
+/* Plays the drafter: leaves draft_len host-given tokens as the device draft (extension tests). */
+int sdv_debug_set_draft(sdv_ctx *ctx, const int32_t *host_draft, int draft_len);
+
+/* Runs the accept scan on host-given predictions y (draft_len+1 ints) against host-given drafts
+ * (host_draft == NULL: against the draft already on the device, whose length draft_len must be),
  * leaving the result where sdv_commit expects it. */
 int sdv_debug_accept(sdv_ctx *ctx, const int32_t *host_draft, int draft_len, const int32_t *host_y,
                      int *accept_len);

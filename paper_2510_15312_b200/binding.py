@@ -10,11 +10,11 @@ import numpy as np
 from .build import LIB_PATH, build
 
 OK, EINVAL, ENOMEM, ECAPACITY, ESTATE, ECUDA, ETIMEOUT, ETOOBIG = 0, -1, -2, -3, -4, -5, -6, -7
-K_MAX = 16
+K_MAX = 31
 
 EXPORTS = [
     "sdv_workspace_bytes", "sdv_create", "sdv_load_weights", "sdv_prefill_chunk", "sdv_draft", "sdv_verify",
-    "sdv_commit", "sdv_rollback", "sdv_kv_len", "sdv_set_parity_mode", "sdv_get_logits", "sdv_destroy",
+    "sdv_commit", "sdv_extend_draft", "sdv_extension_update", "sdv_debug_set_draft", "sdv_rollback", "sdv_kv_len", "sdv_set_parity_mode", "sdv_get_logits", "sdv_destroy",
     "sdv_strerror", "sdv_last_cuda_error", "sdv_step_bytes", "sdv_debug_set_history", "sdv_debug_accept",
     "sdv_debug_force_commit", "sdv_debug_read_kv", "sdv_debug_read_hidden", "sdv_debug_gemm",
     "sdv_debug_timeout_probe", "sdv_debug_profile", "sdv_launch_count", "sdv_last_verify_ms",
@@ -65,6 +65,9 @@ def load_library(path: Optional[str] = None):
     L.sdv_draft.argtypes = [vp, C.c_int, i32p, ip]
     L.sdv_verify.argtypes = [vp, i32p, C.c_int, i32p, ip]
     L.sdv_commit.argtypes = [vp, C.c_int, i32p, ip, ip]
+    L.sdv_extend_draft.argtypes = [vp, C.c_int, i32p, ip]
+    L.sdv_extension_update.argtypes = [vp, C.c_int, i32p, ip, ip]
+    L.sdv_debug_set_draft.argtypes = [vp, i32p, C.c_int]
     L.sdv_rollback.argtypes = [vp, C.c_int]
     L.sdv_kv_len.argtypes = [vp]
     L.sdv_set_parity_mode.argtypes = [vp, C.c_int]
@@ -191,6 +194,27 @@ class Sdv:
         self._check(lib().sdv_verify(self._h, dp, dl, y.ctypes.data, C.byref(a)), "sdv_verify")
         return y, a.value
 
+    def extend_draft(self, max_total: int, fetch: bool = True) -> Optional[List[int]]:
+        """Appends the retained segment of rejected drafts to the device draft (Sec. 4.4)."""
+        if not fetch:
+            self._check(lib().sdv_extend_draft(self._h, max_total, None, None), "sdv_extend_draft")
+            return None
+        out = np.zeros(K_MAX, dtype=np.int32)
+        dl = C.c_int(0)
+        self._check(lib().sdv_extend_draft(self._h, max_total, out.ctypes.data, C.byref(dl)), "sdv_extend_draft")
+        return out[:dl.value].tolist()
+
+    def extension_update(self, max_life: int, fetch: bool = True) -> Optional[Tuple[List[int], int]]:
+        """Eq. 3 on the last verify step; returns (retained segment, lifetime) when fetch."""
+        if not fetch:
+            self._check(lib().sdv_extension_update(self._h, max_life, None, None, None), "sdv_extension_update")
+            return None
+        seg = np.zeros(K_MAX, dtype=np.int32)
+        n, life = C.c_int(0), C.c_int(0)
+        self._check(lib().sdv_extension_update(self._h, max_life, seg.ctypes.data, C.byref(n), C.byref(life)),
+                    "sdv_extension_update")
+        return seg[:n.value].tolist(), life.value
+
     def commit(self, max_emit: int = 0) -> Tuple[List[int], int]:
         out = np.zeros(K_MAX + 1, dtype=np.int32)
         n, kv = C.c_int(0), C.c_int(0)
@@ -229,10 +253,19 @@ class Sdv:
         h = np.ascontiguousarray(hist, dtype=np.int32)
         self._check(lib().sdv_debug_set_history(self._h, h.ctypes.data, len(h), n_ctx), "sdv_debug_set_history")
 
-    def debug_accept(self, draft, y) -> int:
+    def debug_set_draft(self, draft):
         d = np.ascontiguousarray(draft, dtype=np.int32)
+        dp = d.ctypes.data if len(d) else None
+        self._check(lib().sdv_debug_set_draft(self._h, dp, len(d)), "sdv_debug_set_draft")
+
+    def debug_accept(self, draft, y) -> int:
+        """draft=None: the accept scan runs on the draft already on the device (len(y) - 1 tokens)."""
         yy = np.ascontiguousarray(y, dtype=np.int32)
         a = C.c_int(0)
+        if draft is None:
+            self._check(lib().sdv_debug_accept(self._h, None, len(yy) - 1, yy.ctypes.data, C.byref(a)), "sdv_debug_accept")
+            return a.value
+        d = np.ascontiguousarray(draft, dtype=np.int32)
         dp = d.ctypes.data if len(d) else None
         self._check(lib().sdv_debug_accept(self._h, dp, len(d), yy.ctypes.data, C.byref(a)), "sdv_debug_accept")
         return a.value

@@ -154,10 +154,15 @@ enum StateWord {
     ST_KV_LEN = 0, ST_HIST_LEN, ST_N_CTX, ST_PENDING, ST_DRAFT_LEN, ST_ACCEPT_LEN, ST_N_EMITTED, ST_ERR,
     ST_VERIFIED,      // 1 when a verify result awaits commit
     ST_MATCH_POS, ST_MATCH_LEN,
+    ST_SEG_LEN,       // retained segment of rejected drafts (draft extension): tokens,
+    ST_SEG_LIFE,      //   verify steps it has been appended to,
+    ST_SEG_USED,      //   1 while it is part of the draft under verification,
+    ST_BASE_LEN,      //   and that draft's length before it was appended
     ST_DRAFT = 16,    // [32]
     ST_Y = 48,        // [33]
     ST_EMITTED = 96,  // [33]
-    ST_WORDS = 160
+    ST_SEG = 160,     // [32]
+    ST_WORDS = 192
 };
 
 struct FwdParams {

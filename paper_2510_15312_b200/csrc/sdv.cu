@@ -725,6 +725,46 @@ int sdv_verify(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, int32_t* 
     return SDV_OK;
 }
 
+int sdv_extend_draft(sdv_ctx* ctx, int max_total, int32_t* host_draft, int* draft_len) {
+    if (!ctx || max_total < 1 || max_total > ctx->cfg.k_max) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->prefill_done || !ctx->draft_pending) return SDV_ESTATE;
+    extend_draft_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, max_total);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    // rows of the next verify: the exact draft length when the caller reads it, else the bound
+    if (ctx->draft_k < max_total) ctx->draft_k = max_total;
+    if (host_draft || draft_len) {
+        int rc = read_state(ctx);
+        if (rc) return rc;
+        const int dl = ctx->pinned[ST_DRAFT_LEN];
+        ctx->draft_k = dl;
+        if (draft_len) *draft_len = dl;
+        if (host_draft)
+            for (int i = 0; i < dl; ++i) host_draft[i] = ctx->pinned[ST_DRAFT + i];
+    }
+    return SDV_OK;
+}
+
+int sdv_extension_update(sdv_ctx* ctx, int max_life, int32_t* host_segment, int* segment_len, int* lifetime) {
+    if (!ctx || max_life < 1) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->verified) return SDV_ESTATE;
+    extension_update_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, max_life);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    if (host_segment || segment_len || lifetime) {
+        int rc = read_state(ctx);
+        if (rc) return rc;
+        const int sl = ctx->pinned[ST_SEG_LEN];
+        if (segment_len) *segment_len = sl;
+        if (lifetime) *lifetime = ctx->pinned[ST_SEG_LIFE];
+        if (host_segment)
+            for (int i = 0; i < sl; ++i) host_segment[i] = ctx->pinned[ST_SEG + i];
+    }
+    return SDV_OK;
+}
+
 int sdv_commit(sdv_ctx* ctx, int max_emit, int32_t* host_emitted, int* n_emitted, int* kv_len) {
     if (!ctx) return SDV_EINVAL;
     if (ctx->poisoned) return SDV_ETIMEOUT;
@@ -804,15 +844,32 @@ int sdv_debug_set_history(sdv_ctx* ctx, const int32_t* host_hist, int hist_len, 
     return SDV_OK;
 }
 
-int sdv_debug_accept(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, const int32_t* host_y, int* accept_len) {
-    if (!ctx || !host_y || draft_len < 0 || draft_len > ctx->cfg.k_max || (draft_len && !host_draft)) return SDV_EINVAL;
-    DraftArg a, y;
+int sdv_debug_set_draft(sdv_ctx* ctx, const int32_t* host_draft, int draft_len) {
+    if (!ctx || draft_len < 0 || draft_len > ctx->cfg.k_max || (draft_len && !host_draft)) return SDV_EINVAL;
+    DraftArg a;
     fill_draft_arg(a, host_draft, draft_len);
-    fill_draft_arg(y, host_y, draft_len + 1);
     set_draft_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, a);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    ctx->draft_pending = true;
+    ctx->draft_k = draft_len;
+    ctx->verified = false;
+    return SDV_OK;
+}
+
+int sdv_debug_accept(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, const int32_t* host_y, int* accept_len) {
+    if (!ctx || !host_y || draft_len < 0 || draft_len > ctx->cfg.k_max) return SDV_EINVAL;
+    DraftArg a, y;
+    fill_draft_arg(y, host_y, draft_len + 1);
+    if (host_draft) {
+        // host_draft == NULL: the draft already on the device (draft_len must be its length)
+        fill_draft_arg(a, host_draft, draft_len);
+        set_draft_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, a);
+        ctx->launches++;
+    }
     set_y_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, y);
     accept_kernel<<<1, 32 * (draft_len + 1), 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 1);
-    ctx->launches += 3;
+    ctx->launches += 2;
     CK(cudaGetLastError());
     ctx->verified = true;
     ctx->last_rows = draft_len + 1;

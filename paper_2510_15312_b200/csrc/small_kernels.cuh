@@ -92,6 +92,8 @@ __global__ void ngram_draft_kernel(int* state, const int* hist, int n, int n_min
         }
         if (threadIdx.x == 0) {
             state[ST_DRAFT_LEN] = dl;
+            state[ST_BASE_LEN] = dl;
+            state[ST_SEG_USED] = 0;
             state[ST_MATCH_POS] = pos;
             state[ST_MATCH_LEN] = mlen;
         }
@@ -106,11 +108,82 @@ struct DraftArg {
 // Caller-supplied drafts (by value: no host buffer has to outlive the call).
 __global__ void set_draft_kernel(int* state, DraftArg a) {
     if ((int)threadIdx.x < a.n) state[ST_DRAFT + threadIdx.x] = a.tok[threadIdx.x];
-    if (threadIdx.x == 0) state[ST_DRAFT_LEN] = a.n;
+    if (threadIdx.x == 0) {
+        state[ST_DRAFT_LEN] = a.n;
+        state[ST_BASE_LEN] = a.n;
+        state[ST_SEG_USED] = 0;
+    }
 }
 // Caller-supplied predictions for the stand-alone accept scan.
 __global__ void set_y_kernel(int* state, DraftArg a) {
     if ((int)threadIdx.x < a.n) state[ST_Y + threadIdx.x] = a.tok[threadIdx.x];
+}
+
+// ------------------------------------------------------------------------------------------
+// Draft extension (reuse of rejected drafts).  One warp each.
+//
+// extend: the retained segment is appended to the draft the drafter left, unless the draft would
+// grow beyond max_total tokens, in which case the segment is dropped.
+__global__ void extend_draft_kernel(int* state, int max_total) {
+    const int lane = threadIdx.x;
+    const int m = state[ST_DRAFT_LEN], sl = state[ST_SEG_LEN];
+    const bool fits = sl > 0 && m + sl <= max_total;
+    const int tok = (fits && lane < sl) ? state[ST_SEG + lane] : 0;
+    __syncwarp();
+    if (fits && lane < sl) state[ST_DRAFT + m + lane] = tok;
+    if (lane == 0) {
+        state[ST_BASE_LEN] = m;
+        state[ST_SEG_USED] = fits ? 1 : 0;
+        if (fits) {
+            state[ST_DRAFT_LEN] = m + sl;
+        } else if (sl > 0) {
+            state[ST_SEG_LEN] = 0;
+            state[ST_SEG_LIFE] = 0;
+        }
+    }
+}
+
+// update, after the accept scan of a verify step: lane i tests x_{i+1} == y_{i+1} beyond the reject
+// point; the longest run of agreeing drafts (the earliest among equals) is the candidate.  Runs of
+// length t survive t - 1 rounds of r &= r >> 1 (bit i of r: a run of the current length starts at
+// i).  Then the retention rules: a segment that was appended ages by one step; it is dropped when
+// the accepted prefix reached into it or its age passes max_life; a strictly longer candidate
+// replaces what is retained.
+__global__ void extension_update_kernel(int* state, int max_life) {
+    const int lane = threadIdx.x;
+    const int dl = state[ST_DRAFT_LEN], a = state[ST_ACCEPT_LEN];
+    const int x = state[ST_DRAFT + lane], y = state[ST_Y + lane];
+    const bool agree = lane < dl && lane > a && x == y;
+    unsigned r = __ballot_sync(0xffffffffu, agree);
+    int len = 0, first = 0;
+    if (r) {
+        len = 1;
+        for (unsigned nr = r & (r >> 1); nr; nr = r & (r >> 1)) {
+            r = nr;
+            ++len;
+        }
+        first = __ffs((int)r) - 1;
+    }
+    int sl = state[ST_SEG_LEN], life = state[ST_SEG_LIFE];
+    const int used = state[ST_SEG_USED], base = state[ST_BASE_LEN];
+    if (used) ++life;
+    if (sl > 0 && ((used && a > base) || life > max_life)) {
+        sl = 0;
+        life = 0;
+    }
+    const bool replace = len > sl;
+    const int tok = (replace && lane < len) ? state[ST_DRAFT + first + lane] : 0;
+    __syncwarp();
+    if (replace) {
+        if (lane < len) state[ST_SEG + lane] = tok;
+        sl = len;
+        life = 0;
+    }
+    if (lane == 0) {
+        state[ST_SEG_LEN] = sl;
+        state[ST_SEG_LIFE] = life;
+        state[ST_SEG_USED] = 0;
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -213,6 +286,10 @@ __global__ void set_state_kernel(int* state, int kv_len, int hist_len, int n_ctx
     if (pending_from_hist && hist_len > 0) state[ST_PENDING] = hist[hist_len - 1];
     state[ST_DRAFT_LEN] = 0;
     state[ST_VERIFIED] = 0;
+    state[ST_SEG_LEN] = 0;   // a new request starts without a retained segment
+    state[ST_SEG_LIFE] = 0;
+    state[ST_SEG_USED] = 0;
+    state[ST_BASE_LEN] = 0;
 }
 
 // A bounded wait on a word nothing ever sets: exercises the give-up path of the device waits.

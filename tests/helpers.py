@@ -51,12 +51,17 @@ def steps_from_golden(g) -> List[RefStep]:
     return out
 
 
-def compare_step(sdv, step: RefStep, k: int, stats: dict):
+def compare_step(sdv, step: RefStep, k: int, stats: dict, predrafted: bool = False, before_commit=None):
     """Runs draft + verify for one reference step on a context already in the step's state and
-    checks everything the step fixes.  Commits the ORACLE's outcome so the states stay aligned."""
+    checks everything the step fixes.  Commits the ORACLE's outcome so the states stay aligned.
+    predrafted: the device already holds the step's draft (verify runs on it as it is);
+    before_commit(y, a): called with the device's predictions and accept length before the commit."""
     dl = len(step.draft)
     assert sdv.kv_len() == step.kv_len_before
-    if step.from_drafter:
+    if predrafted:
+        y, a = sdv.verify(None)
+        rows = dl + 1
+    elif step.from_drafter:
         got_draft = sdv.draft(k)
         assert got_draft == step.draft, f"draft differs at L={step.kv_len_before}: {got_draft} vs {step.draft}"
         y, a = sdv.verify(None)
@@ -93,6 +98,8 @@ def compare_step(sdv, step: RefStep, k: int, stats: dict):
         assert a == step.accept, f"accept length {a} vs {step.accept} at L={step.kv_len_before}"
     stats["steps"] = stats.get("steps", 0) + 1
     stats.setdefault("accepts", []).append(step.accept)
+    if before_commit is not None:
+        before_commit([int(t) for t in y[:dl + 1]], int(a))
     # teacher forcing: commit what the oracle committed
     sdv.debug_force_commit(len(step.emitted) - 1, step.emitted[-1])
     assert sdv.kv_len() == step.kv_len_before + len(step.emitted)
