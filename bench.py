@@ -173,6 +173,10 @@ def main():
     ap.add_argument("--k", type=int, default=0)
     ap.add_argument("--sweep-k", default="", help="comma-separated draft lengths: adds verify-step us and GB/s per k "
                                                  "at the fixed KV length reached after prefill (rolled back after each step)")
+    ap.add_argument("--extension", type=int, default=0, metavar="MAX_TOTAL",
+                    help="adds a third timed loop with draft extension (Sec. 4.4): drafts grow to at most MAX_TOTAL "
+                         "tokens by reuse of rejected drafts; reported under \"extension\"")
+    ap.add_argument("--extension-life", type=int, default=32)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -198,9 +202,11 @@ def main():
 
     k = cfg.k
     sweep = [int(x) for x in args.sweep_k.split(",") if x.strip()]
-    k_max = max([k] + sweep)
+    k_max = max([k] + sweep + [args.extension])
     total = args.warmup + args.steps
     max_seq = cfg.n_ctx + 2 * total * (k + 1) + 64          # room for two timed loops at full acceptance
+    if args.extension:
+        max_seq += total * (args.extension + 1)
     cores = len(os.sched_getaffinity(0))
     w = make_weights(cfg, threads=max(8, cores // max(1, world)))
     ctx = make_context(cfg)
@@ -271,6 +277,33 @@ def main():
     barrier()
     ms_e2e = e0.elapsed_time(e1)
 
+    # ---- optional: device-resident loop with draft extension (every step computes MAX_TOTAL + 1 rows)
+    ext = None
+    if args.extension:
+        def ext_loop(n):
+            tokens, kms = 0, []
+            for _ in range(n):
+                s.draft(k, fetch=False)
+                s.extend_draft(args.extension, fetch=False)
+                s.verify(None, fetch=False)
+                s.extension_update(args.extension_life, fetch=False)
+                em, _ = s.commit()
+                tokens += len(em)
+                kms.append(s.last_verify_ms())
+            return tokens, kms
+        ext_loop(args.warmup)
+        barrier()
+        x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        x0.record(stream)
+        tokens_x, kms_x = ext_loop(args.steps)
+        x1.record(stream)
+        barrier()
+        ms_x = x0.elapsed_time(x1)
+        ext = {"max_total": args.extension, "max_life": args.extension_life, "rows_per_verify": args.extension + 1,
+               "value": tokens_x / (ms_x * 1e-3), "unit": UNIT, "ms_per_step": ms_x / args.steps,
+               "verify_kernel_us": statistics.mean(kms_x) * 1e3,
+               "accepted_drafts_per_step": tokens_x / args.steps - 1.0, "scope": "rank 0"}
+
     (ms_total, ms_e2e), (tokens_all, tokens_e_all) = aggregate_over_ranks([ms_total, ms_e2e], [tokens, tokens_e], world,
                                                                           "cuda")
 
@@ -304,6 +337,8 @@ def main():
             "gpu_launches": launches,
             "clocks": clocks,
         }
+        if ext:
+            line["extension"] = ext
         if sweep:
             line["k_sweep"] = []
             for kk in sweep:
