@@ -134,6 +134,16 @@ void choose_partition(OpDesc& o, int G, int rows, bool merge, bool always_add) {
         }
     }
 }
+// A block whose share has fewer row tiles than a pass may hold walks it in one pass all the same:
+// RW then only sets the stage length.  Shrinking RW to the tiles a block really has (a power of two)
+// doubles SK until a stage is back at the ring slot's size, i.e. fewer, longer bulk copies.
+void fit_pass_width(OpDesc& o) {
+    if (o.follow) return;
+    const int per = o.unit * ((o.T / o.unit + o.P_row - 1) / o.P_row);  // row tiles of the largest share
+    while (o.RW > 1 && o.RW / 2 >= per) o.RW /= 2;
+    o.SK = kStageBytes / kStepBytes / o.RW;
+}
+
 // Operations whose epilogue needs complete sums: all columns in one block, rows spread evenly.
 void full_k_partition(OpDesc& o, int G, int unit) {
     o.RW = 16;
@@ -208,6 +218,7 @@ void setup_ops(FwdParams& P, const sdv_config* cfg, int G) {
                 o.RW = 16; o.SK = kStageBytes / kStepBytes / 16; o.unit = 1; o.follow = 1; o.P_row = 1; o.P_k = P.op[OP_GU].P_row;
                 break;
         }
+        fit_pass_width(o);
         if (ops[i].idx == OP_DOWN) {
             o.rot = P.op[OP_GU].rot;
         } else {
@@ -922,6 +933,7 @@ int sdv_debug_gemm(sdv_ctx* ctx, const float* host_x, const uint16_t* host_w, fl
     o.T = N / 16;
     o.K16 = K / 16;
     choose_partition(o, ctx->G, M, false, false);
+    fit_pass_width(o);
     CK(cudaMemcpyAsync(ws + ctx->r.staging, host_w, (size_t)N * K * 2, cudaMemcpyDefault, s));
     int rc = pack_op(ctx, o, ws + ctx->r.wraw, (const uint16_t*)(ws + ctx->r.staging), N, nullptr, 0, nullptr, K, 0, 0,
                      o.T, 0);
@@ -1094,6 +1106,7 @@ int sdv_gemm_noalloc(const float* dev_x, const uint16_t* dev_w, float* dev_y, in
     o.T = N / 16;
     o.K16 = K / 16;
     choose_partition(o, sms, M, false, false);
+    fit_pass_width(o);
     P.wraw = sc;
     P.raw_x = dev_x;  // the caller's rows are read in place
     P.raw_out = (float*)(sc + kNaOutOff);
