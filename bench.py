@@ -34,7 +34,7 @@ UNIT = "tokens/s"
 # algorithmic bytes: captured on the 0.5B-shaped workload (profiles/sdv_forward_kernel_qwen0.5b_ncu_full.md)
 # and scaled to the timed workload by its algorithmic bytes (traffic grows with the bytes streamed).
 # None once the kernel has changed since the capture.
-NCU_TRAFFIC_RATIO = 1.0047
+NCU_TRAFFIC_RATIO = 1.0051
 
 
 def load_peaks():
