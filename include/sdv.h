@@ -41,6 +41,7 @@ enum {
     SDV_ETOOBIG = -7    /* sdv_gemm_noalloc: the problem exceeds its fixed scratch area */
 };
 
+#define SDV_NGRAM_MAX 4096 /* longest history suffix the drafter can be asked to match */
 #define SDV_K_MAX 31 /* longest draft per verify step (M = k+1 <= 32 rows) */
 
 typedef struct sdv_ctx sdv_ctx;
@@ -49,7 +50,10 @@ typedef struct sdv_ctx sdv_ctx;
  * of 64; vocab a multiple of 16; n_q_heads a multiple of n_kv_heads with at most 8 query heads
  * per KV head; 1 <= k_max <= SDV_K_MAX, further limited by shared memory (the k_max + 1 token rows
  * of d_model columns must fit next to the weight ring: sdv_create returns SDV_EINVAL otherwise);
- * 1 <= ngram_min <= ngram_n <= 8. */
+ * 1 <= ngram_min <= ngram_n <= SDV_NGRAM_MAX.  ngram_n = SDV_NGRAM_MAX with search_history = 1 is
+ * longest-suffix retrieval over the request context and the generated tokens: the match a suffix
+ * automaton over that text returns (the retrieval algorithm the paper's baselines use, Sec. 5.1 (3)),
+ * found here by a parallel scan of all end positions instead of an automaton. */
 typedef struct {
     int n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
     int max_seq;        /* KV rows / history entries the context can hold */

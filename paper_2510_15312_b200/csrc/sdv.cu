@@ -39,7 +39,7 @@ bool config_ok(const sdv_config* c) {
     if (g > 8) return false;
     if (c->k_max < 1 || c->k_max > SDV_K_MAX) return false;
     if (c->max_seq < c->k_max + 2) return false;
-    if (c->ngram_n < 1 || c->ngram_n > 8 || c->ngram_min < 1 || c->ngram_min > c->ngram_n) return false;
+    if (c->ngram_n < 1 || c->ngram_n > SDV_NGRAM_MAX || c->ngram_min < 1 || c->ngram_min > c->ngram_n) return false;
     if (!(c->rope_theta > 0.f) || !(c->rms_eps > 0.f)) return false;
     return true;
 }

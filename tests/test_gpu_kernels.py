@@ -73,6 +73,40 @@ def test_drafter_bit_exact_on_random_arrays(search_history):
         s.close()
 
 
+@pytest.mark.parametrize("search_history", [False, True])
+def test_longest_suffix_drafter_bit_exact(search_history):
+    """Suffix length up to 4096 (longest-suffix retrieval): planted repeats of 5..3000 tokens,
+    contexts up to 8200, and the degenerate constant and periodic texts (longest compare loops)."""
+    cfg = get_config("tiny").with_(ngram_n=4096, ngram_min=2)
+    s = Sdv(config_from(cfg, k_max=16, max_seq=9000, search_history=search_history))
+    rng = np.random.default_rng(31 + search_history)
+    longest = 0
+    cases = []
+    for trial in range(120):
+        V = int(rng.integers(2, 50))
+        n_ctx = int(rng.integers(10, 200)) if trial % 3 else int(rng.integers(3500, 8200))
+        n_gen = int(rng.integers(1, 400)) if n_ctx > 3000 else int(rng.integers(1, 30))
+        hist = rng.integers(0, V, n_ctx + n_gen).astype(np.int32)
+        if n_ctx > 3000:
+            L = int(rng.integers(5, 3000))
+            p = int(rng.integers(L, n_ctx - 20))
+            hist[p - L:p] = hist[-L:]
+        cases.append((hist, n_ctx))
+    cases.append((np.full(8000, 7, dtype=np.int32), 7000))                 # constant text
+    cases.append((np.array([1, 2, 3, 4, 5] * 1600, dtype=np.int32), 6000))   # periodic text
+    for hist, n_ctx in cases:
+        k = int(rng.integers(1, 17))
+        got = _draft_case(s, search_history, hist, n_ctx, k)
+        if search_history:
+            ref, _, ml = O.ngram_draft(hist, hist, 4096, 2, k, exclude_from=len(hist) - 1)
+        else:
+            ref, _, ml = O.ngram_draft(hist[:n_ctx], hist, 4096, 2, k)
+        assert got == ref.tolist(), (len(hist), n_ctx, k, ml)
+        longest = max(longest, ml)
+    assert longest == 4096
+    s.close()
+
+
 def test_drafter_edge_cases(ctx_tiny):
     s = ctx_tiny
     assert _draft_case(s, False, [1, 2, 3, 9, 3], 3, 4) == []           # only match ends at the last context token

@@ -31,7 +31,7 @@ def test_host_side_argument_checks():
     good = SdvConfig(2, 256, 4, 4, 64, 1024, 4096, 600, 4, 0, 0, 3, 1, 0, 1e4, 1e-6)
     assert L.sdv_workspace_bytes(ctypes.byref(good)) > 0
     for field, bad in (("head_dim", 96), ("d_model", 250), ("vocab", 4097), ("k_max", 32), ("n_kv_heads", 3),
-                       ("ngram_min", 4), ("max_seq", 3), ("d_ffn", 1000)):
+                       ("ngram_min", 4), ("ngram_n", 4097), ("max_seq", 3), ("d_ffn", 1000)):
         c = SdvConfig.from_buffer_copy(good)
         setattr(c, field, bad)
         assert L.sdv_workspace_bytes(ctypes.byref(c)) == 0, field
