@@ -168,6 +168,20 @@ def ngram_draft(search, hist, n: int, n_min: int, k: int, exclude_from: Optional
     return out[:dl].copy(), mp.value, ml.value
 
 
+def retrieve_draft(search, hist, database, n: int, n_min: int, k: int, exclude_from: Optional[int] = None):
+    """Drafting from the request's text and an extra token database (Sec. 5.1 (3), Sec. 5.5): both
+    arrays are searched with the same suffix matcher; the longer match supplies the draft, the
+    request's own text on equal length (the paper names no rule).  Returns (draft, source, match_pos,
+    match_len) with source "own", "db" or None."""
+    d1, p1, m1 = ngram_draft(search, hist, n, n_min, k, exclude_from)
+    if database is None or len(database) < 2:
+        return d1, ("own" if m1 else None), p1, m1
+    d2, p2, m2 = ngram_draft(database, hist, n, n_min, k)
+    if m2 > m1:
+        return d2, "db", p2, m2
+    return d1, ("own" if m1 else None), p1, m1
+
+
 def accept_len(x: Sequence[int], y: Sequence[int]) -> int:
     x = np.ascontiguousarray(x, dtype=np.int32)
     y = np.ascontiguousarray(y, dtype=np.int32)

@@ -14,7 +14,7 @@ K_MAX = 31
 
 EXPORTS = [
     "sdv_workspace_bytes", "sdv_create", "sdv_load_weights", "sdv_prefill_chunk", "sdv_draft", "sdv_verify",
-    "sdv_commit", "sdv_extend_draft", "sdv_extension_update", "sdv_debug_set_draft", "sdv_rollback", "sdv_kv_len", "sdv_set_parity_mode", "sdv_get_logits", "sdv_destroy",
+    "sdv_commit", "sdv_set_database", "sdv_extend_draft", "sdv_extension_update", "sdv_debug_set_draft", "sdv_rollback", "sdv_kv_len", "sdv_set_parity_mode", "sdv_get_logits", "sdv_destroy",
     "sdv_strerror", "sdv_last_cuda_error", "sdv_step_bytes", "sdv_debug_set_history", "sdv_debug_accept",
     "sdv_debug_force_commit", "sdv_debug_read_kv", "sdv_debug_read_hidden", "sdv_debug_gemm",
     "sdv_debug_timeout_probe", "sdv_debug_profile", "sdv_launch_count", "sdv_last_verify_ms",
@@ -65,6 +65,7 @@ def load_library(path: Optional[str] = None):
     L.sdv_draft.argtypes = [vp, C.c_int, i32p, ip]
     L.sdv_verify.argtypes = [vp, i32p, C.c_int, i32p, ip]
     L.sdv_commit.argtypes = [vp, C.c_int, i32p, ip, ip]
+    L.sdv_set_database.argtypes = [vp, i32p, C.c_int]
     L.sdv_extend_draft.argtypes = [vp, C.c_int, i32p, ip]
     L.sdv_extension_update.argtypes = [vp, C.c_int, i32p, ip, ip]
     L.sdv_debug_set_draft.argtypes = [vp, i32p, C.c_int]
@@ -193,6 +194,11 @@ class Sdv:
         a = C.c_int(0)
         self._check(lib().sdv_verify(self._h, dp, dl, y.ctypes.data, C.byref(a)), "sdv_verify")
         return y, a.value
+
+    def set_database(self, tokens):
+        """Extra token database the drafter searches besides the request's own text (empty: none)."""
+        t = np.ascontiguousarray(tokens, dtype=np.int32)
+        self._check(lib().sdv_set_database(self._h, t.ctypes.data if len(t) else None, len(t)), "sdv_set_database")
 
     def extend_draft(self, max_total: int, fetch: bool = True) -> Optional[List[int]]:
         """Appends the retained segment of rejected drafts to the device draft (Sec. 4.4)."""

@@ -158,6 +158,7 @@ enum StateWord {
     ST_SEG_LIFE,      //   verify steps it has been appended to,
     ST_SEG_USED,      //   1 while it is part of the draft under verification,
     ST_BASE_LEN,      //   and that draft's length before it was appended
+    ST_DB_LEN,        // tokens in the extra token database the drafter also searches (0: none)
     ST_DRAFT = 16,    // [32]
     ST_Y = 48,        // [33]
     ST_EMITTED = 96,  // [33]

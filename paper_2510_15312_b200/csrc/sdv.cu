@@ -22,7 +22,7 @@ namespace {
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Regions {
-    size_t state, bar, never, hist, rope, norm_w, bias, wlayers, wlm, emb, kcache, vcache, h, qkv_acc, sumsq, part_o,
+    size_t state, bar, never, hist, db, rope, norm_w, bias, wlayers, wlm, emb, kcache, vcache, h, qkv_acc, sumsq, part_o,
         part_ml, cand_val, cand_idx, logits, raw_out, staging, wraw, xstage, prof, total;
     size_t layer_stride, staging_bytes, raw_kmax;
 };
@@ -59,6 +59,7 @@ Regions carve(const sdv_config* c) {
     r.bar = take(256);
     r.never = take(256);
     r.hist = take(((size_t)c->max_seq + 64) * 4);
+    r.db = take(((size_t)c->max_seq + 64) * 4);
     r.rope = take((size_t)c->max_seq * (hd / 2) * sizeof(float2));
     r.norm_w = take(((size_t)c->n_layers * 2 + 1) * d * 4);
     r.bias = take((size_t)c->n_layers * nqkv * 4);
@@ -678,8 +679,8 @@ int sdv_draft(sdv_ctx* ctx, int k, int32_t* host_draft, int* draft_len) {
     if (ctx->poisoned) return SDV_ETIMEOUT;
     if (!ctx->prefill_done) return SDV_ESTATE;
     int* hist = (int*)(ctx->ws + ctx->r.hist);
-    ngram_draft_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->P.state, hist, ctx->cfg.ngram_n, ctx->cfg.ngram_min, k,
-                                                    ctx->cfg.search_history);
+    ngram_draft_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->P.state, hist, (const int*)(ctx->ws + ctx->r.db), ctx->cfg.ngram_n,
+                                                    ctx->cfg.ngram_min, k, ctx->cfg.search_history);
     ctx->launches++;
     CK(cudaGetLastError());
     ctx->draft_pending = true;
@@ -733,6 +734,19 @@ int sdv_verify(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, int32_t* 
         if (host_y)
             for (int i = 0; i <= dl; ++i) host_y[i] = ctx->pinned[ST_Y + i];
     }
+    return SDV_OK;
+}
+
+int sdv_set_database(sdv_ctx* ctx, const int32_t* host_tokens, int n) {
+    if (!ctx || n < 0 || n > ctx->cfg.max_seq || (n && !host_tokens)) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    for (int i = 0; i < n; ++i)
+        if (host_tokens[i] < 0 || host_tokens[i] >= ctx->cfg.vocab) return SDV_EINVAL;
+    if (n) CK(cudaMemcpyAsync(ctx->ws + ctx->r.db, host_tokens, (size_t)n * 4, cudaMemcpyDefault, ctx->stream));
+    set_word_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, ST_DB_LEN, n);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    CK(cudaStreamSynchronize(ctx->stream));  // the caller's buffer may go away
     return SDV_OK;
 }
 

@@ -52,23 +52,39 @@ __global__ void fill_i32_kernel(int* p, int v, long long n) {
 // suffix of search[0..p] and the history (capped at n), then a block-wide maximum of (m(p), p)
 // picks the longest and, among those, the latest match; up to k following tokens are the draft.
 // The search array is the history's own prefix: the request context (first n_ctx tokens), or,
-// with search_history, everything but the last token (the suffix must not match itself).
-__global__ void ngram_draft_kernel(int* state, const int* hist, int n, int n_min, int k, int search_history) {
-    __shared__ unsigned long long best_s[32];
-    const int hist_len = state[ST_HIST_LEN];
-    const int n_search = search_history ? hist_len : state[ST_N_CTX];
-    const int exclude_from = search_history ? hist_len - 1 : n_search;
+// with search_history, everything but the last token (the suffix must not match itself).  A second
+// array, the extra token database, is searched the same way; an equally long match in the request's
+// own text wins over one in the database (bit 32 of the key).  ST_MATCH_POS reports a database
+// position p as -(p + 2).
+__device__ __forceinline__ unsigned long long suffix_scan(const int* search, int n_search, int exclude_from,
+                                                          const int* hist, int hist_len, int n, int n_min,
+                                                          unsigned long long src_bit) {
     unsigned long long best = 0;
     for (int p = threadIdx.x; p + 1 < n_search && p < exclude_from; p += blockDim.x) {
         int cap = n;
         if (p + 1 < cap) cap = p + 1;
         if (hist_len < cap) cap = hist_len;
         int mlen = 0;
-        while (mlen < cap && hist[p - mlen] == hist[hist_len - 1 - mlen]) ++mlen;
+        while (mlen < cap && search[p - mlen] == hist[hist_len - 1 - mlen]) ++mlen;
         if (mlen >= n_min && mlen > 0) {
-            const unsigned long long key = ((unsigned long long)mlen << 32) | (unsigned)p;
+            const unsigned long long key = ((unsigned long long)mlen << 33) | src_bit | (unsigned)p;
             if (key > best) best = key;
         }
+    }
+    return best;
+}
+
+__global__ void ngram_draft_kernel(int* state, const int* hist, const int* db, int n, int n_min, int k,
+                                   int search_history) {
+    __shared__ unsigned long long best_s[32];
+    const int hist_len = state[ST_HIST_LEN];
+    const int n_search = search_history ? hist_len : state[ST_N_CTX];
+    const int exclude_from = search_history ? hist_len - 1 : n_search;
+    const int db_len = state[ST_DB_LEN];
+    unsigned long long best = suffix_scan(hist, n_search, exclude_from, hist, hist_len, n, n_min, 1ull << 32);
+    if (db_len > 1) {
+        const unsigned long long b2 = suffix_scan(db, db_len, db_len, hist, hist_len, n, n_min, 0ull);
+        if (b2 > best) best = b2;
     }
     for (int off = 16; off; off >>= 1) {
         const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, off);
@@ -84,11 +100,15 @@ __global__ void ngram_draft_kernel(int* state, const int* hist, int n, int n_min
         }
         int dl = 0, pos = -1, mlen = 0;
         if (best != 0) {
-            pos = (int)(best & 0xffffffffu);
-            mlen = (int)(best >> 32);
-            dl = n_search - 1 - pos;
+            const bool own = ((best >> 32) & 1ull) != 0;
+            const int* src = own ? hist : db;
+            const int n_src = own ? n_search : db_len;
+            const int p = (int)(best & 0xffffffffu);
+            mlen = (int)(best >> 33);
+            pos = own ? p : -(p + 2);
+            dl = n_src - 1 - p;
             if (dl > k) dl = k;
-            if ((int)threadIdx.x < dl) state[ST_DRAFT + threadIdx.x] = hist[pos + 1 + threadIdx.x];
+            if ((int)threadIdx.x < dl) state[ST_DRAFT + threadIdx.x] = src[p + 1 + threadIdx.x];
         }
         if (threadIdx.x == 0) {
             state[ST_DRAFT_LEN] = dl;
@@ -98,6 +118,10 @@ __global__ void ngram_draft_kernel(int* state, const int* hist, int n, int n_min
             state[ST_MATCH_LEN] = mlen;
         }
     }
+}
+
+__global__ void set_word_kernel(int* state, int word, int value) {
+    if (threadIdx.x == 0) state[word] = value;
 }
 
 struct DraftArg {

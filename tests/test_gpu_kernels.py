@@ -107,6 +107,41 @@ def test_longest_suffix_drafter_bit_exact(search_history):
     s.close()
 
 
+def test_drafter_with_extra_database_bit_exact():
+    """The drafter over the request's text and an extra token database against the oracle's rule."""
+    cfg = get_config("tiny").with_(ngram_n=64, ngram_min=1)
+    s = Sdv(config_from(cfg, k_max=16, max_seq=9000))
+    rng = np.random.default_rng(77)
+    from_db = 0
+    for trial in range(200):
+        V = int(rng.integers(2, 8))
+        n_ctx = int(rng.integers(2, 300))
+        hist = rng.integers(0, V, n_ctx + int(rng.integers(1, 30))).astype(np.int32)
+        db = rng.integers(0, V, int(rng.integers(0, 6000)) if trial % 4 else int(rng.integers(0, 3))).astype(np.int32)
+        if trial % 3 == 0 and len(db) > 100:
+            L = min(int(rng.integers(3, 40)), len(hist))
+            p = int(rng.integers(L, len(db) - 20))
+            db[p - L:p] = hist[-L:]
+        k = int(rng.integers(1, 17))
+        s.set_database(db)
+        got = _draft_case(s, False, hist, n_ctx, k)
+        ref, src, _, _ = O.retrieve_draft(hist[:n_ctx], hist, db, 64, 1, k)
+        assert got == ref.tolist(), (trial, len(db), n_ctx, k, src)
+        from_db += src == "db"
+    assert from_db > 20
+    s.set_database([])                                      # removed: back to the request's text alone
+    hist = np.array([5, 1, 2, 7, 7, 9, 9, 1, 2], dtype=np.int32)
+    s.set_database([3, 9, 1, 2, 4, 4])
+    assert _draft_case(s, False, hist, 5, 2) == [4, 4]      # the longer match is in the database
+    s.set_database([1, 2, 4, 4])
+    assert _draft_case(s, False, hist, 5, 2) == [7, 7]      # equal length: the request's own text
+    s.set_database([])
+    assert _draft_case(s, False, hist, 5, 2) == [7, 7]
+    with pytest.raises(pkg.SdvError):
+        s.set_database([cfg.vocab])                         # token out of range
+    s.close()
+
+
 def test_drafter_edge_cases(ctx_tiny):
     s = ctx_tiny
     assert _draft_case(s, False, [1, 2, 3, 9, 3], 3, 4) == []           # only match ends at the last context token

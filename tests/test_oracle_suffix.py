@@ -73,3 +73,44 @@ def test_periodic_text():
     draft, p, m = O.ngram_draft(hist, hist, N_MAX, 1, 5, exclude_from=len(hist) - 1)
     assert (p, m) == (len(hist) - 4, len(hist) - 3)
     assert draft.tolist() == [1, 2, 3]          # only three tokens follow the match
+
+
+def test_database_retrieval_rule():
+    """Request text and extra database (Sec. 5.1 (3)): the longer suffix match supplies the draft,
+    the request's own text on equal length; checked against substring search on both arrays."""
+    rng = np.random.default_rng(9)
+    seen = {"own": 0, "db": 0, None: 0}
+    for trial in range(300):
+        V = int(rng.integers(2, 5))
+        n_ctx = int(rng.integers(2, 80))
+        hist = rng.integers(0, V, n_ctx + int(rng.integers(1, 20))).astype(np.int32)
+        db = rng.integers(0, V, int(rng.integers(0, 120))).astype(np.int32)
+        if trial % 3 == 0 and len(db) > 30:               # plant the suffix in the database
+            L = int(rng.integers(3, 15))
+            L = min(L, len(hist))
+            p = int(rng.integers(L, len(db) - 5))
+            db[p - L:p] = hist[-L:]
+        n_min = int(rng.integers(1, 3))
+        k = int(rng.integers(1, 9))
+        draft, src, mp, ml = O.retrieve_draft(hist[:n_ctx], hist, db, N_MAX, n_min, k)
+        p1, l1 = _by_substring_search(bytes(hist[:n_ctx].astype(np.uint8)), bytes(hist.astype(np.uint8)), n_min, n_ctx)
+        p2, l2 = (-1, 0)
+        if len(db) >= 2:
+            p2, l2 = _by_substring_search(bytes(db.astype(np.uint8)), bytes(hist.astype(np.uint8)), n_min, len(db))
+        if l2 > l1:
+            assert (src, mp, ml) == ("db", p2, l2)
+            assert draft.tolist() == db[p2 + 1:p2 + 1 + k].tolist()
+        elif l1 > 0:
+            assert (src, mp, ml) == ("own", p1, l1)
+            assert draft.tolist() == hist[:n_ctx][p1 + 1:p1 + 1 + k].tolist()
+        else:
+            assert src is None and len(draft) == 0
+        seen[src] += 1
+    assert seen["own"] > 30 and seen["db"] > 30
+    # by hand: equal length -> the request's own text; longer -> the database
+    hist = np.array([5, 1, 2, 7, 7, 9, 9, 1, 2], dtype=np.int32)
+    ctx = hist[:5]
+    d, src, mp, ml = O.retrieve_draft(ctx, hist, np.array([1, 2, 4, 4], dtype=np.int32), 8, 1, 2)
+    assert (d.tolist(), src, mp, ml) == ([7, 7], "own", 2, 2)
+    d, src, mp, ml = O.retrieve_draft(ctx, hist, np.array([3, 9, 1, 2, 4, 4], dtype=np.int32), 8, 1, 2)
+    assert (d.tolist(), src, mp, ml) == ([4, 4], "db", 3, 3)
