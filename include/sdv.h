@@ -115,14 +115,14 @@ int sdv_prefill_chunk(sdv_ctx *ctx, const int32_t *host_tokens, int n, int is_la
 int sdv_draft(sdv_ctx *ctx, int k, int32_t *host_draft, int *draft_len);
 
 /* Extra token database for the drafter (paper Sec. 5.1 (3), Sec. 5.5: the retrieval algorithm of
- * the baselines drafts "from both current context and an extra database").  Copies n host tokens
+ * the baselines searches the request context and an additional token corpus).  Copies n host tokens
  * (0 <= n <= max_seq; 0 removes the database) into the context; sdv_draft then searches them like
  * the request's text and copies the draft from wherever the longer suffix match ends (an equally
  * long match in the request's own text wins).  The database survives prefill and rollback.
  * Synchronises.  Errors: SDV_EINVAL (count, token range). */
 int sdv_set_database(sdv_ctx *ctx, const int32_t *host_tokens, int n);
 
-/* Verify step (paper Sec. 3.2 "verifies them in parallel", Sec. 4.4: x = [T, x_1..x_n],
+/* Verify step (paper Sec. 3.2: all drafts are checked in one parallel pass; Sec. 4.4: x = [T, x_1..x_n],
  * y = [y_1..y_{n+1}]): runs the decoder once over the pending token T and the drafts at
  * positions L..L+n, writing their KV rows speculatively, takes the greedy token y_{j+1} of
  * every row (lowest id wins ties) and the accept length a = number of leading x_i == y_i.

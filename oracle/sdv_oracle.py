@@ -215,8 +215,8 @@ class DraftExtension:
     """Reuse of rejected drafts (Sec. 4.4 "Reuse strategy"): one retained segment with a lifetime.
 
     The paper fixes: the segment is the solution of Eq. 3; it is appended to later drafts; it is
-    kept for at least one decoding step and dropped once its accumulated lifetime or the total
-    draft length exceeds a threshold (32 in Sec. 5.1).  Readings taken where it is silent:
+    kept for at least one decoding step and dropped when either its age or the length of the
+    whole draft passes a limit (32 in Sec. 5.1).  Readings taken where it is silent:
     * lifetime counts the verify steps the segment was appended to;
     * a draft that would grow beyond `max_total` with the segment drops the segment instead of
       cutting it;
