@@ -92,7 +92,20 @@ static inline float bf16_to_f32(uint16_t b) {
 DEF_MATMUL(matmul_mb16, 16)
 DEF_MATMUL(matmul_mb64, 64)
 
-/* y[m][n] = sum_k x[m][k] * w[n][k]  (+ bias[n]).  One accumulator per output, k ascending. */
+/* The definition written out: y[m][n] = sum_k x[m][k] * w[n][k]  (+ bias[n]), one accumulator per
+ * output, k ascending; no blocking, no transposition, no threads.  orc_matmul below must equal it
+ * bit for bit (tests/test_oracle_ops.py); it exists so that the arithmetic can be checked by eye. */
+void orc_matmul_plain(const float *x, const uint16_t *w, const float *bias, float *y, int M, int N, int K) {
+    for (int m = 0; m < M; ++m)
+        for (int n = 0; n < N; ++n) {
+            float acc = 0.0f;
+            for (int k = 0; k < K; ++k) acc += bf16_to_f32(w[(size_t)n * K + k]) * x[(size_t)m * K + k];
+            y[(size_t)m * N + n] = acc + (bias ? bias[n] : 0.0f);
+        }
+}
+
+/* The same sums as orc_matmul_plain, arranged for speed (the full-size workloads need it).
+ * y[m][n] = sum_k x[m][k] * w[n][k]  (+ bias[n]).  One accumulator per output, k ascending. */
 void orc_matmul(const float *x, const uint16_t *w, const float *bias, float *y, int M, int N, int K) {
     const int MB = M > 32 ? 64 : 16;
     const int Mp = (M + MB - 1) / MB * MB;
@@ -162,10 +175,6 @@ int orc_argmax(const float *x, int n) {
     for (int i = 0; i < n; ++i)
         if (x[i] > bv) { bv = x[i]; best = i; }
     return best;
-}
-
-size_t orc_kv_elems(const orc_config *c) {
-    return (size_t)c->n_layers * c->n_kv_heads * c->max_seq * c->head_dim;
 }
 
 /*

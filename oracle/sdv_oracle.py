@@ -77,6 +77,8 @@ def lib():
         L = C.CDLL(build())
         L.orc_matmul.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int]
         L.orc_matmul.restype = None
+        L.orc_matmul_plain.argtypes = L.orc_matmul.argtypes
+        L.orc_matmul_plain.restype = None
         L.orc_rmsnorm.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_int]
         L.orc_rmsnorm.restype = None
         L.orc_rope.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_float]
@@ -118,6 +120,19 @@ def matmul(x, w_bits, bias=None) -> np.ndarray:
     b = None if bias is None else _f32(bias)
     y = np.empty((M, N), dtype=np.float32)
     lib().orc_matmul(_p(x), _p(w_bits), _p(b), _p(y), M, N, K)
+    return y
+
+
+def matmul_plain(x, w_bits, bias=None) -> np.ndarray:
+    """The same product by the plain triple loop (the definition; slow)."""
+    x = _f32(x)
+    w_bits = np.ascontiguousarray(w_bits, dtype=np.uint16)
+    M, K = x.shape
+    N = w_bits.shape[0]
+    assert w_bits.shape[1] == K
+    b = None if bias is None else _f32(bias)
+    y = np.empty((M, N), dtype=np.float32)
+    lib().orc_matmul_plain(_p(x), _p(w_bits), _p(b), _p(y), M, N, K)
     return y
 
 
@@ -337,9 +352,24 @@ class StepRecord:
     margin: List[float] = field(default_factory=list)  # top-1 minus top-2 logit per row
 
 
+def top2(row: np.ndarray):
+    """The greedy choice of a logits row, the token that would replace it, and the gap between them.
+
+    Returns (best id, runner-up id, margin): best = the greedy token (largest value, lowest id among
+    equals); runner-up = the greedy token of the row with `best` removed; margin = their difference
+    (0.0 on an exact tie).  The parity tolerance forgives a flipped token only where this margin is
+    small, and then only towards this runner-up.
+    """
+    row = np.asarray(row)
+    best = argmax(row)
+    rest = np.array(row, dtype=np.float32, copy=True)
+    rest[best] = -np.inf
+    second = argmax(rest)
+    return best, second, float(row[best] - row[second])
+
+
 def top2_margin(row: np.ndarray) -> float:
-    part = np.partition(row, -2)[-2:]
-    return float(part[1] - part[0])
+    return top2(row)[2]
 
 
 def greedy_decode(model: OracleModel, context, gen: int, chunk: int):

@@ -6,6 +6,8 @@ from typing import List, Optional
 
 import numpy as np
 
+from oracle import sdv_oracle as O
+
 LOGIT_TOL = 0.05      # max |logit difference| allowed against the oracle
 COS_TOL = 0.999       # minimum cosine similarity per logits row
 MARGIN_TOL = 0.05     # below this top-2 margin of the oracle a different greedy token is legitimate
@@ -32,7 +34,7 @@ class RefStep:
 def steps_from_oracle(steps, from_drafter: bool) -> List[RefStep]:
     out = []
     for s in steps:
-        ru = [int(np.argsort(-s.logits[r], kind="stable")[1]) for r in range(len(s.draft) + 1)]
+        ru = [O.top2(s.logits[r])[1] for r in range(len(s.draft) + 1)]
         out.append(RefStep(s.kv_len_before, s.pending, list(s.draft), from_drafter, list(s.y), s.accept,
                            list(s.emitted), list(s.margin), ru, logits=s.logits))
     return out
@@ -104,3 +106,37 @@ def compare_step(sdv, step: RefStep, k: int, stats: dict, predrafted: bool = Fal
     sdv.debug_force_commit(len(step.emitted) - 1, step.emitted[-1])
     assert sdv.kv_len() == step.kv_len_before + len(step.emitted)
     return rows
+
+
+def compare_prefix_rows(sdv, step: RefStep, kp: int, stats: dict):
+    """Verifies only the first kp drafts of a forced-draft step and compares rows 0..kp with the stored
+    rows.  Under the linear-chain mask row j sees the cache and new rows 0..j only, so those rows do
+    not depend on the drafts behind them: the stored step fixes them for every shorter draft, and
+    the accept length is min(a, kp).  This reaches the launch shapes of shorter drafts (other
+    instruction widths and attention splits) at full size without another oracle run.  Nothing is
+    committed: the next verify overwrites the same KV rows."""
+    assert 0 < kp < len(step.draft)
+    y, a = sdv.verify(step.draft[:kp])
+    logits = sdv.get_logits(kp + 1)
+    flipped = None
+    for r in range(kp + 1):
+        if step.logits is not None:
+            ref, got = step.logits[r], logits[r]
+        else:
+            ids = np.concatenate([step.sample_ids, step.top_ids[r]])
+            ref = np.concatenate([step.logit_sample[r], step.top_vals[r]])
+            got = logits[r][ids]
+        err = float(np.abs(got - ref).max())
+        cos = float(np.dot(got, ref) / (np.linalg.norm(got) * np.linalg.norm(ref)))
+        stats["max_err"] = max(stats.get("max_err", 0.0), err)
+        stats["min_cos"] = min(stats.get("min_cos", 1.0), cos)
+        assert err <= LOGIT_TOL, f"{kp} drafts, row {r} at L={step.kv_len_before}: |dlogit| {err}"
+        assert cos >= COS_TOL, f"{kp} drafts, row {r} at L={step.kv_len_before}: cosine {cos}"
+        if int(y[r]) != step.y[r]:
+            assert step.margin[r] < MARGIN_TOL and int(y[r]) == step.runner_up[r], f"{kp} drafts, row {r}: token {y[r]}"
+            if flipped is None:
+                flipped = r
+    want = min(step.accept, kp)
+    if flipped is None or flipped > want:
+        assert a == want, f"{kp} drafts: accept length {a} vs {want} at L={step.kv_len_before}"
+    stats["prefix_checks"] = stats.get("prefix_checks", 0) + 1

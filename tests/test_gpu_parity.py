@@ -223,7 +223,34 @@ def test_full_size_workloads_against_stored_oracle_trajectory(name):
                 assert np.abs(got - ref[:, j]).max() <= 0.02 * np.abs(ref).max() + 1e-3
     s.debug_set_history(list(ctx) + [int(g["first_token"])], cfg.n_ctx)
     stats = {}
+    sweep = (1, 2, 4, 8)   # the draft lengths of the 7B-shaped sweep below its stored k = 16; 1, 2, 4 elsewhere
     for st in steps_from_golden(g):
+        if not st.from_drafter:
+            for kp in sweep:
+                if kp < len(st.draft):
+                    compare_prefix_rows(s, st, kp, stats)
         compare_step(s, st, int(g["k"]), stats)
-    print(name, stats.get("max_err"), stats.get("min_cos"), stats.get("near_tie_flips", 0))
+    print(name, stats.get("max_err"), stats.get("min_cos"), stats.get("near_tie_flips", 0), stats.get("prefix_checks", 0))
+    assert stats.get("prefix_checks", 0) >= 6
+    s.close()
+
+
+@pytest.mark.parametrize("name", ["tiny", "qwen0.5b", "qwen1.5b", "llama3b", "qwen7b"])
+def test_drafter_on_the_real_contexts_finds_what_the_oracle_finds(name):
+    """The n-gram drafter over each configuration's own context array at full length, on histories that
+    do end in a context trigram (after a random-init model's token the drafter finds nothing, so the
+    trajectories above only ever compare empty drafts): 200 seeded positions per configuration."""
+    cfg = get_config(name)
+    ctx = make_context(cfg)
+    s = Sdv(config_from(cfg))
+    rng = np.random.default_rng(77)
+    nonempty = 0
+    for p in rng.integers(0, cfg.n_ctx - 3, size=200).tolist():
+        hist = np.concatenate([ctx, ctx[p:p + 3]]).astype(np.int32)
+        s.debug_set_history(hist.tolist(), cfg.n_ctx)
+        want, mpos, mlen = O.ngram_draft(ctx, hist, cfg.ngram_n, cfg.ngram_min, cfg.k)
+        got = s.draft(cfg.k)
+        assert got == want.tolist(), (name, p)
+        nonempty += len(got) > 0
+    assert nonempty >= 190
     s.close()

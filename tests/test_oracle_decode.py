@@ -281,3 +281,32 @@ def test_paper_running_example_accepts_one_token():
     inv = {v: k for k, v in vocab.items()}
     assert a == int(fields["accepted_drafts"][0])
     assert [inv[t] for t in emitted] == fields["emitted"]
+
+
+@pytest.mark.parametrize("name", ["qwen1.5b", "llama3b", "qwen7b"])
+def test_stored_trajectories_are_self_consistent(name):
+    """The stored full-size trajectories (written by tests/golden/make_golden.py from the oracle
+    alone) obey what the method fixes: y is the greedy token of its row, the stored margin is the
+    gap to the runner-up, the accept length is the length of the matching prefix, the emitted
+    tokens are x_1..x_a, y_{a+1} (Sec. 4.4) and the KV length advances by the emitted count."""
+    g = np.load(os.path.join(GOLD, f"{name}.npz"))
+    S = len(g["accept"])
+    emitted_all = [int(g["first_token"])]
+    for i in range(S):
+        dl, a, ne = int(g["draft_len"][i]), int(g["accept"][i]), int(g["n_emitted"][i])
+        x, y = g["draft"][i, :dl].tolist(), g["y"][i, :dl + 1].tolist()
+        assert a == O.accept_len(x, y)
+        want = x[:a] + [y[a]]
+        assert g["emitted"][i, :ne].tolist() == want[:ne] and (ne == len(want) or i == S - 1)
+        if i + 1 < S:
+            assert int(g["kv_len_before"][i + 1]) == int(g["kv_len_before"][i]) + ne
+            assert int(g["pending"][i + 1]) == want[ne - 1]
+        for r in range(dl + 1):
+            ids, vals = g["top_ids"][i, r], g["top_vals"][i, r]
+            assert int(ids[0]) == y[r]
+            assert np.all(vals[:-1] >= vals[1:])
+            ties = vals[:-1] == vals[1:]
+            assert np.all(ids[:-1][ties] < ids[1:][ties])          # equal values: lower id first
+            assert float(g["margin"][i, r]) == float(vals[0] - vals[1])
+        emitted_all += want[:ne]
+    assert emitted_all == g["tokens"].tolist()[:len(emitted_all)]

@@ -30,6 +30,51 @@ def test_matmul_against_fp64_einsum(M, N, K):
     np.testing.assert_array_equal(O.matmul(e, wb)[M - 1], bf16_bits_to_f32(wb)[:, K - 2])
 
 
+@pytest.mark.parametrize("M,N,K", [(1, 5, 7), (9, 33, 64), (17, 21, 130), (33, 7, 96), (70, 19, 50), (3, 130, 257)])
+def test_fast_matmul_equals_the_plain_triple_loop_bit_for_bit(M, N, K):
+    """orc_matmul (blocked, transposed, threaded) against orc_matmul_plain (the definition as three
+    nested loops): the same sums in the same order, so not one bit may differ, bias included."""
+    x = (RNG.standard_normal((M, K)) * 3).astype(np.float32)
+    wb = _bf16(RNG.standard_normal((N, K)))
+    bias = RNG.standard_normal(N).astype(np.float32)
+    np.testing.assert_array_equal(O.matmul(x, wb, bias), O.matmul_plain(x, wb, bias))
+    np.testing.assert_array_equal(O.matmul(x, wb), O.matmul_plain(x, wb))
+
+
+def test_plain_matmul_against_hand_values():
+    # y[m][n] = sum_k x[m][k] w[n][k] + b[n], worked by hand
+    x = np.array([[1, 2, 3], [0, -1, 4]], dtype=np.float32)
+    w = np.array([[1, 0, 2], [0.5, 0.5, 0.5], [-1, 1, 0], [0, 0, 1]], dtype=np.float32)
+    b = np.array([10, 0, 0, -1], dtype=np.float32)
+    want = np.array([[17, 3, 1, 2], [18, 1.5, -1, 3]], dtype=np.float32)
+    np.testing.assert_array_equal(O.matmul_plain(x, _bf16(w), b), want)
+    np.testing.assert_array_equal(O.matmul(x, _bf16(w), b), want)
+
+
+def test_top2_margin_and_runner_up():
+    """The margin decides which flipped greedy tokens the parity tests forgive, the runner-up which
+    token they may flip to."""
+    # exact tie: margin 0, greedy = the lower id, runner-up = the other tied id
+    assert O.top2(np.array([1.0, 5.0, 5.0, 2.0], dtype=np.float32)) == (1, 2, 0.0)
+    # known gap, maximum at either end
+    assert O.top2(np.array([9.0, 1.0, 2.0, 8.5], dtype=np.float32)) == (0, 3, 0.5)
+    assert O.top2(np.array([-3.0, -7.0, -2.25, -2.0], dtype=np.float32)) == (3, 2, 0.25)
+    # three-way tie: the two lowest ids
+    assert O.top2(np.array([4.0, 4.0, 4.0], dtype=np.float32)) == (0, 1, 0.0)
+    assert O.top2_margin(np.array([0.0, 1.5], dtype=np.float32)) == 1.5
+    for _ in range(200):
+        n = int(RNG.integers(2, 300))
+        row = RNG.standard_normal(n).astype(np.float32)
+        if RNG.random() < 0.3:      # plant ties
+            row[RNG.integers(0, n, size=3)] = row.max()
+        best, second, margin = O.top2(row)
+        srt = sorted(row.tolist())
+        assert margin == np.float32(srt[-1]) - np.float32(srt[-2])
+        order = sorted(range(n), key=lambda i: (-row[i], i))     # value descending, id ascending
+        assert (best, second) == (order[0], order[1])
+        assert best == O.argmax(row)
+
+
 def test_matmul_rows_do_not_depend_on_batch():
     x = RNG.standard_normal((70, 96)).astype(np.float32)
     wb = _bf16(RNG.standard_normal((24, 96)))
