@@ -31,10 +31,13 @@ import numpy as np  # noqa: E402
 METRIC = "generated_tokens_per_sec"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of sdv_forward_kernel, as a multiple of the
-# algorithmic bytes: captured on the 0.5B-shaped workload (profiles/sdv_forward_kernel_qwen0.5b_ncu_full.md)
-# and scaled to the timed workload by its algorithmic bytes (traffic grows with the bytes streamed).
-# None once the kernel has changed since the capture.
+# algorithmic bytes: from an ncu capture on the 0.5B-shaped workload, scaled to the timed workload by its
+# algorithmic bytes (traffic grows with the bytes streamed).  None once the kernel has changed since the
+# capture.
 NCU_TRAFFIC_RATIO = 1.0051
+
+
+NOMINAL_HBM_GBS = 8000.0   # the "about 8 TB/s" the target is worded against
 
 
 def load_peaks():
@@ -47,26 +50,36 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi (read-only queries) while the timed regions
+    run.  Started before the warm-up so that even a short timed region has samples; samples taken while
+    the GPU was idle (before the first launch) are dropped by the caller's `mark()`."""
 
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    REASONS = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index = index
-        self.rows = []
-        self.proc = None
-        self.thread = None
+    def __init__(self, index: int, period_ms: int = 20):
+        self.index, self.period_ms = index, period_ms
+        self.rows, self.err, self.proc, self.thread, self.t_mark = [], "", None, None, None
+
+    def _fields(self, prefix):
+        return "clocks.sm,clocks.max.sm,power.draw," + ",".join(f"{prefix}.{r}" for r in self.REASONS)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
-                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except OSError:
-            self.proc = None
+        for prefix in ("clocks_event_reasons", "clocks_throttle_reasons"):   # older drivers know the second name only
+            try:
+                probe = subprocess.run(["nvidia-smi", f"--query-gpu={self._fields(prefix)}", "--format=csv,noheader,nounits",
+                                        "-i", str(self.index)], capture_output=True, text=True, timeout=20)
+            except (OSError, subprocess.TimeoutExpired) as e:
+                self.err = str(e)
+                return
+            if probe.returncode == 0 and "not a valid field" not in probe.stdout.lower():
+                break
+            self.err = (probe.stderr or probe.stdout).strip()[:200]
+        else:
             return
+        self.err = ""
+        self.proc = subprocess.Popen(
+            ["nvidia-smi", f"--query-gpu={self._fields(prefix)}", "--format=csv,noheader,nounits", "-lms",
+             str(self.period_ms), "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True)
         self.thread = threading.Thread(target=self._read, daemon=True)
         self.thread.start()
 
@@ -74,28 +87,43 @@ class ClockSampler:
         for line in self.proc.stdout:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) >= 7:
-                self.rows.append(parts)
+                self.rows.append((time.perf_counter(), parts))
+
+    def mark(self):
+        """Samples from here on count (the GPU is under load from now)."""
+        self.t_mark = time.perf_counter()
 
     def stop(self):
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"], "samples": 0,
+                    "error": self.err}
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
-        for r in self.rows:
+        for t, r in self.rows:
+            if self.t_mark is not None and t < self.t_mark:
+                continue
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
             except ValueError:
                 continue
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+            for name, v in zip(self.REASONS, r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "period_ms": self.period_ms}
+
+
+def workload_string(cfg, k):
+    """Names the workload; the GPU arm and the CPU reference arm print the same string."""
+    return (f"{cfg.name}: {cfg.n_layers} layers d={cfg.d_model} {cfg.n_q_heads}q/{cfg.n_kv_heads}kv "
+            f"hd={cfg.head_dim} ffn={cfg.d_ffn} vocab={cfg.vocab}; context {cfg.n_ctx} Zipf tokens "
+            f"with planted repeats prefilled in {cfg.chunk}-token chunks; k={k} (n-gram drafter, "
+            f"context search); verify steps of {k + 1} rows from KV length {cfg.n_ctx}")
 
 
 def oracle_steps_per_sec(cfg, weights, ctx, n_prefill, n_steps, k):
@@ -138,6 +166,21 @@ def aggregate_over_ranks(times_ms, counts, world, device):
     return t.tolist(), c.tolist()
 
 
+def oracle_prefill_tokens(cfg):
+    """Context tokens the CPU oracle prefills before its timed steps: the whole context where that takes the
+    host cores tens of seconds (the workloads up to the 1.5B shape), else the first chunk only."""
+    return cfg.n_ctx if cfg.linear_params() * cfg.n_ctx <= 4.0e12 else min(cfg.chunk, cfg.n_ctx)
+
+
+def oracle_sample_string(cfg, k, n_steps, n_prefill, ms_per_step=None):
+    txt = f"{n_steps} verify steps of {k + 1} rows from KV length {n_prefill}"
+    if n_prefill != cfg.n_ctx:
+        txt += f" (the oracle prefilled only the first {n_prefill} of {cfg.n_ctx} context tokens)"
+    if ms_per_step is not None:
+        txt += f"; {ms_per_step:.1f} ms per step"
+    return txt + "; oracle prefill not timed"
+
+
 def run_reference(args, cfg):
     from sdv_inputs import make_context, make_weights
     rank = int(os.environ.get("RANK", "0"))
@@ -146,20 +189,68 @@ def run_reference(args, cfg):
     cores = len(os.sched_getaffinity(0))
     w = make_weights(cfg, threads=max(8, cores))
     ctx = make_context(cfg)
-    n_prefill = min(cfg.chunk, cfg.n_ctx)
+    n_prefill = oracle_prefill_tokens(cfg)
     total = args.warmup + args.steps
     tps, s_per_step, emitted = oracle_steps_per_sec(cfg, w, ctx, n_prefill, total, cfg.k)
-    sample = (f"{total} verify steps of {cfg.k + 1} rows after prefilling the first {n_prefill} context tokens "
-              f"(KV length {n_prefill}+, not {cfg.n_ctx}+)")
+    sample = oracle_sample_string(cfg, cfg.k, total, n_prefill, s_per_step * 1e3)
     line = {
         "impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": s_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{cfg.name}: {cfg.n_layers} layers d={cfg.d_model}, k={cfg.k}", "sample": sample},
+        "config": {"workload": workload_string(cfg, cfg.k), "rows_per_verify": cfg.k + 1, "sample": sample,
+                   "same_state_as_gpu_arm": n_prefill == cfg.n_ctx},
         "cpu_baseline": {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
+
+
+def phase_timeline(s, cfg, k):
+    """One profiled verify step: the kernel's own per-phase, per-block timestamps (%globaltimer) as a
+    table.  dur = first block in to last block out; gap = grid barrier to the next phase."""
+    names = ["QKV projection", "attention", "output projection", "gate|up + SwiGLU + down"]
+    nph = 2 + 4 * cfg.n_layers
+    s.debug_profile(True)
+    s.draft(k, fetch=False)
+    s.verify(None, fetch=False)
+    s.commit()
+    prof_us = s.last_verify_ms() * 1e3
+    p = s.debug_profile(False, nph).astype(np.int64)
+    st, en = p[:, :, 0], p[:, :, 1]
+    rows = {}
+    for ph in range(nph):
+        m = en[ph] > 0
+        a, d = st[ph][m].min(), en[ph][m].max()
+        nxt = st[ph + 1][en[ph + 1] > 0].min() if ph + 1 < nph else d
+        nm = "embedding" if ph == 0 else ("LM head + argmax" if ph == nph - 1 else names[(ph - 1) % 4])
+        r = rows.setdefault(nm, {"dur": [], "gap": [], "marks": []})
+        r["dur"].append((d - a) / 1e3)
+        r["gap"].append((nxt - d) / 1e3)
+        marks = []
+        for wd in (2, 3, 4, 5, 6):       # per-role timestamps inside the phase, relative to its start
+            x = p[ph][:, wd]
+            mm = (x > 0) & m
+            marks.append((float((x[mm].min() - a) / 1e3), float((x[mm].max() - a) / 1e3)) if mm.any() else None)
+        r["marks"].append(marks)
+    out = [f"verify step of {k + 1} rows, KV length {s.kv_len()}, {cfg.name}: {prof_us:.1f} us with the per-phase stamps on",
+           "", "| phase | launches of it | dur us (mean) | gap us (mean) | marks inside the phase, us after its start: first block / last block |",
+           "|---|---|---|---|---|"]
+    legend = {"attention": ["loads issued", "Q tile and new rows ready", "first key block in place", "key loop done", "unit done"],
+              "default": ["token operand built", "tensor-core warp done issuing", "epilogue done", "reached the down projection",
+                          "SwiGLU operand complete"]}
+    total = 0.0
+    for nm, r in rows.items():
+        lg = legend.get(nm, legend["default"])
+        mk = []
+        for i, name in enumerate(lg):
+            vals = [x[i] for x in r["marks"] if x[i] is not None]
+            if vals:
+                mk.append(f"{name} {np.mean([v[0] for v in vals]):.1f} / {np.mean([v[1] for v in vals]):.1f}")
+        total += sum(r["dur"]) + sum(r["gap"])
+        out.append(f"| {nm} | {len(r['dur'])} | {np.mean(r['dur']):.2f} | {np.mean(r['gap']):.2f} | {'; '.join(mk)} |")
+    out.append("")
+    out.append(f"sum of dur + gap over all phases: {total:.1f} us")
+    return "\n".join(out)
 
 
 def main():
@@ -177,6 +268,9 @@ def main():
                     help="adds a third timed loop with draft extension (Sec. 4.4): drafts grow to at most MAX_TOTAL "
                          "tokens by reuse of rejected drafts; reported under \"extension\"")
     ap.add_argument("--extension-life", type=int, default=32)
+    ap.add_argument("--phase-timeline", action="store_true",
+                    help="prints the per-phase timeline of one profiled verify step (a table) instead of the JSON line")
+    ap.add_argument("--no-extras", action="store_true", help="skips the history-search and forced-acceptance loops")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -204,9 +298,16 @@ def main():
     sweep = [int(x) for x in args.sweep_k.split(",") if x.strip()]
     k_max = max([k] + sweep + [args.extension])
     total = args.warmup + args.steps
+    extras = not args.no_extras and not args.phase_timeline and world == 1
     max_seq = cfg.n_ctx + 2 * total * (k + 1) + 64          # room for two timed loops at full acceptance
     if args.extension:
         max_seq += total * (args.extension + 1)
+    # forced acceptance: seeded accept lengths whose mean number of emitted tokens per step lies in the range
+    # the paper reports for its 1.5B model (Table "ablation on accept length": 2.5 to 5.5 tokens per step)
+    rng = np.random.default_rng(20251015)
+    forced_a = [int(x) for x in np.minimum(rng.geometric(1.0 / 3.6, size=total) - 1, k)] if extras else []
+    stream_len = sum(forced_a) + len(forced_a) + k + 2 if extras else 0
+    max_seq = max(max_seq, cfg.n_ctx + stream_len + 2 * (k + 2) + 64)
     cores = len(os.sched_getaffinity(0))
     w = make_weights(cfg, threads=max(8, cores // max(1, world)))
     ctx = make_context(cfg)
@@ -251,21 +352,31 @@ def main():
             kms.append(s.last_verify_ms())
         return tokens, kms
 
+    if args.phase_timeline:
+        loop(max(args.warmup, 25), False)
+        if rank == 0:
+            print(phase_timeline(s, cfg, k), flush=True)
+        s.close()
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
     # ---- device-resident loop
-    loop(args.warmup, False)
     sampler = ClockSampler(local)
+    sampler.start()                      # before the warm-up: the first samples arrive while it runs
+    loop(args.warmup, False)
     launches0 = s.launch_count()
     barrier()
-    sampler.start()
+    sampler.mark()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record(stream)
     tokens, kms = loop(args.steps, False)
     ev1.record(stream)
     barrier()
-    clocks = sampler.stop()
     launches = s.launch_count() - launches0
     ms_total = ev0.elapsed_time(ev1)
-    L_mid = (L0 + s.kv_len()) // 2
+    kv_end = s.kv_len()
+    L_mid = (L0 + kv_end) // 2
 
     # ---- end-to-end loop with host buffers
     loop(args.warmup, True)
@@ -276,6 +387,7 @@ def main():
     e1.record(stream)
     barrier()
     ms_e2e = e0.elapsed_time(e1)
+    clocks = sampler.stop()              # sampled over both timed loops (and the warm-up between them)
 
     # ---- optional: device-resident loop with draft extension (every step computes MAX_TOTAL + 1 rows)
     ext = None
@@ -304,6 +416,63 @@ def main():
                "verify_kernel_us": statistics.mean(kms_x) * 1e3,
                "accepted_drafts_per_step": tokens_x / args.steps - 1.0, "scope": "rank 0"}
 
+    # ---- the two other labelled throughput numbers (single-GPU runs only; synthetic acceptance)
+    forced = hist_mode = None
+    if extras and world == 1:
+        # (C) forced acceptance.  The greedy continuation comes from this path's own plain decoding (one token
+        # per step, no oracle involved), recorded before the timed region; each timed step then verifies a
+        # draft that agrees with it for a seeded number of tokens and is wrong right after.
+        s.rollback(L0)
+        greedy = []
+        while len(greedy) < stream_len:
+            s.verify([], fetch=False)
+            em, _ = s.commit()
+            greedy += em
+        s.rollback(L0)
+
+        def forced_loop(steps_a, pos):
+            toks, kms_f, hits = 0, [], 0
+            for a_t in steps_a:
+                d = greedy[pos:pos + a_t] + [(greedy[pos + a_t] + 1) % cfg.vocab] * (k - a_t)
+                s.verify(d[:k], fetch=False)
+                em, _ = s.commit()
+                hits += int(len(em) == a_t + 1)
+                toks += len(em)
+                pos += len(em)
+                kms_f.append(s.last_verify_ms())
+            return toks, kms_f, pos, hits
+        _, _, pos, _ = forced_loop(forced_a[:args.warmup], 0)
+        torch.cuda.synchronize()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        toks_f, kms_f, pos, hits = forced_loop(forced_a[args.warmup:], pos)
+        f1.record(stream)
+        torch.cuda.synchronize()
+        ms_f = f0.elapsed_time(f1)
+        forced = {"label": "synthetic: drafts forced to agree with the model's own greedy continuation for a seeded "
+                           "number of tokens (geometric, mean emitted 3.6 per step, the range of the paper's accept-length "
+                           "table for its 1.5B model); random-init weights accept nothing on their own",
+                  "value": toks_f / (ms_f * 1e-3), "unit": UNIT, "ms_per_step": ms_f / args.steps,
+                  "emitted_per_step": toks_f / args.steps, "steps_with_the_forced_accept_length": hits,
+                  "verify_kernel_us": statistics.mean(kms_f) * 1e3}
+        # (B) the drafter also searches the generated tokens (search_history): a second context of the same model
+        s.close()
+        s = Sdv(config_from(cfg, k_max=k_max, max_seq=max_seq, search_history=True), stream=stream)
+        s.load_weights(w)
+        for i in range(0, cfg.n_ctx, cfg.chunk):
+            s.prefill_chunk(ctx[i:i + cfg.chunk], is_last=(i + cfg.chunk >= cfg.n_ctx))
+        loop(args.warmup, False)
+        torch.cuda.synchronize()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record(stream)
+        toks_h, kms_h = loop(args.steps, False)
+        h1.record(stream)
+        torch.cuda.synchronize()
+        ms_h = h0.elapsed_time(h1)
+        hist_mode = {"label": "drafter searches the request context and the generated tokens (search_history)",
+                     "value": toks_h / (ms_h * 1e-3), "unit": UNIT, "ms_per_step": ms_h / args.steps,
+                     "emitted_per_step": toks_h / args.steps, "verify_kernel_us": statistics.mean(kms_h) * 1e3}
+
     (ms_total, ms_e2e), (tokens_all, tokens_e_all) = aggregate_over_ranks([ms_total, ms_e2e], [tokens, tokens_e], world,
                                                                           "cuda")
 
@@ -317,18 +486,16 @@ def main():
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {
-                "workload": (f"{cfg.name}: {cfg.n_layers} layers d={cfg.d_model} {cfg.n_q_heads}q/{cfg.n_kv_heads}kv "
-                             f"hd={cfg.head_dim} ffn={cfg.d_ffn} vocab={cfg.vocab}; context {cfg.n_ctx} Zipf tokens "
-                             f"with planted repeats prefilled in {cfg.chunk}-token chunks; k={k} (n-gram drafter, "
-                             f"context search); KV length {L0}..{s.kv_len()}"),
-                "rows_per_verify": k + 1, "replicas": world,
+                "workload": workload_string(cfg, k),
+                "rows_per_verify": k + 1, "replicas": world, "kv_len_range": [L0, kv_end],
                 "l2": "inputs larger than L2: every step streams all weights (>= 1 GB) once",
                 "accepted_drafts_per_step": tokens_all / (args.steps * world) - 1.0,
             },
             "verify_kernel_us": kernel_ms * 1e3,
             "verify_kernel_us_p10_p90": [float(np.percentile(kms, 10)) * 1e3, float(np.percentile(kms, 90)) * 1e3],
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_kind": f"of {peak_kind}", "bytes_per_launch": wbytes + kvbytes,
+                         "peak_kind": f"of {peak_kind}", "frac_nominal": achieved / NOMINAL_HBM_GBS,
+                         "nominal_peak": NOMINAL_HBM_GBS, "bytes_per_launch": wbytes + kvbytes,
                          "traffic": None if NCU_TRAFFIC_RATIO is None else (wbytes + kvbytes) * NCU_TRAFFIC_RATIO,
                          "traffic_source": "ncu capture on the 0.5B-shaped workload, scaled by algorithmic bytes",
                          "kernel": "sdv_forward_kernel"},
@@ -337,6 +504,13 @@ def main():
             "gpu_launches": launches,
             "clocks": clocks,
         }
+        line["config"]["tokens_per_sec_variants"] = ("value: n-gram drafter over the request context (accepts ~0 with "
+                                                     "random-init weights); history: search_history drafter; "
+                                                     "forced_acceptance: synthetic accept lengths")
+        if forced:
+            line["forced_acceptance"] = forced
+        if hist_mode:
+            line["history"] = hist_mode
         if ext:
             line["extension"] = ext
         if sweep:
@@ -347,13 +521,12 @@ def main():
                 line["k_sweep"].append({"k": kk, "kv_len": L0, "verify_kernel_us": sweep_ms[kk] * 1e3, "GB/s": gbs,
                                         "frac": gbs / peak})
         if world == 1 and not args.no_cpu_baseline:
-            n_prefill = min(cfg.chunk, cfg.n_ctx)
+            n_prefill = oracle_prefill_tokens(cfg)
             n_steps = 48 if cfg.linear_params() < 1.0e9 else (24 if cfg.linear_params() < 4.0e9 else 8)
             tps, sps, _ = oracle_steps_per_sec(cfg, w, ctx, n_prefill, n_steps, k)
             line["cpu_baseline"] = {
                 "value": tps, "unit": UNIT, "cores": cores, "kind": "oracle",
-                "sample": (f"{n_steps} verify steps of {k + 1} rows after prefilling the first {n_prefill} context "
-                           f"tokens; {sps * 1e3:.1f} ms per step"),
+                "sample": oracle_sample_string(cfg, k, n_steps, n_prefill, sps * 1e3),
             }
         print(json.dumps(line), flush=True)
     s.close()

@@ -97,7 +97,7 @@ int sdv_create(const sdv_config *cfg, void *dev_workspace, size_t bytes, void *c
  * Synchronises the stream.  May be called again to replace the weights. */
 int sdv_load_weights(sdv_ctx *ctx, const sdv_weights *w);
 
-/* Chunked prefill (paper Sec. 4.1 "the prompt is split into fixed-size chunks", Sec. 4.2 graph
+/* Chunked prefill (paper Sec. 4.1: the prompt is cut into chunks of one fixed size; Sec. 4.2: graph
  * equivalence): appends n context tokens (host int32, each in [0, vocab)) to the history, runs
  * the decoder over them at positions L..L+n-1 and advances L by n.  Chunks of any length n >= 1
  * give the same cache as one long call.  With is_last != 0 the logits of the last token are
@@ -163,8 +163,10 @@ int sdv_extension_update(sdv_ctx *ctx, int max_life, int32_t *host_segment, int 
  * Errors: SDV_ESTATE when no verify result is outstanding. */
 int sdv_commit(sdv_ctx *ctx, int max_emit, int32_t *host_emitted, int *n_emitted, int *kv_len);
 
-/* Sets L to new_kv_len (1 <= new_kv_len <= current L): the history is cut to new_kv_len + 1
- * tokens and its last token becomes the pending token again. */
+/* KV rollback (paper Sec. 3.2: everything behind the first mismatch is thrown away and computed
+ * again; the cache rows stay where they are, only the committed length moves).  Sets L to
+ * new_kv_len (1 <= new_kv_len <= current L): the history is cut to new_kv_len + 1 tokens and its
+ * last token becomes the pending token again.  Errors: SDV_ESTATE before prefill, SDV_EINVAL. */
 int sdv_rollback(sdv_ctx *ctx, int new_kv_len);
 
 /* Current committed KV length L, or a negative error code. */
@@ -270,7 +272,11 @@ int sdv_last_verify_ms(sdv_ctx *ctx, float *ms);
  * streams.
  *
  * All three buffers are DEVICE pointers on the current device and stay owned by the caller:
- * dev_x fp32 [M][K], dev_w bf16 bits [N][K] row-major, dev_y fp32 [M][N] (overwritten).
+ * dev_x fp32 [M][K], dev_w bf16 bits [N][K] row-major, dev_y fp32 [M][N] (overwritten).  dev_x and
+ * dev_w are read with 16-byte vector loads and must be 16-byte aligned, dev_y 4-byte aligned (a
+ * view into a larger tensor that starts at an odd element offset is not); a misaligned pointer
+ * returns SDV_EINVAL before anything runs.  Where the runtime can tell, a pointer that is not device
+ * memory of the current device is refused the same way.
  * cuda_stream is a cudaStream_t (NULL = the default stream); the work is queued on it and the
  * call returns after it has finished (it synchronises that stream).
  *

@@ -340,7 +340,9 @@ def gemm_noalloc(x, w_bits, y, stream=None) -> int:
     """y[M][N] = x[M][K] * w[N][K]^T on device tensors, through the entry point that allocates no
     memory.  x: CUDA float32 [M][K]; w_bits: CUDA tensor of bf16 values (dtype bfloat16, or their
     bits as int16 / uint16) [N][K]; y: CUDA float32 [M][N], overwritten.  All contiguous and on the
-    current device.  Returns the library's status code (OK, ETOOBIG, ...): marshalling only."""
+    current device; x and w_bits must start on a 16-byte boundary (a view such as x[1:] of a tensor
+    with an odd row length does not: the library then returns EINVAL and runs nothing).  Returns the
+    library's status code (OK, EINVAL, ETOOBIG, ...): marshalling only."""
     import torch
     for t in (x, w_bits, y):
         if not (t.is_cuda and t.is_contiguous()):

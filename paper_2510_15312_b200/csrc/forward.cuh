@@ -3,17 +3,19 @@
 //
 // One thread block per SM, 12 warps:
 //   warp 11      weight streamer: walks the block's static share of every GEMM in launch order
-//                and keeps a ring of 16 KB shared-memory stages full with bulk asynchronous copies.
+//                and keeps a ring of 32 KB shared-memory stages full with bulk asynchronous copies.
 //                It never waits for activations or grid barriers, only for free ring slots, so HBM
 //                traffic continues across operation boundaries.
-//   warp 10      its lane 0 issues the tensor-core instructions (tcgen05.mma, M = 128 weight rows
-//                x N = 16 or 32 token rows x K = 16 per instruction): the streamed stage is the A
+//   warp 10      one elected lane issues the tensor-core instructions (tcgen05.mma, M = 128 weight
+//                rows x N = 16 or 32 token rows x K = 16 per instruction): the streamed stage is the A
 //                operand, the token rows, resident in shared memory for the whole operation, the
-//                B operand; accumulators live in tensor memory (two buffers, so the next pass
-//                starts while the previous one is read out).
-//   warps 0..3   read the accumulators back (tcgen05.ld) and run the fused epilogues.
-//   warps 0..10  together build the token operand at the start of an operation (RMSNorm scale,
-//                merge of the split-KV partial results, ...) and run the attention step.
+//                B operand; accumulators live in tensor memory (two buffers of two 128-row
+//                accumulators, so the next pass starts while the previous one is read out).
+//   warps 0..7   read the accumulators back (tcgen05.ld) and run the fused epilogues: warps 0..3 the
+//                first accumulator of a pass, warps 4..7 the second (or, for passes of up to 128
+//                rows, alternate pairs of token columns of the one accumulator).
+//   warps 0..9   build the token operand at the start of an operation (RMSNorm scale, merge of the
+//                split-KV partial results, ...); warps 0..10 run the attention step.
 // A layer is four operations separated by a bounded grid barrier: QKV projection; attention;
 // output projection (+ residual); gate|up with SwiGLU followed, inside the same block and without
 // a barrier, by the slice of the down projection (+ residual) that consumes this block's SwiGLU
@@ -77,13 +79,13 @@ static_assert(sizeof(Misc) <= kMiscSmemBytes, "misc shared memory");
 // Grid barrier: every block adds one to a counter (release) and waits (bounded, acquire) until all
 // have.  Called by all worker threads.  Returns, identically for all of them, whether some bounded
 // wait in this block has been abandoned (the remaining phases then do no work).
-__device__ __forceinline__ bool grid_barrier(const FwdParams& P, int target, Misc* misc, int wtid) {
+__device__ __forceinline__ bool grid_barrier(const FwdParams& P, unsigned target, Misc* misc, int wtid) {
     named_bar_sync(1, kWorkerThreads);
     if (wtid == 0) {
-        red_release_add_s32(P.bar, 1);  // no return value to wait for: polling starts at once
+        red_release_add_u32(P.bar, 1u);  // no return value to wait for: polling starts at once
         uint64_t t0 = 0;  // the global timer is slow to read: only once the wait has lasted a while
         uint32_t spins = 0;
-        while ((int)(ld_acquire_gpu(P.bar) - target) < 0) {
+        while ((int)(ld_acquire_gpu_u32(P.bar) - target) < 0) {  // wrap-safe: the difference, read as signed
             if ((++spins & 63u) == 0) {
                 if (*(volatile int*)&misc->abort_flag) break;
                 const uint64_t now = global_timer_ns();
@@ -361,13 +363,8 @@ __device__ __forceinline__ void mma_op(const FwdParams& P, const Part& pt, uint8
 }
 
 // ------------------------------------------------------------------------------------------
-// Epilogues (warps 0..3).  Thread t = 32 * warp + lane owns accumulator row t of the pass, i.e.
-// weight row 16 * tile_base + t, for all token columns.
-struct ArgBest {
-    float v[kMaxRows];
-    int i[kMaxRows];
-};
-
+// Epilogues (warps 0..7).  Thread t = 32 * (warp & 3) + lane owns row t of its 128-row accumulator,
+// i.e. one weight row (output feature), for the token columns its warp group takes.
 template <int NBT>  // token columns read: 16 or 32
 __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op, int layer, const Part& pt, uint8_t* act, Misc* misc,
                                             PipePos& pos, bool& dead, int warp, int lane, float (&bv)[NBT], int (&bi)[NBT]) {
@@ -1050,7 +1047,7 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
         }
         if (ph + 1 < P.ph_end) {
             ++nbar;
-            skip = grid_barrier(P, P.bar_base + nbar * P.G, misc, wtid);
+            skip = grid_barrier(P, P.bar_base + (unsigned)(nbar * P.G), misc, wtid);
         }
     }
     // all tensor-core work must have completed before tensor memory is returned

@@ -196,7 +196,7 @@ struct FwdParams {
     int raw_N, raw_K;
     int* state;
     const int* hist;
-    int* bar;          // grid barrier counter
+    unsigned* bar;     // grid barrier counter (wraps round; only differences are compared)
     unsigned long long* prof;  // optional [phase][block][kProfWords] timestamps (ns)
     // per launch
     int L;             // committed KV length = position of row 0
@@ -205,7 +205,7 @@ struct FwdParams {
     int att_gh;        // attention split: query heads per unit (the key ranges follow from it)
     int mode;          // 0: rows are [pending, draft...]; 1: rows are hist[L..L+M)
     int ph_begin, ph_end;
-    int bar_base;      // barrier counter value before this launch
+    unsigned bar_base; // barrier counter value before this launch
     int store_logits;
     // shared-memory plan of this launch (bytes from the 1024-aligned base)
     int nstage;        // ring slots of kStageBytes, at offset 0

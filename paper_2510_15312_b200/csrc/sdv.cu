@@ -248,7 +248,7 @@ struct sdv_ctx {
     bool prefill_done, weights_loaded, verified, draft_pending;
     int draft_k;    // k of the pending sdv_draft
     int last_rows;  // rows of the last verify
-    int bar_base;
+    unsigned bar_base;  // grid-barrier counter value before the next launch (wraps; only differences are used)
     int parity;
     int profile;
     int last_cuda;
@@ -333,7 +333,7 @@ int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph
     P.store_logits = ctx->parity;
     P.prof = ctx->profile ? (unsigned long long*)(ctx->ws + ctx->r.prof) : nullptr;
     const int nbar = ph_end - ph_begin - 1;
-    ctx->bar_base += nbar * ctx->G;
+    ctx->bar_base += (unsigned)(nbar * ctx->G);
     if (timed) CK(cudaEventRecord(ctx->ev0, ctx->stream));
     cudaError_t e = launch_kernel(P, smem_bytes, ctx->stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
@@ -443,13 +443,18 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
     if (sms > kMaxGrid) sms = kMaxGrid;
     ctx->G = sms;  // one persistent block per SM
     ctx->r = carve(cfg);
+    // every failure below leaves through this: what was created so far is released
+    auto fail = [&](int code) {
+        if (ctx->pinned) cudaFreeHost(ctx->pinned);
+        if (ctx->ev0) cudaEventDestroy(ctx->ev0);
+        if (ctx->ev1) cudaEventDestroy(ctx->ev1);
+        delete ctx;
+        return code;
+    };
     e = cudaHostAlloc((void**)&ctx->pinned, 4096, cudaHostAllocDefault);
     if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev0);
     if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev1);
-    if (e != cudaSuccess) {
-        delete ctx;
-        return SDV_ECUDA;
-    }
+    if (e != cudaSuccess) return fail(SDV_ECUDA);
 
     const int d = cfg->d_model, f = cfg->d_ffn, hd = cfg->head_dim;
     const int nq = cfg->n_q_heads * hd, nkv = cfg->n_kv_heads * hd, nqkv = nq + 2 * nkv;
@@ -486,17 +491,13 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
     P.raw_K = 0;
     P.state = (int*)(ws + ctx->r.state);
     P.hist = (const int*)(ws + ctx->r.hist);
-    P.bar = (int*)(ws + ctx->r.bar);
+    P.bar = (unsigned*)(ws + ctx->r.bar);
     P.wait_limit_ns = 2000000000ull;
     {
         // the widest verify step must fit the shared-memory plan
         FwdParams probe = P;
         int smem_bytes = 0;
-        if (!apply_plan(probe, rows_max, false, &smem_bytes)) {
-            cudaFreeHost(ctx->pinned);
-            delete ctx;
-            return SDV_EINVAL;
-        }
+        if (!apply_plan(probe, rows_max, false, &smem_bytes)) return fail(SDV_EINVAL);
     }
 
     // rotary table in double, rounded once to fp32
@@ -526,11 +527,7 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
         e = cudaGetLastError();
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
-    if (e != cudaSuccess) {
-        cudaFreeHost(ctx->pinned);
-        delete ctx;
-        return SDV_ECUDA;
-    }
+    if (e != cudaSuccess) return fail(SDV_ECUDA);
     *out = ctx;
     return SDV_OK;
 }
@@ -1100,9 +1097,24 @@ int sdv_gemm_noalloc(const float* dev_x, const uint16_t* dev_w, float* dev_y, in
     if (!dev_x || !dev_w || !dev_y) return SDV_EINVAL;
     if (M < 1 || N < 16 || N % 16 || K < 64 || K % 64) return SDV_EINVAL;
     if (M > kMaxRows || N > kNaMaxN || K > kNaMaxK || (size_t)N * K * 2 > kNaWeightBytes) return SDV_ETOOBIG;
+    // the kernels read x and w with 16-byte vector loads
+    if ((((uintptr_t)dev_x | (uintptr_t)dev_w) & 15) || ((uintptr_t)dev_y & 3)) return SDV_EINVAL;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNaMaxDevices) return SDV_ECUDA;
+    {
+        // host memory or another device's memory would fault inside the kernel: refuse it here
+        const void* ptrs[3] = {dev_x, dev_w, dev_y};
+        for (int i = 0; i < 3; ++i) {
+            cudaPointerAttributes at;
+            if (cudaPointerGetAttributes(&at, ptrs[i]) != cudaSuccess) {
+                cudaGetLastError();
+                return SDV_EINVAL;
+            }
+            if (at.type == cudaMemoryTypeManaged) continue;
+            if (at.type != cudaMemoryTypeDevice || at.device != dev) return SDV_EINVAL;
+        }
+    }
     if (!g_na_ptr[dev]) {
         // first call on this device: look the array's device address up (do this before any stream capture)
         void* p = nullptr;
@@ -1127,7 +1139,7 @@ int sdv_gemm_noalloc(const float* dev_x, const uint16_t* dev_w, float* dev_y, in
     P.raw_N = N;
     P.raw_K = K;
     P.state = (int*)(sc + kNaStateOff);
-    P.bar = P.state + 200;  // unused by a one-phase launch, kept inside the cleared words
+    P.bar = (unsigned*)(P.state + 200);  // unused by a one-phase launch, kept inside the cleared words
     P.mode = 1;
     P.ph_begin = 2;  // with n_layers = 0 phase 2 is the stand-alone GEMM
     P.ph_end = 3;

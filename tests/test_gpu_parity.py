@@ -10,7 +10,7 @@ import pytest
 from oracle import sdv_oracle as O
 from sdv_inputs import get_config, make_context, make_weights
 from paper_2510_15312_b200.binding import Sdv, config_from
-from helpers import LOGIT_TOL, MARGIN_TOL, compare_step, steps_from_golden, steps_from_oracle
+from helpers import LOGIT_TOL, MARGIN_TOL, compare_prefix_rows, compare_step, steps_from_golden, steps_from_oracle
 
 pytestmark = pytest.mark.gpu
 GOLD = os.path.join(os.path.dirname(__file__), "golden")

@@ -1,10 +1,12 @@
-"""The GEMM entry point that allocates nothing, against the context-based one (same kernel, scratch
-from the context's workspace).  Named so that it is collected after every other test file: it must
-pass on a GPU that earlier tests have already used, and on its own."""
+"""The GEMM entry point that allocates nothing, against the oracle's matmul and against the
+context-based entry point (same kernel, scratch from the context's workspace).  Named so that it is
+collected after every other test file: it must pass on a GPU that earlier tests have already used,
+and on its own."""
 import numpy as np
 import pytest
 
-from sdv_inputs import f32_to_bf16_bits, get_config
+from oracle import sdv_oracle as O
+from sdv_inputs import bf16_bits_to_f32, f32_to_bf16_bits, get_config
 import paper_2510_15312_b200 as pkg
 from paper_2510_15312_b200.binding import Sdv, config_from
 
@@ -30,11 +32,20 @@ def test_noalloc_gemm_matches_context_gemm_twice_in_a_row():
             dx = torch.from_numpy(x).cuda()
             dw = torch.from_numpy(wb.view(np.int16)).cuda()
             dy = torch.full((M, N), float("nan"), device="cuda")
-            before = torch.cuda.memory_allocated()
+            if seed == 0:
+                assert pkg.gemm_noalloc(dx, dw, dy) == pkg.OK   # first call: module load and the symbol look-up
+            torch.cuda.synchronize()
+            before, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
             rc = pkg.gemm_noalloc(dx, dw, dy)
             assert rc == pkg.OK
+            # neither torch's allocator nor the driver handed out memory during the call
             assert torch.cuda.memory_allocated() == before
+            assert torch.cuda.mem_get_info()[0] == free_before
             y = dy.cpu().numpy()
+            # the oracle's product of the same operands: x is rounded to bf16 on the way in (the weights are
+            # bf16 already), accumulation is fp32 on both sides
+            xr = bf16_bits_to_f32(f32_to_bf16_bits(x))
+            np.testing.assert_allclose(y, O.matmul(xr, wb), rtol=0, atol=2e-5 * np.sqrt(K))
             # same kernel, same partition: only the order of the fp32 atomic adds may differ
             np.testing.assert_allclose(y, ref, rtol=0, atol=2e-5 * np.sqrt(K))
         # one more call that repeats the first case must give the first case's answer again
@@ -60,4 +71,17 @@ def test_noalloc_gemm_rejects_sizes_beyond_its_scratch():
     assert L.sdv_gemm_noalloc(p, p, p, 4, 24, 64, None) == pkg.EINVAL          # N not a multiple of 16
     assert L.sdv_gemm_noalloc(p, p, p, 4, 64, 96, None) == pkg.EINVAL          # K not a multiple of 64
     assert L.sdv_gemm_noalloc(None, p, p, 4, 64, 64, None) == pkg.EINVAL
+    # x and w are read 16 bytes at a time: a view that starts 4 bytes into a tensor is refused, not faulted on
+    assert L.sdv_gemm_noalloc(p + 4, p, p, 4, 64, 64, None) == pkg.EINVAL
+    assert L.sdv_gemm_noalloc(p, p + 2, p, 4, 64, 64, None) == pkg.EINVAL
+    assert L.sdv_gemm_noalloc(p, p, p + 2, 4, 64, 64, None) == pkg.EINVAL
+    odd = torch.zeros((5, 65), device="cuda")[1:, :64].contiguous()[0:4]      # contiguous again: aligned
+    assert odd.data_ptr() % 16 == 0
+    view = torch.zeros(4 * 64 + 1, device="cuda")[1:].view(4, 64)            # starts at element 1: 4-byte aligned only
+    dw = torch.zeros((64, 64), dtype=torch.int16, device="cuda")
+    dy = torch.zeros((4, 64), device="cuda")
+    assert pkg.gemm_noalloc(view, dw, dy) == pkg.EINVAL
+    # host memory is refused as well
+    host = np.zeros(64 * 64, dtype=np.float32)
+    assert L.sdv_gemm_noalloc(host.ctypes.data - host.ctypes.data % 16 + 16, p, p, 4, 64, 64, None) == pkg.EINVAL
     assert len(L.sdv_strerror(pkg.ETOOBIG)) > 0
