@@ -178,6 +178,13 @@ int orc_argmax(const float *x, int n) {
 }
 
 /*
+ * Tree-structured drafts (paper Sec. 4.1 "Speculative decoding": drafts are trees, verified in one
+ * pass): with parent != NULL token row j (j >= 1) continues row parent[j] < j (row 0 is the root, the
+ * committed token).  Row j then sits at absolute position start_pos + depth(j), its K/V rows are
+ * written at cache slot start_pos + j, and it attends to cache rows 0 .. start_pos-1 and to the rows
+ * on its own path from the root (itself included), in that order.  parent == NULL is the linear
+ * chain parent[j] = j-1, for which all of this reduces to the description below.
+ *
  * Run the decoder over m tokens at absolute positions start_pos .. start_pos+m-1.
  * kcache/vcache: fp32 [layer][kv_head][max_seq][hd]; rows start_pos.. are written, rows
  * below start_pos are read.  Token row j attends to positions 0 .. start_pos+j.
@@ -185,13 +192,20 @@ int orc_argmax(const float *x, int n) {
  * hidden_out (optional): [m][d] residual stream after the last layer (before the final norm).
  * Returns 0, or -1 on a bad argument.
  */
-int orc_forward(const orc_config *c, const orc_weights *w, const int32_t *tokens, int m, int start_pos,
-                float *kcache, float *vcache, float *logits, int logits_from, float *hidden_out) {
+int orc_forward_tree(const orc_config *c, const orc_weights *w, const int32_t *tokens, const int32_t *parent, int m,
+                     int start_pos, float *kcache, float *vcache, float *logits, int logits_from, float *hidden_out) {
     const int d = c->d_model, hd = c->head_dim, nq = c->n_q_heads, nkv = c->n_kv_heads, f = c->d_ffn;
     const int g = nq / nkv, Nq = nq * hd, Nkv = nkv * hd;
     if (m <= 0 || start_pos < 0 || start_pos + m > c->max_seq) return -1;
     for (int j = 0; j < m; ++j)
         if (tokens[j] < 0 || tokens[j] >= c->vocab) return -1;
+    int *depth = (int *)malloc(sizeof(int) * (size_t)m);
+    for (int j = 0; j < m; ++j) {
+        if (!parent) depth[j] = j;
+        else if (j == 0) depth[j] = 0;
+        else if (parent[j] < 0 || parent[j] >= j) { free(depth); return -1; }
+        else depth[j] = depth[parent[j]] + 1;
+    }
 
     float *h = (float *)malloc(sizeof(float) * (size_t)m * d);
     float *xn = (float *)malloc(sizeof(float) * (size_t)m * d);
@@ -216,26 +230,44 @@ int orc_forward(const orc_config *c, const orc_weights *w, const int32_t *tokens
         orc_matmul(xn, L->wk, c->qkv_bias ? L->bk : NULL, kk, m, Nkv, d);
         orc_matmul(xn, L->wv, c->qkv_bias ? L->bv : NULL, vv, m, Nkv, d);
         for (int j = 0; j < m; ++j) {
-            const int pos = start_pos + j;
+            const int pos = start_pos + depth[j]; /* rotary position */
+            const int slot = start_pos + j;       /* cache row */
             for (int a = 0; a < nq; ++a) orc_rope(q + (size_t)j * Nq + a * hd, hd, pos, c->rope_theta);
             for (int a = 0; a < nkv; ++a) {
                 orc_rope(kk + (size_t)j * Nkv + a * hd, hd, pos, c->rope_theta);
-                memcpy(kc + ((size_t)a * c->max_seq + pos) * hd, kk + (size_t)j * Nkv + a * hd, sizeof(float) * hd);
-                memcpy(vc + ((size_t)a * c->max_seq + pos) * hd, vv + (size_t)j * Nkv + a * hd, sizeof(float) * hd);
+                memcpy(kc + ((size_t)a * c->max_seq + slot) * hd, kk + (size_t)j * Nkv + a * hd, sizeof(float) * hd);
+                memcpy(vc + ((size_t)a * c->max_seq + slot) * hd, vv + (size_t)j * Nkv + a * hd, sizeof(float) * hd);
             }
         }
 #pragma omp parallel
         {
             float *scr = (float *)malloc(sizeof(float) * (size_t)(start_pos + m));
+            /* tree: the keys and values a row sees, gathered in order (cache rows, then its path from the root) */
+            float *kg = parent ? (float *)malloc(sizeof(float) * (size_t)(start_pos + m) * hd) : NULL;
+            float *vg = parent ? (float *)malloc(sizeof(float) * (size_t)(start_pos + m) * hd) : NULL;
+            int *path = parent ? (int *)malloc(sizeof(int) * (size_t)m) : NULL;
 #pragma omp for collapse(2) schedule(dynamic, 1)
             for (int j = 0; j < m; ++j)
                 for (int a = 0; a < nq; ++a) {
                     const int kvh = a / g;
-                    orc_attention_row(q + (size_t)j * Nq + a * hd, kc + (size_t)kvh * c->max_seq * hd,
-                                      vc + (size_t)kvh * c->max_seq * hd, start_pos + j + 1, hd,
-                                      o + (size_t)j * Nq + a * hd, scr);
+                    const float *kh = kc + (size_t)kvh * c->max_seq * hd, *vh = vc + (size_t)kvh * c->max_seq * hd;
+                    if (!parent) {
+                        orc_attention_row(q + (size_t)j * Nq + a * hd, kh, vh, start_pos + j + 1, hd,
+                                          o + (size_t)j * Nq + a * hd, scr);
+                    } else {
+                        const int np = depth[j] + 1;
+                        for (int r = j, i = np - 1; i >= 0; --i, r = (r > 0 ? parent[r] : 0)) path[i] = r;
+                        memcpy(kg, kh, sizeof(float) * (size_t)start_pos * hd);
+                        memcpy(vg, vh, sizeof(float) * (size_t)start_pos * hd);
+                        for (int i = 0; i < np; ++i) {
+                            memcpy(kg + (size_t)(start_pos + i) * hd, kh + (size_t)(start_pos + path[i]) * hd, sizeof(float) * hd);
+                            memcpy(vg + (size_t)(start_pos + i) * hd, vh + (size_t)(start_pos + path[i]) * hd, sizeof(float) * hd);
+                        }
+                        orc_attention_row(q + (size_t)j * Nq + a * hd, kg, vg, start_pos + np, hd,
+                                          o + (size_t)j * Nq + a * hd, scr);
+                    }
                 }
-            free(scr);
+            free(scr); free(kg); free(vg); free(path);
         }
         orc_matmul(o, L->wo, NULL, t1, m, d, Nq);
         for (size_t i = 0; i < (size_t)m * d; ++i) h[i] += t1[i];
@@ -254,8 +286,14 @@ int orc_forward(const orc_config *c, const orc_weights *w, const int32_t *tokens
             orc_rmsnorm(h + (size_t)(logits_from + j) * d, w->final_norm, c->rms_eps, xn + (size_t)j * d, d);
         orc_matmul(xn, c->tied_lm_head ? w->emb : w->lm_head, NULL, logits, r, c->vocab, d);
     }
-    free(h); free(xn); free(q); free(kk); free(vv); free(o); free(t1); free(gt); free(up); free(act);
+    free(h); free(xn); free(q); free(kk); free(vv); free(o); free(t1); free(gt); free(up); free(act); free(depth);
     return 0;
+}
+
+/* The linear chain: row j continues row j-1 (Sec. 3.2, the drafts of one retrieval are checked in one pass). */
+int orc_forward(const orc_config *c, const orc_weights *w, const int32_t *tokens, int m, int start_pos,
+                float *kcache, float *vcache, float *logits, int logits_from, float *hidden_out) {
+    return orc_forward_tree(c, w, tokens, NULL, m, start_pos, kcache, vcache, logits, logits_from, hidden_out);
 }
 
 /*

@@ -92,6 +92,9 @@ def lib():
         L.orc_forward.argtypes = [C.POINTER(_Cfg), C.POINTER(_Weights), C.c_void_p, C.c_int, C.c_int, C.c_void_p,
                                   C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         L.orc_forward.restype = C.c_int
+        L.orc_forward_tree.argtypes = [C.POINTER(_Cfg), C.POINTER(_Weights), C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
+        L.orc_forward_tree.restype = C.c_int
         L.orc_ngram_draft.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                       C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
         L.orc_ngram_draft.restype = C.c_int
@@ -270,6 +273,114 @@ class DraftExtension:
         self.used = False
 
 
+# ---------------------------------------------------------------- in-context calibration and tree drafts (Sec. 4.3, Sec. 4.1)
+def top_successors(logits_row, b: int) -> List[int]:
+    """"Sample" (Sec. 4.3): the b highest-logit token ids of one prefill position, best first; among equal
+    logits the lower id first (the greedy tie rule).  Taken one at a time: the greedy token, then the
+    greedy token of what is left."""
+    row = np.array(logits_row, dtype=np.float32, copy=True)
+    out = []
+    for _ in range(min(b, len(row))):
+        i = argmax(row)
+        out.append(i)
+        row[i] = -np.inf
+    return out
+
+
+def calibrate(context: Sequence[int], prefill_logits: np.ndarray, b: int):
+    """The calibration structure of Sec. 4.3 for one request.
+
+    succ[p] = top_successors(logits of context position p): with the context token C[p] each of them
+    is an anchor <C[p], prediction>.  "Search": occ[p][i] = the position in the context where the
+    prediction succ[p][i] occurs (the paper names no rule for several occurrences: the latest one,
+    as in the retrieval drafter), -1 where it does not occur; a matched anchor is expanded with
+    that position's own successors, which gives the two-level token tree of the text.
+    Returns (succ [n, b] int32, occ [n, b] int32)."""
+    ctx = [int(t) for t in context]
+    n = len(ctx)
+    assert prefill_logits.shape[0] == n
+    succ = np.zeros((n, b), dtype=np.int32)
+    occ = np.full((n, b), -1, dtype=np.int32)
+    for p in range(n):
+        s = top_successors(prefill_logits[p], b)
+        succ[p, :len(s)] = s
+        for i, tok in enumerate(s):
+            for q in range(n - 1, -1, -1):
+                if ctx[q] == tok:
+                    occ[p, i] = q
+                    break
+    return succ, occ
+
+
+def build_draft_tree(T: int, chain: Sequence[int], context: Sequence[int], succ: np.ndarray, occ: np.ndarray,
+                     max_nodes: int):
+    """Tree-structured draft for one step (Sec. 4.1, Sec. 4.3).  Node 0 is the committed token T.
+
+    The retrieval drafter's chain x_1..x_m comes first, as one path.  Then the calibrated tree of T:
+    with p the latest position of T in the context (none: no calibrated branches), each successor
+    succ[p][i] becomes a child of the root, followed at once by its own children succ[q] when the
+    anchor was matched at q = occ[p][i] (depth first, two levels, as the text describes).  A token
+    that a node already has as a child is not added twice (the existing child is used).  At most
+    max_nodes draft nodes; what does not fit is left out.  Returns (tokens, parent) including node 0,
+    parent[0] = -1; every parent index is smaller than its child's."""
+    tokens, parent = [int(T)], [-1]
+
+    def child_with(node, tok):
+        for c in range(1, len(tokens)):
+            if parent[c] == node and tokens[c] == tok:
+                return c
+        return -1
+
+    def add(node, tok):
+        c = child_with(node, tok)
+        if c >= 0:
+            return c
+        if len(tokens) - 1 >= max_nodes:
+            return -1
+        tokens.append(int(tok))
+        parent.append(node)
+        return len(tokens) - 1
+
+    cur = 0
+    for x in chain:
+        cur = add(cur, int(x))
+        if cur < 0:
+            break
+    ctx = [int(t) for t in context]
+    p = -1
+    for q in range(len(ctx) - 1, -1, -1):
+        if ctx[q] == int(T):
+            p = q
+            break
+    if p >= 0:
+        for i in range(succ.shape[1]):
+            c = add(0, int(succ[p, i]))
+            q = int(occ[p, i])
+            if c >= 0 and q >= 0:
+                for i2 in range(succ.shape[1]):
+                    add(c, int(succ[q, i2]))
+    return tokens, parent
+
+
+def tree_accept(tokens: Sequence[int], parent: Sequence[int], y: Sequence[int]) -> List[int]:
+    """Strict acceptance on a tree: starting at the root, step to the child whose token is the model's
+    prediction at the current node (the lowest-numbered one, should several carry it), until no child
+    does.  Returns the accepted path (node indices, root excluded).  The emitted tokens are the
+    path's tokens followed by the prediction at its last node: on a single path this is the
+    accepted-prefix rule x_1..x_{e-1}, y_e of Sec. 4.4."""
+    path, cur = [], 0
+    while True:
+        nxt = -1
+        for c in range(1, len(tokens)):
+            if parent[c] == cur and tokens[c] == y[cur]:
+                nxt = c
+                break
+        if nxt < 0:
+            return path
+        path.append(nxt)
+        cur = nxt
+
+
 # ---------------------------------------------------------------- the model
 class OracleModel:
     """Holds the weight arrays (bf16 bit patterns from sdv_inputs) and an fp32 KV cache."""
@@ -303,22 +414,35 @@ class OracleModel:
         a = self.kcache if which == "k" else self.vcache
         return a.reshape(c.n_layers, c.n_kv_heads, self.max_seq, c.head_dim)
 
-    def forward(self, tokens, start_pos: int, logits_from: Optional[int] = 0, want_hidden: bool = False):
+    def forward(self, tokens, start_pos: int, logits_from: Optional[int] = 0, want_hidden: bool = False,
+                parent: Optional[Sequence[int]] = None):
         """Runs the decoder over `tokens` at positions start_pos.. and writes their KV rows.
+
+        parent (tree-structured drafts, Sec. 4.1): row j continues row parent[j] < j (parent[0] is
+        ignored); row j is at position start_pos + depth(j), its KV rows go to cache slot
+        start_pos + j, and it attends to the cache and to its own path from the root.
 
         Returns logits [m - logits_from, V] (None when logits_from is None), and the final
         residual stream [m, d] when want_hidden.
         """
         tokens = np.ascontiguousarray(tokens, dtype=np.int32)
         m = len(tokens)
+        par = None
+        if parent is not None:
+            par = np.ascontiguousarray(parent, dtype=np.int32)
+            assert len(par) == m
         logits = None
         lf = m
         if logits_from is not None:
             lf = int(logits_from)
             logits = np.empty((m - lf, self.cfg.vocab), dtype=np.float32)
         hid = np.empty((m, self.cfg.d_model), dtype=np.float32) if want_hidden else None
-        rc = lib().orc_forward(C.byref(self._c), C.byref(self._w), _p(tokens), m, int(start_pos), _p(self.kcache),
-                               _p(self.vcache), _p(logits), lf, _p(hid))
+        if par is None:
+            rc = lib().orc_forward(C.byref(self._c), C.byref(self._w), _p(tokens), m, int(start_pos), _p(self.kcache),
+                                   _p(self.vcache), _p(logits), lf, _p(hid))
+        else:
+            rc = lib().orc_forward_tree(C.byref(self._c), C.byref(self._w), _p(tokens), _p(par), m, int(start_pos),
+                                        _p(self.kcache), _p(self.vcache), _p(logits), lf, _p(hid))
         if rc != 0:
             raise ValueError("orc_forward: bad argument")
         return (logits, hid) if want_hidden else logits
@@ -336,6 +460,26 @@ class OracleModel:
                 self.forward(context[s:e], s, logits_from=None)
         self.kv_len = n
         return last
+
+    def prefill_all_logits(self, context, chunk: int) -> np.ndarray:
+        """Chunked prefill that keeps the logits of every context position, [n, V] (what the
+        calibration of Sec. 4.3 starts from)."""
+        context = np.ascontiguousarray(context, dtype=np.int32)
+        n = len(context)
+        rows = []
+        for s in range(0, n, chunk):
+            e = min(n, s + chunk)
+            rows.append(self.forward(context[s:e], s, logits_from=0))
+        self.kv_len = n
+        return np.concatenate(rows, axis=0)
+
+    def move_kv_rows(self, src: Sequence[int], dst: Sequence[int]) -> None:
+        """Copies cache rows src[i] -> dst[i] (all layers and KV heads), in the order given."""
+        for which in ("k", "v"):
+            a = self.kv_view(which)
+            for s_, d_ in zip(src, dst):
+                if s_ != d_:
+                    a[:, :, d_, :] = a[:, :, s_, :]
 
 
 # ---------------------------------------------------------------- decoding loops
@@ -432,3 +576,44 @@ def spec_decode(model: OracleModel, context, gen: int, chunk: int, k: int, ngram
         T = emitted[-1]
     model.kv_len = L
     return out, steps
+
+
+def spec_decode_tree(model: OracleModel, context, gen: int, chunk: int, k: int, ngram_n: int, ngram_min: int,
+                     calib_top: int, max_nodes: int, tree_builder=None, keep_logits: bool = False):
+    """Greedy speculative decoding with tree-structured drafts: the retrieval chain plus the branches
+    of the calibrated token tree (Sec. 4.3), verified in one pass; the accepted path's KV rows are
+    moved to consecutive cache slots.  `tree_builder(history) -> (tokens, parent)` overrides the
+    draft construction (tests force trees with it).  Returns (tokens, steps, (succ, occ)); a step
+    is a dict with the tree, the predictions, the accepted path and the emitted tokens."""
+    context = np.ascontiguousarray(context, dtype=np.int32)
+    logits_all = model.prefill_all_logits(context, chunk)
+    succ, occ = calibrate(context, logits_all, calib_top)
+    hist = [int(t) for t in context]
+    T = argmax(logits_all[-1])
+    hist.append(T)
+    out = [T]
+    L = len(context)
+    steps = []
+    while len(out) < gen:
+        if tree_builder is not None:
+            tokens, parent = tree_builder(hist)
+        else:
+            chain = ngram_draft(context, hist, ngram_n, ngram_min, k)[0].tolist()
+            tokens, parent = build_draft_tree(T, chain, context, succ, occ, max_nodes)
+        assert tokens[0] == T
+        logits = model.forward(tokens, L, logits_from=0, parent=[0] + list(parent[1:]))
+        y = [argmax(logits[j]) for j in range(len(tokens))]
+        path = tree_accept(tokens, parent, y)
+        emitted = [tokens[c] for c in path] + [y[path[-1] if path else 0]]
+        emitted = emitted[:gen - len(out)]
+        keep = path[:len(emitted) - 1] if len(emitted) <= len(path) else path
+        model.move_kv_rows([L + c for c in keep], [L + 1 + i for i in range(len(keep))])
+        steps.append(dict(kv_len_before=L, pending=T, tokens=list(tokens), parent=list(parent), y=y, path=list(path),
+                          emitted=list(emitted), logits=logits.copy() if keep_logits else None,
+                          margin=[top2_margin(logits[j]) for j in range(len(tokens))]))
+        L += len(emitted)
+        out.extend(emitted)
+        hist.extend(emitted)
+        T = emitted[-1]
+    model.kv_len = L
+    return out, steps, (succ, occ)
