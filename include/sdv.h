@@ -43,6 +43,7 @@ enum {
 
 #define SDV_NGRAM_MAX 4096 /* longest history suffix the drafter can be asked to match */
 #define SDV_K_MAX 31 /* longest draft per verify step (M = k+1 <= 32 rows) */
+#define SDV_CALIB_MAX 4 /* most successors sampled per context position by the calibration */
 
 typedef struct sdv_ctx sdv_ctx;
 
@@ -155,6 +156,42 @@ int sdv_verify(sdv_ctx *ctx, const int32_t *host_draft, int draft_len, int32_t *
 int sdv_extend_draft(sdv_ctx *ctx, int max_total, int32_t *host_draft, int *draft_len);
 int sdv_extension_update(sdv_ctx *ctx, int max_life, int32_t *host_segment, int *segment_len, int *lifetime);
 
+/* In-context distribution calibration (paper Sec. 4.3 "Workflow") and tree-structured drafts
+ * (Sec. 4.1 "Speculative decoding": drafts are trees, verified in one pass).
+ *
+ * sdv_set_calibration: call before the first sdv_prefill_chunk.  With top_b in 1..SDV_CALIB_MAX every
+ * prefill tile also runs the LM head and keeps, for each context position, the top_b token ids of
+ * its logits (largest first, lowest id among equals): "Sample", the model-preferred anchors
+ * <context token, prediction>.  After the last chunk each prediction is looked up in the request
+ * ("Search": its latest position, -1 where it does not occur).  top_b = 0 switches it off.
+ * sdv_get_calibration copies the two tables for the first n_positions context positions to the
+ * host as int32 [n_positions][top_b] (either pointer may be NULL).
+ *
+ * sdv_draft_tree: the draft of one step as a tree with at most max_nodes (<= k_max) nodes.  The
+ * retrieval drafter's chain of up to k tokens (k = 0: none) is its first path; then, with p the
+ * latest position of the committed token T in the request, each sampled successor of p becomes a
+ * child of the root, followed at once by the successors of the position where that anchor was
+ * matched (two levels, depth first).  A token a node already has as a child is not added twice.
+ * Node i (1-based) continues row host_parent[i-1] < i, row 0 being T; host_tokens / host_parent
+ * (k_max ints each) and n_nodes may be NULL; if any is given the stream is synchronised and the
+ * next sdv_verify_tree computes exactly n_nodes + 1 rows, else max_nodes + 1.
+ *
+ * sdv_verify_tree: one forward pass over [T, nodes]: node i sits at position L + depth(i), its K/V
+ * rows go to cache slot L + i, and it attends to the cache and to its own path from the root.
+ * host_tokens == NULL verifies the tree sdv_draft_tree left on the device.  Acceptance is strict: from
+ * the root, step to the child (the lowest-numbered one) whose token equals the model's greedy
+ * prediction at the current row, until no child does; the emitted tokens are the path's tokens and
+ * the prediction at its last row.  host_y (n_nodes+1 ints), host_path (k_max ints: the accepted
+ * rows) and path_len may be NULL.  sdv_commit then first moves the accepted rows' K/V to the
+ * consecutive slots L+1.. before L advances.  A chain is the tree parent[i-1] = i-1.
+ * Errors: SDV_ESTATE (order), SDV_EINVAL (a parent that is not an earlier row, token range),
+ * SDV_ECAPACITY. */
+int sdv_set_calibration(sdv_ctx *ctx, int top_b);
+int sdv_get_calibration(sdv_ctx *ctx, int32_t *host_succ, int32_t *host_occ, int n_positions);
+int sdv_draft_tree(sdv_ctx *ctx, int k, int max_nodes, int32_t *host_tokens, int32_t *host_parent, int *n_nodes);
+int sdv_verify_tree(sdv_ctx *ctx, const int32_t *host_tokens, const int32_t *host_parent, int n_nodes,
+                    int32_t *host_y, int32_t *host_path, int *path_len);
+
 /* Commit / rollback (paper Sec. 3.2: tokens after the first mismatch are discarded; Sec. 4.4:
  * the accepted prefix is x_1..x_{e-1}, y_e): emits x_1..x_a, y_{a+1} of the last verify, cut to
  * max_emit tokens when max_emit > 0; appends them to the history; L += number emitted; the last
@@ -207,6 +244,13 @@ int sdv_debug_accept(sdv_ctx *ctx, const int32_t *host_draft, int draft_len, con
 /* Like sdv_commit, but with a caller-chosen accept length (<= draft_len of the last verify) and
  * next token: teacher forcing for step-by-step comparisons. */
 int sdv_debug_force_commit(sdv_ctx *ctx, int accept_len, int32_t next_token);
+
+/* The same after sdv_verify_tree: commits a caller-chosen accepted path (rows, ascending) and next token. */
+int sdv_debug_force_commit_tree(sdv_ctx *ctx, const int32_t *host_path, int path_len, int32_t next_token);
+
+/* Runs the calibration's top-successor kernel on caller-supplied logits rows (host fp32 [rows][vocab],
+ * rows <= 32) and returns int32 [rows][top_b]: the integer part of "Sample" on its own. */
+int sdv_debug_top_successors(sdv_ctx *ctx, const float *host_logits, int rows, int top_b, int32_t *host_out);
 
 /* Copies rows [pos0, pos0+n) of one layer's key (which = 0) or value (which = 1) cache to the
  * host as fp32 [n_kv_heads][n][head_dim]. */

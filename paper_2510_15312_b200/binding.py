@@ -19,6 +19,8 @@ EXPORTS = [
     "sdv_debug_force_commit", "sdv_debug_read_kv", "sdv_debug_read_hidden", "sdv_debug_gemm",
     "sdv_debug_timeout_probe", "sdv_debug_profile", "sdv_launch_count", "sdv_last_verify_ms",
     "sdv_gemm_noalloc", "sdv_debug_layout_check", "sdv_debug_plan",
+    "sdv_set_calibration", "sdv_get_calibration", "sdv_draft_tree", "sdv_verify_tree", "sdv_debug_force_commit_tree",
+    "sdv_debug_top_successors",
 ]
 
 
@@ -92,6 +94,12 @@ def load_library(path: Optional[str] = None):
     L.sdv_gemm_noalloc.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp]
     L.sdv_debug_layout_check.argtypes = [C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_int]
     L.sdv_debug_plan.argtypes = [C.POINTER(SdvConfig), C.c_int, C.c_int, C.POINTER(C.c_int)]
+    L.sdv_set_calibration.argtypes = [vp, C.c_int]
+    L.sdv_get_calibration.argtypes = [vp, vp, vp, C.c_int]
+    L.sdv_draft_tree.argtypes = [vp, C.c_int, C.c_int, i32p, i32p, ip]
+    L.sdv_verify_tree.argtypes = [vp, i32p, i32p, C.c_int, i32p, i32p, ip]
+    L.sdv_debug_force_commit_tree.argtypes = [vp, i32p, C.c_int, C.c_int]
+    L.sdv_debug_top_successors.argtypes = [vp, vp, C.c_int, C.c_int, vp]
     for name in EXPORTS:
         if name not in ("sdv_workspace_bytes", "sdv_strerror", "sdv_launch_count"):
             getattr(L, name).restype = C.c_int
@@ -220,6 +228,59 @@ class Sdv:
         self._check(lib().sdv_extension_update(self._h, max_life, seg.ctypes.data, C.byref(n), C.byref(life)),
                     "sdv_extension_update")
         return seg[:n.value].tolist(), life.value
+
+    # ---- in-context calibration and tree drafts (Sec. 4.3, Sec. 4.1)
+    def set_calibration(self, top_b: int):
+        self._check(lib().sdv_set_calibration(self._h, int(top_b)), "sdv_set_calibration")
+        self._calib_b = int(top_b)
+
+    def get_calibration(self, n_positions: int):
+        """(succ, occ) as int32 [n_positions, top_b]."""
+        b = max(1, getattr(self, "_calib_b", 0))
+        succ = np.zeros((n_positions, b), dtype=np.int32)
+        occ = np.zeros((n_positions, b), dtype=np.int32)
+        self._check(lib().sdv_get_calibration(self._h, succ.ctypes.data, occ.ctypes.data, n_positions), "sdv_get_calibration")
+        return succ, occ
+
+    def draft_tree(self, k: int, max_nodes: int, fetch: bool = True):
+        """Returns (tokens, parent) of the draft nodes when fetch: node i+1 continues row parent[i]."""
+        if not fetch:
+            self._check(lib().sdv_draft_tree(self._h, k, max_nodes, None, None, None), "sdv_draft_tree")
+            return None
+        tok = np.zeros(K_MAX, dtype=np.int32)
+        par = np.zeros(K_MAX, dtype=np.int32)
+        n = C.c_int(0)
+        self._check(lib().sdv_draft_tree(self._h, k, max_nodes, tok.ctypes.data, par.ctypes.data, C.byref(n)), "sdv_draft_tree")
+        return tok[:n.value].tolist(), par[:n.value].tolist()
+
+    def verify_tree(self, tokens: Optional[Sequence[int]] = None, parent: Optional[Sequence[int]] = None, fetch: bool = True):
+        """tokens / parent of the draft nodes (None: the device tree); returns (y, accepted path rows) when fetch."""
+        t = None if tokens is None else np.ascontiguousarray(tokens, dtype=np.int32)
+        p = None if parent is None else np.ascontiguousarray(parent, dtype=np.int32)
+        n = 0 if t is None else len(t)
+        one = np.zeros(1, np.int32)
+        tp = None if t is None else (t.ctypes.data if n else one.ctypes.data)
+        pp = None if t is None else (p.ctypes.data if n else one.ctypes.data)
+        if not fetch:
+            self._check(lib().sdv_verify_tree(self._h, tp, pp, n, None, None, None), "sdv_verify_tree")
+            return None
+        y = np.zeros(K_MAX + 1, dtype=np.int32)
+        path = np.zeros(K_MAX, dtype=np.int32)
+        a = C.c_int(0)
+        self._check(lib().sdv_verify_tree(self._h, tp, pp, n, y.ctypes.data, path.ctypes.data, C.byref(a)), "sdv_verify_tree")
+        return y.tolist(), path[:a.value].tolist()
+
+    def debug_force_commit_tree(self, path: Sequence[int], next_token: int):
+        p = np.ascontiguousarray(path, dtype=np.int32)
+        self._check(lib().sdv_debug_force_commit_tree(self._h, p.ctypes.data if len(p) else None, len(p), int(next_token)),
+                    "sdv_debug_force_commit_tree")
+
+    def debug_top_successors(self, logits: np.ndarray, top_b: int) -> np.ndarray:
+        lg = np.ascontiguousarray(logits, dtype=np.float32)
+        out = np.zeros((lg.shape[0], top_b), dtype=np.int32)
+        self._check(lib().sdv_debug_top_successors(self._h, lg.ctypes.data, lg.shape[0], top_b, out.ctypes.data),
+                    "sdv_debug_top_successors")
+        return out
 
     def commit(self, max_emit: int = 0) -> Tuple[List[int], int]:
         out = np.zeros(K_MAX + 1, dtype=np.int32)

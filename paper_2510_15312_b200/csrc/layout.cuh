@@ -161,9 +161,15 @@ enum StateWord {
     ST_DB_LEN,        // tokens in the extra token database the drafter also searches (0: none)
     ST_DRAFT = 16,    // [32]
     ST_Y = 48,        // [33]
+    ST_TREE_ON = 82,  // 1: the draft is a tree (ST_PARENT .. ST_ANC hold its shape), 0: a chain
+    ST_PATH_LEN = 83, // nodes on the accepted path of the last tree verify
     ST_EMITTED = 96,  // [33]
     ST_SEG = 160,     // [32]
-    ST_WORDS = 192
+    ST_PARENT = 192,  // [32] row that row j continues (row 0 = the committed token; draft node i is row i)
+    ST_DEPTH = 224,   // [32] distance of row j from the root = its position minus the KV length
+    ST_ANC = 256,     // [32] bit r set: row r lies on row j's path from the root (j itself included)
+    ST_PATH = 288,    // [32] accepted path (rows), root excluded
+    ST_WORDS = 320
 };
 
 struct FwdParams {
@@ -207,6 +213,7 @@ struct FwdParams {
     int ph_begin, ph_end;
     unsigned bar_base; // barrier counter value before this launch
     int store_logits;
+    int tree;          // 1: the rows form a tree (positions, masks from the state block), 0: a chain
     // shared-memory plan of this launch (bytes from the 1024-aligned base)
     int nstage;        // ring slots of kStageBytes, at offset 0
     int u_off;         // operand region (token operand of the running GEMM; attention tiles)

@@ -23,7 +23,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Regions {
     size_t state, bar, never, hist, db, rope, norm_w, bias, wlayers, wlm, emb, kcache, vcache, h, qkv_acc, sumsq, part_o,
-        part_ml, cand_val, cand_idx, logits, raw_out, staging, wraw, xstage, prof, total;
+        part_ml, cand_val, cand_idx, logits, raw_out, staging, wraw, xstage, prof, succ, occ, total;
     size_t layer_stride, staging_bytes, raw_kmax;
 };
 
@@ -92,6 +92,8 @@ Regions carve(const sdv_config* c) {
     r.raw_out = take((size_t)kMaxRows * (st / 128) * 4);  // N <= staging / (2 bytes * 64 columns)
     r.xstage = take((size_t)kMaxRows * raw_kmax * 4);
     r.prof = take((size_t)(3 + kPhasesPerLayer * c->n_layers) * kMaxGrid * kProfWords * 8);
+    r.succ = take((size_t)c->max_seq * SDV_CALIB_MAX * 4);  // calibration: sampled successors per context position
+    r.occ = take((size_t)c->max_seq * SDV_CALIB_MAX * 4);   // and where each occurs in the context
     r.total = off;
     return r;
 }
@@ -255,6 +257,10 @@ struct sdv_ctx {
     long long launches;
     bool have_verify_time;
     bool poisoned;
+    int calib_b;         // successors sampled per context position during prefill (0: calibration off)
+    bool calibrated;     // the calibration tables cover the whole context
+    bool tree_pending;   // the device draft is a tree
+    bool tree_verified;  // the outstanding verify result is a tree's
 };
 
 namespace {
@@ -319,7 +325,8 @@ void plan_attention(FwdParams& P, int rows, int L) {
 }
 
 // Runs phases [ph_begin, ph_end) over `rows` token rows at position L.
-int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph_end, bool timed) {
+int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph_end, bool timed, bool force_logits = false,
+                   bool tree = false) {
     FwdParams P = ctx->P;
     int smem_bytes = 0;
     const bool raw_only = (ph_begin == 2 + kPhasesPerLayer * ctx->cfg.n_layers);
@@ -330,7 +337,8 @@ int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph
     P.ph_begin = ph_begin;
     P.ph_end = ph_end;
     P.bar_base = ctx->bar_base;
-    P.store_logits = ctx->parity;
+    P.store_logits = (ctx->parity || force_logits) ? 1 : 0;
+    P.tree = tree ? 1 : 0;
     P.prof = ctx->profile ? (unsigned long long*)(ctx->ws + ctx->r.prof) : nullptr;
     const int nbar = ph_end - ph_begin - 1;
     ctx->bar_base += (unsigned)(nbar * ctx->G);
@@ -376,6 +384,13 @@ void fill_draft_arg(DraftArg& a, const int32_t* tok, int n) {
 int commit_common(sdv_ctx* ctx, int max_emit, int force_accept, int force_token, int32_t* host_emitted, int* n_emitted,
                   int* kv_len) {
     int* hist = (int*)(ctx->ws + ctx->r.hist);
+    if (ctx->tree_verified) {
+        // the accepted path's K/V rows move to consecutive cache slots before the length advances
+        kv_compact_kernel<<<dim3(ctx->cfg.n_layers * ctx->cfg.n_kv_heads, 2), 128, 0, ctx->stream>>>(
+            ctx->P.state, ctx->P.kcache, ctx->P.vcache, ctx->cfg.max_seq, ctx->cfg.head_dim, max_emit);
+        ctx->launches++;
+        ctx->tree_verified = false;
+    }
     commit_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, hist, max_emit, force_accept, force_token);
     ctx->launches++;
     CK(cudaGetLastError());
@@ -386,6 +401,7 @@ int commit_common(sdv_ctx* ctx, int max_emit, int force_accept, int force_token,
     ctx->hist_len = ctx->pinned[ST_HIST_LEN];
     ctx->verified = false;
     ctx->draft_pending = false;
+    ctx->tree_pending = false;
     if (n_emitted) *n_emitted = n;
     if (kv_len) *kv_len = ctx->kv_len;
     if (host_emitted)
@@ -646,8 +662,16 @@ int sdv_prefill_chunk(sdv_ctx* ctx, const int32_t* host_tokens, int n, int is_la
     while (done < n) {
         const int rows = (n - done < tile) ? n - done : tile;
         const bool last_tile = is_last && (done + rows == n);
-        int rc = launch_forward(ctx, rows, ctx->kv_len, 1, 0, last_tile ? n_ph + 1 : n_ph, false);
+        const bool calib = ctx->calib_b > 0;
+        int rc = launch_forward(ctx, rows, ctx->kv_len, 1, 0, (last_tile || calib) ? n_ph + 1 : n_ph, false, calib);
         if (rc) return rc;
+        if (calib) {
+            // "Sample": the best successors of every row of this tile, from the logits the LM head just stored
+            top_successors_kernel<<<rows, 1024, 0, ctx->stream>>>(ctx->P.logits, c.vocab, ctx->calib_b,
+                                                               (int*)(ctx->ws + ctx->r.succ) + (size_t)ctx->kv_len * ctx->calib_b);
+            ctx->launches++;
+            CK(cudaGetLastError());
+        }
         ctx->kv_len += rows;
         ctx->hist_len += rows;
         done += rows;
@@ -665,6 +689,15 @@ int sdv_prefill_chunk(sdv_ctx* ctx, const int32_t* host_tokens, int n, int is_la
                 CK(cudaGetLastError());
                 ctx->hist_len += 1;
                 ctx->prefill_done = true;
+                if (ctx->calib_b > 0) {
+                    // "Search": where each sampled successor occurs in the request
+                    const int total = ctx->n_ctx * ctx->calib_b;
+                    anchor_search_kernel<<<(total + 255) / 256, 256, 0, ctx->stream>>>(
+                        hist, ctx->n_ctx, ctx->calib_b, (const int*)(ctx->ws + ctx->r.succ), (int*)(ctx->ws + ctx->r.occ));
+                    ctx->launches++;
+                    CK(cudaGetLastError());
+                    ctx->calibrated = true;
+                }
             }
         }
     }
@@ -681,6 +714,7 @@ int sdv_draft(sdv_ctx* ctx, int k, int32_t* host_draft, int* draft_len) {
     ctx->launches++;
     CK(cudaGetLastError());
     ctx->draft_pending = true;
+    ctx->tree_pending = false;
     ctx->draft_k = k;
     ctx->verified = false;
     if (host_draft || draft_len) {
@@ -716,12 +750,14 @@ int sdv_verify(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, int32_t* 
         ctx->launches++;
         CK(cudaGetLastError());
     }
-    int rc = launch_forward(ctx, rows, ctx->kv_len, 0, 0, 2 + kPhasesPerLayer * c.n_layers, true);
+    const bool tree = !host_draft && ctx->tree_pending;
+    int rc = launch_forward(ctx, rows, ctx->kv_len, 0, 0, 2 + kPhasesPerLayer * c.n_layers, true, false, tree);
     if (rc) return rc;
     accept_kernel<<<1, 32 * rows, 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0);
     ctx->launches++;
     CK(cudaGetLastError());
     ctx->verified = true;
+    ctx->tree_verified = tree;
     ctx->last_rows = rows;
     if (host_y || accept_len) {
         rc = read_state(ctx);
@@ -787,6 +823,123 @@ int sdv_extension_update(sdv_ctx* ctx, int max_life, int32_t* host_segment, int*
     return SDV_OK;
 }
 
+int sdv_set_calibration(sdv_ctx* ctx, int top_b) {
+    if (!ctx || top_b < 0 || top_b > SDV_CALIB_MAX) return SDV_EINVAL;
+    if (ctx->kv_len > 0 || ctx->prefill_done) return SDV_ESTATE;  // the tables are filled while the context is prefilled
+    ctx->calib_b = top_b;
+    ctx->calibrated = false;
+    return SDV_OK;
+}
+
+int sdv_get_calibration(sdv_ctx* ctx, int32_t* host_succ, int32_t* host_occ, int n_positions) {
+    if (!ctx || n_positions < 1 || (!host_succ && !host_occ)) return SDV_EINVAL;
+    if (!ctx->calibrated) return SDV_ESTATE;
+    if (n_positions > ctx->n_ctx) return SDV_EINVAL;
+    const size_t bytes = (size_t)n_positions * ctx->calib_b * 4;
+    if (host_succ) CK(cudaMemcpyAsync(host_succ, ctx->ws + ctx->r.succ, bytes, cudaMemcpyDeviceToHost, ctx->stream));
+    if (host_occ) CK(cudaMemcpyAsync(host_occ, ctx->ws + ctx->r.occ, bytes, cudaMemcpyDeviceToHost, ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
+    return SDV_OK;
+}
+
+int sdv_draft_tree(sdv_ctx* ctx, int k, int max_nodes, int32_t* host_tokens, int32_t* host_parent, int* n_nodes) {
+    if (!ctx || k < 0 || k > ctx->cfg.k_max || max_nodes < 1 || max_nodes > ctx->cfg.k_max) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->prefill_done) return SDV_ESTATE;
+    int* hist = (int*)(ctx->ws + ctx->r.hist);
+    if (k > 0) {
+        ngram_draft_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->P.state, hist, (const int*)(ctx->ws + ctx->r.db), ctx->cfg.ngram_n,
+                                                        ctx->cfg.ngram_min, k, ctx->cfg.search_history);
+    } else {
+        DraftArg none;
+        fill_draft_arg(none, nullptr, 0);
+        set_draft_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, none);
+    }
+    tree_draft_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->P.state, hist, (const int*)(ctx->ws + ctx->r.succ),
+                                                   (const int*)(ctx->ws + ctx->r.occ), ctx->calibrated ? ctx->calib_b : 0, max_nodes);
+    ctx->launches += 2;
+    CK(cudaGetLastError());
+    ctx->draft_pending = true;
+    ctx->tree_pending = true;
+    ctx->draft_k = max_nodes;   // rows of the next verify: the bound, or the exact count when the caller reads it
+    ctx->verified = false;
+    if (host_tokens || host_parent || n_nodes) {
+        int rc = read_state(ctx);
+        if (rc) return rc;
+        const int n = ctx->pinned[ST_DRAFT_LEN];
+        ctx->draft_k = n;
+        if (n_nodes) *n_nodes = n;
+        for (int i = 0; i < n; ++i) {
+            if (host_tokens) host_tokens[i] = ctx->pinned[ST_DRAFT + i];
+            if (host_parent) host_parent[i] = ctx->pinned[ST_PARENT + 1 + i];
+        }
+    }
+    return SDV_OK;
+}
+
+int sdv_verify_tree(sdv_ctx* ctx, const int32_t* host_tokens, const int32_t* host_parent, int n_nodes, int32_t* host_y,
+                    int32_t* host_path, int* path_len) {
+    if (!ctx) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->prefill_done || !ctx->weights_loaded) return SDV_ESTATE;
+    const sdv_config& c = ctx->cfg;
+    int rows;
+    if (host_tokens) {
+        if (!host_parent || n_nodes < 0 || n_nodes > c.k_max) return SDV_EINVAL;
+        for (int i = 0; i < n_nodes; ++i) {
+            if (host_tokens[i] < 0 || host_tokens[i] >= c.vocab) return SDV_EINVAL;
+            if (host_parent[i] < 0 || host_parent[i] > i) return SDV_EINVAL;  // node i + 1 continues an earlier row
+        }
+        rows = n_nodes + 1;
+    } else {
+        if (!ctx->tree_pending) return SDV_ESTATE;
+        rows = ctx->draft_k + 1;
+    }
+    if (ctx->kv_len + rows > c.max_seq) return SDV_ECAPACITY;
+    if (host_tokens) {
+        DraftArg t, p;
+        fill_draft_arg(t, host_tokens, n_nodes);
+        fill_draft_arg(p, host_parent, n_nodes);
+        set_tree_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, t, p);
+        ctx->launches++;
+        CK(cudaGetLastError());
+    }
+    int rc = launch_forward(ctx, rows, ctx->kv_len, 0, 0, 2 + kPhasesPerLayer * c.n_layers, true, false, true);
+    if (rc) return rc;
+    accept_kernel<<<1, 32 * rows, 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    ctx->verified = true;
+    ctx->tree_verified = true;
+    ctx->last_rows = rows;
+    if (host_y || host_path || path_len) {
+        rc = read_state(ctx);
+        if (rc) return rc;
+        const int n = ctx->pinned[ST_DRAFT_LEN], a = ctx->pinned[ST_PATH_LEN];
+        if (path_len) *path_len = a;
+        if (host_path)
+            for (int i = 0; i < a; ++i) host_path[i] = ctx->pinned[ST_PATH + i];
+        if (host_y)
+            for (int i = 0; i <= n; ++i) host_y[i] = ctx->pinned[ST_Y + i];
+    }
+    return SDV_OK;
+}
+
+int sdv_debug_force_commit_tree(sdv_ctx* ctx, const int32_t* host_path, int path_len, int32_t next_token) {
+    if (!ctx || path_len < 0 || (path_len && !host_path)) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->verified || !ctx->tree_verified) return SDV_ESTATE;
+    if (path_len + 1 > ctx->last_rows || next_token < 0 || next_token >= ctx->cfg.vocab) return SDV_EINVAL;
+    for (int i = 0; i < path_len; ++i)
+        if (host_path[i] < 1 || host_path[i] >= ctx->last_rows || (i && host_path[i] <= host_path[i - 1])) return SDV_EINVAL;
+    DraftArg p;
+    fill_draft_arg(p, host_path, path_len);
+    set_path_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, p, next_token);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    return commit_common(ctx, 0, -1, 0, nullptr, nullptr, nullptr);
+}
+
 int sdv_commit(sdv_ctx* ctx, int max_emit, int32_t* host_emitted, int* n_emitted, int* kv_len) {
     if (!ctx) return SDV_EINVAL;
     if (ctx->poisoned) return SDV_ETIMEOUT;
@@ -816,6 +969,8 @@ int sdv_rollback(sdv_ctx* ctx, int new_kv_len) {
     CK(cudaGetLastError());
     ctx->verified = false;
     ctx->draft_pending = false;
+    ctx->tree_pending = false;
+    ctx->tree_verified = false;
     CK(cudaStreamSynchronize(ctx->stream));
     return SDV_OK;
 }
@@ -862,6 +1017,8 @@ int sdv_debug_set_history(sdv_ctx* ctx, const int32_t* host_hist, int hist_len, 
     ctx->prefill_done = true;
     ctx->verified = false;
     ctx->draft_pending = false;
+    ctx->tree_pending = false;
+    ctx->tree_verified = false;
     CK(cudaStreamSynchronize(ctx->stream));
     return SDV_OK;
 }
@@ -874,6 +1031,7 @@ int sdv_debug_set_draft(sdv_ctx* ctx, const int32_t* host_draft, int draft_len) 
     ctx->launches++;
     CK(cudaGetLastError());
     ctx->draft_pending = true;
+    ctx->tree_pending = false;
     ctx->draft_k = draft_len;
     ctx->verified = false;
     return SDV_OK;
@@ -898,6 +1056,20 @@ int sdv_debug_accept(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, con
     int rc = read_state(ctx);
     if (rc) return rc;
     if (accept_len) *accept_len = ctx->pinned[ST_ACCEPT_LEN];
+    return SDV_OK;
+}
+
+int sdv_debug_top_successors(sdv_ctx* ctx, const float* host_logits, int rows, int top_b, int32_t* host_out) {
+    if (!ctx || !host_logits || !host_out || rows < 1 || rows > kMaxRows || top_b < 1 || top_b > SDV_CALIB_MAX)
+        return SDV_EINVAL;
+    const size_t V = ctx->cfg.vocab;
+    CK(cudaMemcpyAsync(ctx->ws + ctx->r.logits, host_logits, (size_t)rows * V * 4, cudaMemcpyDefault, ctx->stream));
+    int* out = (int*)(ctx->ws + ctx->r.xstage);  // scratch of the stand-alone GEMM: at least 32 * d floats
+    top_successors_kernel<<<rows, 1024, 0, ctx->stream>>>(ctx->P.logits, (int)V, top_b, out);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    CK(cudaMemcpyAsync(host_out, out, (size_t)rows * top_b * 4, cudaMemcpyDeviceToHost, ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
     return SDV_OK;
 }
 

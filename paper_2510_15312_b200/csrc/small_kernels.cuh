@@ -116,6 +116,7 @@ __global__ void ngram_draft_kernel(int* state, const int* hist, const int* db, i
             state[ST_SEG_USED] = 0;
             state[ST_MATCH_POS] = pos;
             state[ST_MATCH_LEN] = mlen;
+            state[ST_TREE_ON] = 0;
         }
     }
 }
@@ -136,6 +137,170 @@ __global__ void set_draft_kernel(int* state, DraftArg a) {
         state[ST_DRAFT_LEN] = a.n;
         state[ST_BASE_LEN] = a.n;
         state[ST_SEG_USED] = 0;
+        state[ST_TREE_ON] = 0;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Tree-structured drafts.  Row 0 is the committed token, draft node i is row i; ST_PARENT[i] < i is
+// the row it continues.  One thread derives what the forward pass reads: the depth of every row
+// (its position relative to the KV length) and the bit mask of the rows on its path from the root.
+// Rows past the tree (padding up to the launch's row count) hang off the root on their own.
+__device__ __forceinline__ void tree_finish(int* state, int n_nodes) {
+    state[ST_PARENT] = -1;
+    state[ST_DEPTH] = 0;
+    state[ST_ANC] = 1;
+    for (int j = 1; j < kMaxRows; ++j) {
+        int par = (j <= n_nodes) ? state[ST_PARENT + j] : 0;
+        if (par < 0 || par >= j) par = 0;
+        state[ST_PARENT + j] = par;
+        state[ST_DEPTH + j] = state[ST_DEPTH + par] + 1;
+        state[ST_ANC + j] = state[ST_ANC + par] | (int)(1u << j);
+    }
+    state[ST_TREE_ON] = 1;
+}
+
+// Caller-supplied tree: tokens of the draft nodes and, for node i (1-based), the row it continues.
+__global__ void set_tree_kernel(int* state, DraftArg tok, DraftArg par) {
+    if ((int)threadIdx.x < tok.n) {
+        state[ST_DRAFT + threadIdx.x] = tok.tok[threadIdx.x];
+        state[ST_PARENT + 1 + threadIdx.x] = par.tok[threadIdx.x];
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) {
+        state[ST_DRAFT_LEN] = tok.n;
+        state[ST_BASE_LEN] = tok.n;
+        state[ST_SEG_USED] = 0;
+        tree_finish(state, tok.n);
+    }
+}
+
+// In-context calibration, "Sample": the b best token ids of every logits row (largest logit first,
+// lowest id among equals: the greedy rule applied b times).  One block per row.
+__global__ void top_successors_kernel(const float* logits, int V, int b, int* succ /* [rows][b] */) {
+    __shared__ float bv_s[32];
+    __shared__ int bi_s[32];
+    __shared__ int taken[8];
+    const float* row = logits + (size_t)blockIdx.x * V;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    for (int r = 0; r < b; ++r) {
+        float bv = -CUDART_INF_F;
+        int bi = 0x7fffffff;
+        for (int i = threadIdx.x; i < V; i += blockDim.x) {
+            bool skip = false;
+            for (int t = 0; t < r; ++t) skip |= (taken[t] == i);
+            const float v = row[i];
+            if (!skip && (v > bv || (v == bv && i < bi))) { bv = v; bi = i; }
+        }
+        for (int off = 16; off; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        if (lane == 0) { bv_s[warp] = bv; bi_s[warp] = bi; }
+        __syncthreads();
+        if (warp == 0) {
+            bv = lane < nw ? bv_s[lane] : -CUDART_INF_F;
+            bi = lane < nw ? bi_s[lane] : 0x7fffffff;
+            for (int off = 16; off; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+            }
+            if (lane == 0) {
+                if (bi == 0x7fffffff) bi = 0;
+                taken[r] = bi;
+                succ[(size_t)blockIdx.x * b + r] = bi;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// "Search": where in the context each sampled successor occurs (the latest position; -1: nowhere).
+__global__ void anchor_search_kernel(const int* hist, int n_ctx, int b, const int* succ, int* occ) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= n_ctx * b) return;
+    const int tok = succ[idx];
+    int q = n_ctx - 1;
+    while (q >= 0 && hist[q] != tok) --q;
+    occ[idx] = q;
+}
+
+// Tree draft of one step: the retrieval chain the drafter left in the state block becomes one path;
+// then the calibrated tree of the committed token T: its sampled successors as children of the
+// root, each followed at once by its own successors where the anchor was matched in the context
+// (two levels, depth first).  A token a node already has as a child is not added twice; at most
+// max_nodes draft nodes.  One block: all threads look for the latest position of T in the context,
+// one thread builds.
+__global__ void tree_draft_kernel(int* state, const int* hist, const int* succ, const int* occ, int b, int max_nodes) {
+    __shared__ int best_s[32];
+    const int n_ctx = state[ST_N_CTX], T = state[ST_PENDING];
+    int best = -1;
+    for (int q = threadIdx.x; q < n_ctx; q += blockDim.x)
+        if (hist[q] == T) best = q;   // ascending per thread: the last hit is the thread's latest
+    for (int off = 16; off; off >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
+    if ((threadIdx.x & 31) == 0) best_s[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) best = max(best, best_s[w]);
+    const int p = best;
+    int n = state[ST_DRAFT_LEN];            // the chain: node i continues node i - 1
+    if (n > max_nodes) n = max_nodes;
+    for (int i = 1; i <= n; ++i) state[ST_PARENT + i] = i - 1;
+    auto add = [&](int node, int tok) -> int {
+        for (int c = 1; c <= n; ++c)
+            if (state[ST_PARENT + c] == node && state[ST_DRAFT + c - 1] == tok) return c;
+        if (n >= max_nodes) return -1;
+        ++n;
+        state[ST_DRAFT + n - 1] = tok;
+        state[ST_PARENT + n] = node;
+        return n;
+    };
+    if (p >= 0) {
+        for (int i = 0; i < b; ++i) {
+            const int c = add(0, succ[p * b + i]);
+            const int q = occ[p * b + i];
+            if (c >= 0 && q >= 0)
+                for (int i2 = 0; i2 < b; ++i2) add(c, succ[q * b + i2]);
+        }
+    }
+    state[ST_DRAFT_LEN] = n;
+    state[ST_BASE_LEN] = n;
+    state[ST_SEG_USED] = 0;
+    tree_finish(state, n);
+}
+
+// The accepted path given by the caller (teacher forcing in tests): emitted = its tokens + next_token.
+__global__ void set_path_kernel(int* state, DraftArg path, int next_token) {
+    if (threadIdx.x != 0) return;
+    for (int i = 0; i < path.n; ++i) {
+        state[ST_PATH + i] = path.tok[i];
+        state[ST_EMITTED + i] = state[ST_DRAFT + path.tok[i] - 1];
+    }
+    state[ST_EMITTED + path.n] = next_token;
+    state[ST_PATH_LEN] = path.n;
+    state[ST_ACCEPT_LEN] = path.n;
+    state[ST_N_EMITTED] = path.n + 1;
+}
+
+// Before the commit of a tree step: the accepted path's K/V rows, written at cache slots L + row,
+// move to the consecutive slots L + 1 .. L + a (ascending, sources never lie below their
+// destinations: a row's index is at least its depth).  Rows of emitted tokens that the commit will
+// cut off (max_emit) are not needed.  grid = (layers * KV heads, 2): K and V.
+__global__ void kv_compact_kernel(const int* state, __nv_bfloat16* kcache, __nv_bfloat16* vcache, int max_seq, int hd,
+                                  int max_emit) {
+    if (!state[ST_TREE_ON]) return;
+    const int L = state[ST_KV_LEN], a = state[ST_PATH_LEN];
+    int n = state[ST_N_EMITTED];
+    if (max_emit > 0 && n > max_emit) n = max_emit;
+    const int keep = min(a, n - 1);
+    __nv_bfloat16* base = (blockIdx.y ? vcache : kcache) + (size_t)blockIdx.x * max_seq * hd;
+    for (int i = 1; i <= keep; ++i) {
+        const int src = L + state[ST_PATH + i - 1], dst = L + i;
+        if (src != dst)
+            for (int e = threadIdx.x; e < hd; e += blockDim.x) base[(size_t)dst * hd + e] = base[(size_t)src * hd + e];
+        __syncthreads();
     }
 }
 // Caller-supplied predictions for the stand-alone accept scan.
@@ -242,9 +407,27 @@ __global__ void accept_kernel(int* state, const float* cand_val, const int* cand
     __syncthreads();
     if (threadIdx.x == 0) {
         int a = 0;
-        while (a < dl && state[ST_DRAFT + a] == y_s[a]) ++a;
-        for (int i = 0; i < a; ++i) state[ST_EMITTED + i] = state[ST_DRAFT + i];
-        state[ST_EMITTED + a] = y_s[a];
+        if (state[ST_TREE_ON]) {
+            // strict acceptance on a tree: step to the lowest-numbered child that carries the model's
+            // prediction at the current row, until no child does
+            int cur = 0;
+            for (;;) {
+                int nxt = -1;
+                for (int c = 1; c <= dl && nxt < 0; ++c)
+                    if (state[ST_PARENT + c] == cur && state[ST_DRAFT + c - 1] == y_s[cur]) nxt = c;
+                if (nxt < 0) break;
+                state[ST_PATH + a] = nxt;
+                state[ST_EMITTED + a] = state[ST_DRAFT + nxt - 1];
+                ++a;
+                cur = nxt;
+            }
+            state[ST_EMITTED + a] = y_s[cur];
+            state[ST_PATH_LEN] = a;
+        } else {
+            while (a < dl && state[ST_DRAFT + a] == y_s[a]) ++a;
+            for (int i = 0; i < a; ++i) state[ST_EMITTED + i] = state[ST_DRAFT + i];
+            state[ST_EMITTED + a] = y_s[a];
+        }
         state[ST_ACCEPT_LEN] = a;
         state[ST_N_EMITTED] = a + 1;
         state[ST_VERIFIED] = 1;
@@ -272,6 +455,7 @@ __global__ void commit_kernel(int* state, int* hist, int max_emit, int force_acc
     state[ST_PENDING] = state[ST_EMITTED + n - 1];
     state[ST_DRAFT_LEN] = 0;
     state[ST_VERIFIED] = 0;
+    state[ST_TREE_ON] = 0;
 }
 
 // After the last prefill tile: the greedy token of its last row becomes the pending token.
@@ -310,6 +494,7 @@ __global__ void set_state_kernel(int* state, int kv_len, int hist_len, int n_ctx
     if (pending_from_hist && hist_len > 0) state[ST_PENDING] = hist[hist_len - 1];
     state[ST_DRAFT_LEN] = 0;
     state[ST_VERIFIED] = 0;
+    state[ST_TREE_ON] = 0;
     state[ST_SEG_LEN] = 0;   // a new request starts without a retained segment
     state[ST_SEG_LIFE] = 0;
     state[ST_SEG_USED] = 0;
