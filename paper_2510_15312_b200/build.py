@@ -6,7 +6,7 @@ import subprocess
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsdv.so")
-_SOURCES = ["sdv.cu", "forward.cuh", "layout.cuh", "ptx.cuh", "small_kernels.cuh"]
+_SOURCES = ["sdv.cu", "forward.cuh", "dense.cuh", "layout.cuh", "ptx.cuh", "small_kernels.cuh"]
 
 
 HASH_PATH = LIB_PATH + ".srchash"

@@ -11,6 +11,7 @@
 #include <new>
 #include <vector>
 
+#include "dense.cuh"
 #include "forward.cuh"
 #include "layout.cuh"
 #include "small_kernels.cuh"
@@ -23,7 +24,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Regions {
     size_t state, bar, never, hist, db, rope, norm_w, bias, wlayers, wlm, emb, kcache, vcache, h, qkv_acc, sumsq, part_o,
-        part_ml, cand_val, cand_idx, logits, raw_out, staging, wraw, xstage, prof, succ, occ, total;
+        part_ml, cand_val, cand_idx, logits, raw_out, staging, wraw, xstage, prof, succ, occ, dw, dh, dxn, dqkv, dq, datt, dact, dtok, total;
     size_t layer_stride, staging_bytes, raw_kmax;
 };
 
@@ -92,6 +93,15 @@ Regions carve(const sdv_config* c) {
     r.raw_out = take((size_t)kMaxRows * (st / 128) * 4);  // N <= staging / (2 bytes * 64 columns)
     r.xstage = take((size_t)kMaxRows * raw_kmax * 4);
     r.prof = take((size_t)(3 + kPhasesPerLayer * c->n_layers) * kMaxGrid * kProfWords * 8);
+    // dense prefill path: row-major weight copies and the activations of one sub-chunk
+    r.dw = take(r.layer_stride * c->n_layers);
+    r.dh = take((size_t)kDenseMaxRows * d * 4);
+    r.dxn = take((size_t)kDenseMaxRows * d * 2);
+    r.dqkv = take((size_t)kDenseMaxRows * nqkv * 4);
+    r.dq = take((size_t)kDenseMaxRows * nq * 2);
+    r.datt = take((size_t)kDenseMaxRows * nq * 2);
+    r.dact = take((size_t)kDenseMaxRows * f * 2);
+    r.dtok = take((size_t)kDenseMaxRows * 4);
     r.succ = take((size_t)c->max_seq * SDV_CALIB_MAX * 4);  // calibration: sampled successors per context position
     r.occ = take((size_t)c->max_seq * SDV_CALIB_MAX * 4);   // and where each occurs in the context
     r.total = off;
@@ -257,6 +267,8 @@ struct sdv_ctx {
     long long launches;
     bool have_verify_time;
     bool poisoned;
+    std::vector<CUtensorMap>* maps;  // dense path: [0..2] activations (normalised rows, attention output, SwiGLU output), then 4 per layer
+    bool dense_ok;       // the tensor maps could be built (else every chunk takes the small-row path)
     int calib_b;         // successors sampled per context position during prefill (0: calibration off)
     bool calibrated;     // the calibration tables cover the whole context
     bool tree_pending;   // the device draft is a tree
@@ -409,6 +421,99 @@ int commit_common(sdv_ctx* ctx, int max_emit, int force_accept, int force_token,
     return SDV_OK;
 }
 
+// ---- dense prefill path (csrc/dense.cuh)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+// bf16 matrix [rows][K] row-major on this GPU; box = 128 rows x 64 columns, 128-byte swizzle, zeros outside.
+bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t K) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {K, rows};
+    const cuuint64_t strides[1] = {K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kDenseBK, (cuuint32_t)kDenseBM};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int EPI>
+cudaError_t launch_dense_gemm(sdv_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b, int M, int N, int K, float* out_f32, int ld_f32,
+                              const float* bias, __nv_bfloat16* out_bf16, int ld_bf16) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(dense_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDenseSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    dim3 grid((N + kDenseBN - 1) / kDenseBN, (M + kDenseBM - 1) / kDenseBM);
+    dense_gemm_kernel<EPI><<<grid, kDenseThreads, kDenseSmemBytes, ctx->stream>>>(a, b, M, N, K, out_f32, ld_f32, bias, out_bf16, ld_bf16,
+                                                                               ctx->P.state + ST_ERR, 2000000000ull);
+    ctx->launches++;
+    return cudaGetLastError();
+}
+
+// One sub-chunk of `rows` (32..256) context tokens at positions L..L+rows-1 through every layer:
+// fills their K/V rows.  The tokens are hist[L .. L+rows).
+int dense_prefill_rows(sdv_ctx* ctx, int rows, int L) {
+    const sdv_config& c = ctx->cfg;
+    const int d = c.d_model, f = c.d_ffn, hd = c.head_dim, nq = c.n_q_heads * hd, nkv = c.n_kv_heads * hd, nqkv = nq + 2 * nkv;
+    uint8_t* ws = ctx->ws;
+    cudaStream_t s = ctx->stream;
+    float* h = (float*)(ws + ctx->r.dh);
+    __nv_bfloat16* xn = (__nv_bfloat16*)(ws + ctx->r.dxn);
+    float* qkv = (float*)(ws + ctx->r.dqkv);
+    __nv_bfloat16* q = (__nv_bfloat16*)(ws + ctx->r.dq);
+    __nv_bfloat16* att = (__nv_bfloat16*)(ws + ctx->r.datt);
+    __nv_bfloat16* act = (__nv_bfloat16*)(ws + ctx->r.dact);
+    const int* hist = (const int*)(ws + ctx->r.hist);
+    const std::vector<CUtensorMap>& maps = *ctx->maps;
+    const float* norm_w = (const float*)(ws + ctx->r.norm_w);
+    const float* bias = c.qkv_bias ? (const float*)(ws + ctx->r.bias) : nullptr;
+    const size_t att_smem = (size_t)(64 * hd * 2 + 4 * 64 * hd * 2 + 128);
+    static bool att_attr = false;
+    if (!att_attr) {
+        CK(cudaFuncSetAttribute(dense_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 128 * 2 * 5 + 128));
+        CK(cudaFuncSetAttribute(dense_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 64 * 2 * 5 + 128));
+        att_attr = true;
+    }
+    dense_embed_kernel<<<rows, 128, 0, s>>>(hist + L, ctx->P.emb, h, d, c.vocab);
+    ctx->launches++;
+    for (int l = 0; l < c.n_layers; ++l) {
+        const CUtensorMap* mb = &maps[3 + 4 * l];
+        const size_t layer_off = (size_t)l * c.n_kv_heads * c.max_seq * hd;
+        dense_rmsnorm_kernel<<<rows, 256, 0, s>>>(h, norm_w + (size_t)(2 * l) * d, xn, d, c.rms_eps);
+        CK(launch_dense_gemm<EPI_STORE>(ctx, maps[0], mb[0], rows, nqkv, d, qkv, nqkv, bias ? bias + (size_t)l * nqkv : nullptr, nullptr, 0));
+        dense_rope_append_kernel<<<dim3(rows, c.n_q_heads + c.n_kv_heads), hd / 2, 0, s>>>(
+            qkv, nqkv, ctx->P.rope, q, c.n_q_heads, c.n_kv_heads, hd, ctx->P.kcache, ctx->P.vcache, layer_off, c.max_seq, L);
+        const dim3 ag(c.n_q_heads, (rows + 63) / 64);
+        if (hd == 128)
+            dense_attention_kernel<128><<<ag, 128, att_smem, s>>>(q, ctx->P.kcache, ctx->P.vcache, layer_off, c.max_seq, c.n_q_heads,
+                                                                   ctx->P.g, rows, L, ctx->P.scale_log2e, att);
+        else
+            dense_attention_kernel<64><<<ag, 128, att_smem, s>>>(q, ctx->P.kcache, ctx->P.vcache, layer_off, c.max_seq, c.n_q_heads,
+                                                                  ctx->P.g, rows, L, ctx->P.scale_log2e, att);
+        CK(launch_dense_gemm<EPI_RESIDUAL>(ctx, maps[1], mb[1], rows, d, nq, h, d, nullptr, nullptr, 0));
+        dense_rmsnorm_kernel<<<rows, 256, 0, s>>>(h, norm_w + (size_t)(2 * l + 1) * d, xn, d, c.rms_eps);
+        CK(launch_dense_gemm<EPI_SWIGLU>(ctx, maps[0], mb[2], rows, 2 * f, d, nullptr, 0, nullptr, act, f));
+        CK(launch_dense_gemm<EPI_RESIDUAL>(ctx, maps[2], mb[3], rows, d, f, h, d, nullptr, nullptr, 0));
+        ctx->launches += 4;  // norms, rotary + append, attention
+    }
+    CK(cudaGetLastError());
+    return SDV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -544,6 +649,20 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
     if (e != cudaSuccess) return fail(SDV_ECUDA);
+    // dense prefill path: tensor maps over its activation buffers and its weight copies
+    ctx->maps = new (std::nothrow) std::vector<CUtensorMap>(3 + 4 * (size_t)cfg->n_layers);
+    ctx->dense_ok = ctx->maps != nullptr;
+    if (ctx->dense_ok) {
+        std::vector<CUtensorMap>& m = *ctx->maps;
+        ctx->dense_ok = make_map(&m[0], ws + ctx->r.dxn, kDenseMaxRows, d) && make_map(&m[1], ws + ctx->r.datt, kDenseMaxRows, nq) &&
+                        make_map(&m[2], ws + ctx->r.dact, kDenseMaxRows, f);
+        for (int l = 0; l < cfg->n_layers && ctx->dense_ok; ++l) {
+            uint8_t* lb = ws + ctx->r.dw + (size_t)l * ctx->r.layer_stride;
+            const size_t o1 = (size_t)nqkv * d * 2, o2 = o1 + (size_t)d * nq * 2, o3 = o2 + (size_t)2 * f * d * 2;
+            ctx->dense_ok = make_map(&m[3 + 4 * l], lb, nqkv, d) && make_map(&m[4 + 4 * l], lb + o1, d, nq) &&
+                            make_map(&m[5 + 4 * l], lb + o2, 2 * (uint64_t)f, d) && make_map(&m[6 + 4 * l], lb + o3, d, f);
+        }
+    }
     *out = ctx;
     return SDV_OK;
 }
@@ -554,6 +673,7 @@ int sdv_destroy(sdv_ctx* ctx) {
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
     cudaEventDestroy(ctx->ev0);
     cudaEventDestroy(ctx->ev1);
+    delete ctx->maps;
     delete ctx;
     return SDV_OK;
 }
@@ -582,12 +702,16 @@ int sdv_load_weights(sdv_ctx* ctx, const sdv_weights* w) {
         rc = pack_op(ctx, ctx->P.op[OP_QKV], lbase + ctx->P.op[OP_QKV].w_off, stg, (int)nq, stg + nq * d, (int)nkv,
                      stg + (nq + nkv) * d, (int)d, 0, 0, ctx->P.op[OP_QKV].T, 0);
         if (rc) return rc;
+        // row-major copies for the dense prefill path: q|k|v, o, gate|up (interleaved by 64), down
+        uint16_t* dbase = (uint16_t*)(ws + ctx->r.dw + (size_t)l * ctx->r.layer_stride);
+        CK(cudaMemcpyAsync(dbase, stg, nqkv * d * 2, cudaMemcpyDeviceToDevice, s));
         CK(cudaStreamSynchronize(s));
         // o
         CK(cudaMemcpyAsync(stg, L.wo, d * nq * 2, cudaMemcpyDefault, s));
         rc = pack_op(ctx, ctx->P.op[OP_O], lbase + ctx->P.op[OP_O].w_off, stg, (int)d, nullptr, 0, nullptr, (int)nq, 0, 0,
                      ctx->P.op[OP_O].T, 0);
         if (rc) return rc;
+        CK(cudaMemcpyAsync(dbase + nqkv * d, stg, d * nq * 2, cudaMemcpyDeviceToDevice, s));
         CK(cudaStreamSynchronize(s));
         // gate | up, interleaved 8 + 8 rows per tile
         CK(cudaMemcpyAsync(stg, L.wg, f * d * 2, cudaMemcpyDefault, s));
@@ -595,12 +719,16 @@ int sdv_load_weights(sdv_ctx* ctx, const sdv_weights* w) {
         rc = pack_op(ctx, ctx->P.op[OP_GU], lbase + ctx->P.op[OP_GU].w_off, stg, (int)f, stg + f * d, (int)f, nullptr,
                      (int)d, 1, 0, ctx->P.op[OP_GU].T, 0);
         if (rc) return rc;
+        dense_copy_weights_kernel<<<148 * 8, 256, 0, s>>>(dbase + nqkv * d + d * nq, stg, stg + f * d, (int)(2 * f), (int)d, 1);
+        ctx->launches++;
+        CK(cudaGetLastError());
         CK(cudaStreamSynchronize(s));
         // down
         CK(cudaMemcpyAsync(stg, L.wd, d * f * 2, cudaMemcpyDefault, s));
         rc = pack_op(ctx, ctx->P.op[OP_DOWN], lbase + ctx->P.op[OP_DOWN].w_off, stg, (int)d, nullptr, 0, nullptr, (int)f,
                      0, 0, ctx->P.op[OP_DOWN].T, 0);
         if (rc) return rc;
+        CK(cudaMemcpyAsync(dbase + nqkv * d + d * nq + 2 * f * d, stg, d * f * 2, cudaMemcpyDeviceToDevice, s));
         CK(cudaStreamSynchronize(s));
         CK(cudaMemcpyAsync(norm_w + ((size_t)l * 2 + 0) * d, L.norm1, d * 4, cudaMemcpyDefault, s));
         CK(cudaMemcpyAsync(norm_w + ((size_t)l * 2 + 1) * d, L.norm2, d * 4, cudaMemcpyDefault, s));
@@ -660,6 +788,25 @@ int sdv_prefill_chunk(sdv_ctx* ctx, const int32_t* host_tokens, int n, int is_la
     const int n_ph = 1 + kPhasesPerLayer * c.n_layers;
     int done = 0;
     while (done < n) {
+        // sub-chunks of 32..256 rows go through the dense path (tokens on the tensor cores' M side, every weight
+        // streamed once); the last token of the request (its logits give the first generated token), short
+        // remainders and calibrated prefill (logits of every row) take the small-row kernel
+        const int dense_rows_avail = n - done - (is_last ? 1 : 0);
+        if (ctx->dense_ok && ctx->calib_b == 0 && dense_rows_avail >= 32) {
+            const int rows = dense_rows_avail < kDenseMaxRows ? dense_rows_avail : kDenseMaxRows;
+            int rc = dense_prefill_rows(ctx, rows, ctx->kv_len);
+            if (rc) return rc;
+            ctx->kv_len += rows;
+            ctx->hist_len += rows;
+            done += rows;
+            if (done == n) {   // the chunk ended here (never the last one: its final token takes the path below)
+                ctx->n_ctx = ctx->hist_len;
+                set_state_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, ctx->kv_len, ctx->hist_len, ctx->n_ctx, 0, hist);
+                ctx->launches++;
+                CK(cudaGetLastError());
+            }
+            continue;
+        }
         const int rows = (n - done < tile) ? n - done : tile;
         const bool last_tile = is_last && (done + rows == n);
         const bool calib = ctx->calib_b > 0;
