@@ -19,7 +19,8 @@ constexpr int kDenseBM = 128;      // token rows per tile (the instruction's M)
 constexpr int kDenseBN = 128;      // output features per tile (the instruction's N)
 constexpr int kDenseBK = 64;       // input features per stage: 64 bf16 = one 128-byte swizzled row
 constexpr int kDenseStages = 6;
-constexpr int kDenseStageBytes = (kDenseBM + kDenseBN) * kDenseBK * 2;   // 32 KB
+constexpr int kDenseTileBytes = kDenseBM * kDenseBK * 2;                 // one 128 x 64 operand tile: 16 KB
+constexpr int kDenseStageBytes = 2 * kDenseTileBytes;                    // a token tile + a weight tile: 32 KB
 constexpr int kDenseSmemBytes = kDenseStages * kDenseStageBytes + 1024 + 256;
 constexpr int kDenseThreads = 192;  // warp 0: copies, warp 1: tensor-core issue, warps 2..5: epilogue
 constexpr int kDenseMaxRows = 256;  // rows of the activation buffers (one sub-chunk)
@@ -55,6 +56,7 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
 //   EPI_RESIDUAL: out_f32[m][n] += C             (each element belongs to one tile: no atomics)
 //   EPI_SWIGLU:   the tile's columns 0..63 are gate features, 64..127 the matching up features:
 //                 out_bf16[m][64 * tile + c] = silu(gate) * up
+// gridDim.z > 1 splits K (EPI_STORE then needs a zeroed output; not for EPI_SWIGLU).
 // Rows >= M and columns >= N are computed on whatever the copies deliver (zeros outside the tensors)
 // and never written.  err: set to 1 when a bounded wait runs out.
 template <int EPI>
@@ -72,7 +74,12 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     Ctl* ctl = reinterpret_cast<Ctl*>(smem + kDenseStages * kDenseStageBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * kDenseBN, m0 = blockIdx.y * kDenseBM;
-    const int nkb = K / kDenseBK;
+    // split K: block z of gridDim.z takes an even share of the K/64 stages; partial sums then meet by fp32
+    // reductions in L2 (EPI_STORE: into a zeroed buffer, the bias added by share 0)
+    const int nkb_all = K / kDenseBK, nz = (int)gridDim.z, z = (int)blockIdx.z;
+    const int kb0 = even_start(nkb_all, nz, z), nkb = even_count(nkb_all, nz, z);
+    const bool split = nz > 1;
+    const int rot = nkb > 0 ? (int)((blockIdx.x * 5 + blockIdx.y * 11) % (unsigned)nkb) : 0;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kDenseStages; ++s) {
             mbar_init(&ctl->full[s], 1);
@@ -94,9 +101,12 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             for (int kb = 0; kb < nkb; ++kb) {
                 if (!mbar_wait_bounded(&ctl->empty[s], par ^ 1u, &ctl->abort_flag, wait_limit_ns)) break;
                 uint8_t* a = smem + s * kDenseStageBytes;
+                // blocks start their walk over K at different stages, so that at any moment they ask L2 for
+                // different parts of the activations they all share
+                const int kx = (kb0 + (kb + rot) % nkb) * kDenseBK;
                 mbar_arrive_expect_tx(&ctl->full[s], kDenseStageBytes);
-                tma_load_2d(a, &map_a, kb * kDenseBK, m0, &ctl->full[s]);
-                tma_load_2d(a + kDenseBM * kDenseBK * 2, &map_b, kb * kDenseBK, n0, &ctl->full[s]);
+                tma_load_2d(a, &map_a, kx, m0, &ctl->full[s]);
+                tma_load_2d(a + kDenseTileBytes, &map_b, kx, n0, &ctl->full[s]);
                 if (++s == kDenseStages) { s = 0; par ^= 1u; }
             }
         }
@@ -110,7 +120,7 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t a = smem_u32(smem + s * kDenseStageBytes);
-                const uint64_t da = umma_desc_sw128(a), db = umma_desc_sw128(a + kDenseBM * kDenseBK * 2);
+                const uint64_t da = umma_desc_sw128(a), db = umma_desc_sw128(a + kDenseTileBytes);
 #pragma unroll
                 for (int k4 = 0; k4 < kDenseBK / 16; ++k4)
                     umma_bf16(tmem, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), idesc, (uint32_t)(kb | k4));
@@ -159,13 +169,19 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
                         for (int i = 0; i < 16; i += 4) {
                             float4 o = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-                            if (EPI == EPI_RESIDUAL) {
-                                const float4 old = *reinterpret_cast<const float4*>(dst + c + i);
-                                o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
-                            } else if (bias) {
+                            if (EPI == EPI_STORE && bias && z == 0) {
                                 o.x += bias[n0 + c + i]; o.y += bias[n0 + c + i + 1]; o.z += bias[n0 + c + i + 2]; o.w += bias[n0 + c + i + 3];
                             }
-                            *reinterpret_cast<float4*>(dst + c + i) = o;
+                            if (split) {
+                                red_add_f32(dst + c + i, o.x); red_add_f32(dst + c + i + 1, o.y);
+                                red_add_f32(dst + c + i + 2, o.z); red_add_f32(dst + c + i + 3, o.w);
+                            } else {
+                                if (EPI == EPI_RESIDUAL) {
+                                    const float4 old = *reinterpret_cast<const float4*>(dst + c + i);
+                                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                                }
+                                *reinterpret_cast<float4*>(dst + c + i) = o;
+                            }
                         }
                     }
                 }
@@ -250,15 +266,18 @@ __global__ void dense_rope_append_kernel(const float* qkv, int n_qkv, const floa
 }
 
 // Causal attention of a sub-chunk's queries (rows r = 0..M-1 at positions L + r) over cache rows
-// 0 .. L + r of their KV head.  One block per (query head, 64-query tile); warp w owns 16 query
-// rows; keys in blocks of 64 through two shared-memory buffers; scores, online softmax (log2
-// domain) and P V in registers (mma.sync m16n8k16, the tiles are small).  Output bf16 [M][n_q * hd].
+// 0 .. L + r of their KV head.  One block per (query head, 16-query tile): many small blocks, since
+// a sub-chunk has few rows and the keys are the long dimension.  Keys come in blocks of 64 through
+// two shared-memory buffers; warp w takes the w-th group of 16 keys of every block: scores, online
+// softmax (log2 domain) and P V in its registers (mma.sync m16n8k16), and the four key groups meet in
+// shared memory at the end.  Output bf16 [M][n_q * hd].
 template <int HD>
 __global__ void __launch_bounds__(128) dense_attention_kernel(const __nv_bfloat16* q, const __nv_bfloat16* kcache,
                                                               const __nv_bfloat16* vcache, size_t layer_off, int max_seq, int n_q,
                                                               int g, int M, int L, float scale_log2e, __nv_bfloat16* out) {
-    constexpr int KSTEPS = HD / 16, UNITS = HD / 8, NT_O = HD / 8, KB = 64, QR = 64;
+    constexpr int KSTEPS = HD / 16, UNITS = HD / 8, NT_O = HD / 8, KB = 64, QR = 16;
     constexpr int QBYTES = QR * HD * 2, KVBYTES = KB * HD * 2;
+    static_assert(3 * (NT_O + 1) * 32 * 16 <= 4 * KVBYTES, "exchange area of the key-group merge");
     extern __shared__ uint8_t att_smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem_raw) + 127) & ~(uintptr_t)127);
     uint8_t* Qs = base;
@@ -293,7 +312,7 @@ __global__ void __launch_bounds__(128) dense_attention_kernel(const __nv_bfloat1
         *reinterpret_cast<uint4*>(Qs + (q16 >> 3) * (QR * 128) + swz_unit(r, q16 & 7)) = v;
     }
     const int gq = lane >> 2, q2 = (lane & 3) * 2;
-    const int r_lo = warp * 16 + gq, r_hi = r_lo + 8;
+    const int r_lo = gq, r_hi = gq + 8;
     float o[NT_O][4];
 #pragma unroll
     for (int n = 0; n < NT_O; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
@@ -304,67 +323,63 @@ __global__ void __launch_bounds__(128) dense_attention_kernel(const __nv_bfloat1
         cp_async_wait<1>();
         __syncthreads();
         const uint32_t kb = smem_u32(KVs + (blk & 1) * 2 * KVBYTES), vb = kb + KVBYTES;
-        if (blk * KB <= L + r0 + warp * 16 + 15) {   // some key of the block is visible to this warp's rows
-#pragma unroll 1
-            for (int c = 0; c < KB / 16; ++c) {
-                const int key0 = blk * KB + c * 16;
-                if (key0 > L + r0 + warp * 16 + 15) break;
-                float sc[2][4];
+        const int c = warp, key0 = blk * KB + c * 16;
+        if (key0 <= L + r0 + QR - 1) {   // some key of this group is visible to some row of the tile
+            float sc[2][4];
 #pragma unroll
-                for (int n = 0; n < 2; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
+            for (int n = 0; n < 2; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
 #pragma unroll
-                for (int ks = 0; ks < KSTEPS; ++ks) {
-                    uint32_t a0, a1, a2, a3, b0, b1, b2, b3;
-                    ldsm_x4(qb + (ks >> 2) * (QR * 128) + swz_unit(warp * 16 + (lane & 15), (ks & 3) * 2 + (lane >> 4)), a0, a1, a2, a3);
-                    const int krow = c * 16 + (lane & 7) + ((lane >> 4) << 3);
-                    ldsm_x4(kb + (ks >> 2) * (KB * 128) + swz_unit(krow, (ks & 3) * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
-                    mma_bf16_16816(sc[0], a0, a1, a2, a3, b0, b1);
-                    mma_bf16_16816(sc[1], a0, a1, a2, a3, b2, b3);
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+                uint32_t a0, a1, a2, a3, b0, b1, b2, b3;
+                ldsm_x4(qb + (ks >> 2) * (QR * 128) + swz_unit(lane & 15, (ks & 3) * 2 + (lane >> 4)), a0, a1, a2, a3);
+                const int krow = c * 16 + (lane & 7) + ((lane >> 4) << 3);
+                ldsm_x4(kb + (ks >> 2) * (KB * 128) + swz_unit(krow, (ks & 3) * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
+                mma_bf16_16816(sc[0], a0, a1, a2, a3, b0, b1);
+                mma_bf16_16816(sc[1], a0, a1, a2, a3, b2, b3);
+            }
+            float mx_lo = -CUDART_INF_F, mx_hi = -CUDART_INF_F;
+#pragma unroll
+            for (int n = 0; n < 2; ++n)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int key = key0 + n * 8 + q2 + (e & 1);
+                    const bool hi = e >= 2;
+                    const bool ok = key <= (hi ? lim_hi : lim_lo);
+                    const float v = ok ? sc[n][e] * scale_log2e : -CUDART_INF_F;
+                    sc[n][e] = v;
+                    if (hi) mx_hi = fmaxf(mx_hi, v); else mx_lo = fmaxf(mx_lo, v);
                 }
-                float mx_lo = -CUDART_INF_F, mx_hi = -CUDART_INF_F;
+            mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+            mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+            mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+            mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+            const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+            const float use_lo = (mn_lo == -CUDART_INF_F) ? 0.f : mn_lo, use_hi = (mn_hi == -CUDART_INF_F) ? 0.f : mn_hi;
+            const float c_lo = exp2f(m_lo - use_lo), c_hi = exp2f(m_hi - use_hi);
+            m_lo = mn_lo;
+            m_hi = mn_hi;
+            float p[2][4];
 #pragma unroll
-                for (int n = 0; n < 2; ++n)
+            for (int n = 0; n < 2; ++n) {
+                p[n][0] = exp2f(sc[n][0] - use_lo);
+                p[n][1] = exp2f(sc[n][1] - use_lo);
+                p[n][2] = exp2f(sc[n][2] - use_hi);
+                p[n][3] = exp2f(sc[n][3] - use_hi);
+            }
+            l_lo = l_lo * c_lo + p[0][0] + p[0][1] + p[1][0] + p[1][1];
+            l_hi = l_hi * c_hi + p[0][2] + p[0][3] + p[1][2] + p[1][3];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int key = key0 + n * 8 + q2 + (e & 1);
-                        const bool hi = e >= 2;
-                        const bool ok = key <= (hi ? lim_hi : lim_lo);
-                        const float v = ok ? sc[n][e] * scale_log2e : -CUDART_INF_F;
-                        sc[n][e] = v;
-                        if (hi) mx_hi = fmaxf(mx_hi, v); else mx_lo = fmaxf(mx_lo, v);
-                    }
-                mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
-                mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
-                mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
-                mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
-                const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
-                const float use_lo = (mn_lo == -CUDART_INF_F) ? 0.f : mn_lo, use_hi = (mn_hi == -CUDART_INF_F) ? 0.f : mn_hi;
-                const float c_lo = exp2f(m_lo - use_lo), c_hi = exp2f(m_hi - use_hi);
-                m_lo = mn_lo;
-                m_hi = mn_hi;
-                float p[2][4];
+            for (int n = 0; n < NT_O; ++n) { o[n][0] *= c_lo; o[n][1] *= c_lo; o[n][2] *= c_hi; o[n][3] *= c_hi; }
+            const uint32_t a0 = pack_bf16(p[0][0], p[0][1]), a1 = pack_bf16(p[0][2], p[0][3]);
+            const uint32_t a2 = pack_bf16(p[1][0], p[1][1]), a3 = pack_bf16(p[1][2], p[1][3]);
 #pragma unroll
-                for (int n = 0; n < 2; ++n) {
-                    p[n][0] = exp2f(sc[n][0] - use_lo);
-                    p[n][1] = exp2f(sc[n][1] - use_lo);
-                    p[n][2] = exp2f(sc[n][2] - use_hi);
-                    p[n][3] = exp2f(sc[n][3] - use_hi);
-                }
-                l_lo = l_lo * c_lo + p[0][0] + p[0][1] + p[1][0] + p[1][1];
-                l_hi = l_hi * c_hi + p[0][2] + p[0][3] + p[1][2] + p[1][3];
-#pragma unroll
-                for (int n = 0; n < NT_O; ++n) { o[n][0] *= c_lo; o[n][1] *= c_lo; o[n][2] *= c_hi; o[n][3] *= c_hi; }
-                const uint32_t a0 = pack_bf16(p[0][0], p[0][1]), a1 = pack_bf16(p[0][2], p[0][3]);
-                const uint32_t a2 = pack_bf16(p[1][0], p[1][1]), a3 = pack_bf16(p[1][2], p[1][3]);
-#pragma unroll
-                for (int cg = 0; cg < NT_O / 2; ++cg) {
-                    uint32_t b0, b1, b2, b3;
-                    const int key = c * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
-                    const int cu = cg * 2 + (lane >> 4);
-                    ldsm_x4_trans(vb + (cu >> 3) * (KB * 128) + swz_unit(key, cu & 7), b0, b1, b2, b3);
-                    mma_bf16_16816(o[2 * cg], a0, a1, a2, a3, b0, b1);
-                    mma_bf16_16816(o[2 * cg + 1], a0, a1, a2, a3, b2, b3);
-                }
+            for (int cg = 0; cg < NT_O / 2; ++cg) {
+                uint32_t b0, b1, b2, b3;
+                const int key = c * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+                const int cu = cg * 2 + (lane >> 4);
+                ldsm_x4_trans(vb + (cu >> 3) * (KB * 128) + swz_unit(key, cu & 7), b0, b1, b2, b3);
+                mma_bf16_16816(o[2 * cg], a0, a1, a2, a3, b0, b1);
+                mma_bf16_16816(o[2 * cg + 1], a0, a1, a2, a3, b2, b3);
             }
         }
         __syncthreads();
@@ -375,6 +390,41 @@ __global__ void __launch_bounds__(128) dense_attention_kernel(const __nv_bfloat1
     l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+    // the key groups of warps 1..3 meet warp 0's in shared memory (the K/V buffers are free now)
+    {
+        float4* ex_o = reinterpret_cast<float4*>(KVs);   // [warp - 1][output tile][lane]
+        float4* ex_ml = ex_o + 3 * NT_O * 32;            // [warp - 1][lane]
+        __syncthreads();
+        if (warp > 0) {
+            float4* dst = ex_o + (warp - 1) * NT_O * 32;
+#pragma unroll
+            for (int n = 0; n < NT_O; ++n) dst[n * 32 + lane] = make_float4(o[n][0], o[n][1], o[n][2], o[n][3]);
+            ex_ml[(warp - 1) * 32 + lane] = make_float4(m_lo, m_hi, l_lo, l_hi);
+        }
+        __syncthreads();
+        if (warp > 0) return;
+#pragma unroll 1
+        for (int og = 0; og < 3; ++og) {
+            const float4 ml = ex_ml[og * 32 + lane];
+            const float mn_lo = fmaxf(m_lo, ml.x), mn_hi = fmaxf(m_hi, ml.y);
+            const float use_lo = (mn_lo == -CUDART_INF_F) ? 0.f : mn_lo, use_hi = (mn_hi == -CUDART_INF_F) ? 0.f : mn_hi;
+            const float e0_lo = exp2f(m_lo - use_lo), e1_lo = exp2f(ml.x - use_lo);
+            const float e0_hi = exp2f(m_hi - use_hi), e1_hi = exp2f(ml.y - use_hi);
+            m_lo = mn_lo;
+            m_hi = mn_hi;
+            l_lo = l_lo * e0_lo + ml.z * e1_lo;
+            l_hi = l_hi * e0_hi + ml.w * e1_hi;
+            const float4* src = ex_o + og * NT_O * 32;
+#pragma unroll
+            for (int n = 0; n < NT_O; ++n) {
+                const float4 t = src[n * 32 + lane];
+                o[n][0] = o[n][0] * e0_lo + t.x * e1_lo;
+                o[n][1] = o[n][1] * e0_lo + t.y * e1_lo;
+                o[n][2] = o[n][2] * e0_hi + t.z * e1_hi;
+                o[n][3] = o[n][3] * e0_hi + t.w * e1_hi;
+            }
+        }
+    }
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
         const int r = half ? r_hi : r_lo;

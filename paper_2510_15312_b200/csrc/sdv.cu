@@ -457,7 +457,20 @@ cudaError_t launch_dense_gemm(sdv_ctx* ctx, const CUtensorMap& a, const CUtensor
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    dim3 grid((N + kDenseBN - 1) / kDenseBN, (M + kDenseBM - 1) / kDenseBM);
+    dim3 grid((N + kDenseBN - 1) / kDenseBN, (M + kDenseBM - 1) / kDenseBM, 1);
+    if (EPI != EPI_SWIGLU) {
+        // few tiles and a long K (the down projection): split K so that about one block per SM runs; every share
+        // keeps at least 16 stages, below that the partial-sum reductions cost more than the idle SMs
+        const int tiles = (int)(grid.x * grid.y), nkb = K / kDenseBK;
+        int sp = ctx->G / tiles;
+        if (sp > nkb / 16) sp = nkb / 16;
+        if (sp < 1) sp = 1;
+        grid.z = (unsigned)sp;
+        if (EPI == EPI_STORE && sp > 1) {
+            cudaError_t e = cudaMemsetAsync(out_f32, 0, (size_t)M * ld_f32 * 4, ctx->stream);
+            if (e != cudaSuccess) return e;
+        }
+    }
     dense_gemm_kernel<EPI><<<grid, kDenseThreads, kDenseSmemBytes, ctx->stream>>>(a, b, M, N, K, out_f32, ld_f32, bias, out_bf16, ld_bf16,
                                                                                ctx->P.state + ST_ERR, 2000000000ull);
     ctx->launches++;
@@ -481,11 +494,11 @@ int dense_prefill_rows(sdv_ctx* ctx, int rows, int L) {
     const std::vector<CUtensorMap>& maps = *ctx->maps;
     const float* norm_w = (const float*)(ws + ctx->r.norm_w);
     const float* bias = c.qkv_bias ? (const float*)(ws + ctx->r.bias) : nullptr;
-    const size_t att_smem = (size_t)(64 * hd * 2 + 4 * 64 * hd * 2 + 128);
+    const size_t att_smem = (size_t)(16 * hd * 2 + 4 * 64 * hd * 2 + 128);  // query tile + two K|V blocks
     static bool att_attr = false;
     if (!att_attr) {
-        CK(cudaFuncSetAttribute(dense_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 128 * 2 * 5 + 128));
-        CK(cudaFuncSetAttribute(dense_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 64 * 2 * 5 + 128));
+        CK(cudaFuncSetAttribute(dense_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 128 * 2 + 4 * 64 * 128 * 2 + 128));
+        CK(cudaFuncSetAttribute(dense_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 64 * 2 + 4 * 64 * 64 * 2 + 128));
         att_attr = true;
     }
     dense_embed_kernel<<<rows, 128, 0, s>>>(hist + L, ctx->P.emb, h, d, c.vocab);
@@ -497,7 +510,7 @@ int dense_prefill_rows(sdv_ctx* ctx, int rows, int L) {
         CK(launch_dense_gemm<EPI_STORE>(ctx, maps[0], mb[0], rows, nqkv, d, qkv, nqkv, bias ? bias + (size_t)l * nqkv : nullptr, nullptr, 0));
         dense_rope_append_kernel<<<dim3(rows, c.n_q_heads + c.n_kv_heads), hd / 2, 0, s>>>(
             qkv, nqkv, ctx->P.rope, q, c.n_q_heads, c.n_kv_heads, hd, ctx->P.kcache, ctx->P.vcache, layer_off, c.max_seq, L);
-        const dim3 ag(c.n_q_heads, (rows + 63) / 64);
+        const dim3 ag(c.n_q_heads, (rows + 15) / 16);
         if (hd == 128)
             dense_attention_kernel<128><<<ag, 128, att_smem, s>>>(q, ctx->P.kcache, ctx->P.vcache, layer_off, c.max_seq, c.n_q_heads,
                                                                    ctx->P.g, rows, L, ctx->P.scale_log2e, att);
