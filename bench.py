@@ -40,6 +40,15 @@ NCU_TRAFFIC_RATIO = 1.0051
 NOMINAL_HBM_GBS = 8000.0   # the "about 8 TB/s" the target is worded against
 
 
+def load_tflops():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return float(p.get("bf16_tflops_sustained", p.get("bf16_tflops", 1400.0))), "measured"
+    return 1400.0, "fallback"
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -417,7 +426,7 @@ def main():
                "accepted_drafts_per_step": tokens_x / args.steps - 1.0, "scope": "rank 0"}
 
     # ---- the two other labelled throughput numbers (single-GPU runs only; synthetic acceptance)
-    forced = hist_mode = None
+    forced = hist_mode = prefill = None
     if extras and world == 1:
         # (C) forced acceptance.  The greedy continuation comes from this path's own plain decoding (one token
         # per step, no oracle involved), recorded before the timed region; each timed step then verifies a
@@ -455,12 +464,30 @@ def main():
                   "value": toks_f / (ms_f * 1e-3), "unit": UNIT, "ms_per_step": ms_f / args.steps,
                   "emitted_per_step": toks_f / args.steps, "steps_with_the_forced_accept_length": hits,
                   "verify_kernel_us": statistics.mean(kms_f) * 1e3}
-        # (B) the drafter also searches the generated tokens (search_history): a second context of the same model
+        # (B) the drafter also searches the generated tokens (search_history): a second context of the same model;
+        # its prefill is the timed prefill number
+        # chunked prefill of the whole context on a fresh context: the dense path (tokens on the tensor cores' M side)
         s.close()
         s = Sdv(config_from(cfg, k_max=k_max, max_seq=max_seq, search_history=True), stream=stream)
         s.load_weights(w)
+        torch.cuda.synchronize()
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = s.launch_count()
+        p0.record(stream)
         for i in range(0, cfg.n_ctx, cfg.chunk):
             s.prefill_chunk(ctx[i:i + cfg.chunk], is_last=(i + cfg.chunk >= cfg.n_ctx))
+        p1.record(stream)
+        torch.cuda.synchronize()
+        ms_p = p0.elapsed_time(p1)
+        lin = 2.0 * (cfg.linear_params() - cfg.vocab * cfg.d_model) * cfg.n_ctx   # the LM head runs on the last row only
+        att = 4.0 * cfg.n_layers * cfg.n_q_heads * cfg.head_dim * (cfg.n_ctx * (cfg.n_ctx + 1) / 2.0)
+        tf = load_tflops()
+        prefill = {"label": f"chunked prefill of the {cfg.n_ctx}-token context in {cfg.chunk}-token chunks (host loop included: "
+                            "one call per chunk, each synchronises)",
+                   "ms": ms_p, "tokens_per_sec": cfg.n_ctx / (ms_p * 1e-3), "launches": s.launch_count() - l0,
+                   "tflops_linear": lin / (ms_p * 1e-3) / 1e12, "tflops_linear_plus_attention": (lin + att) / (ms_p * 1e-3) / 1e12,
+                   "bf16_peak_tflops": tf[0], "peak_kind": f"of {tf[1]} (sustained)",
+                   "frac": (lin + att) / (ms_p * 1e-3) / 1e12 / tf[0]}
         loop(args.warmup, False)
         torch.cuda.synchronize()
         h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -511,6 +538,7 @@ def main():
             line["forced_acceptance"] = forced
         if hist_mode:
             line["history"] = hist_mode
+            line["prefill"] = prefill
         if ext:
             line["extension"] = ext
         if sweep:

@@ -546,7 +546,7 @@ __device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps)
     S = (P.L + kps - 1) / kps;
 }
 
-template <int HD>
+template <int HD, bool TREE>   // TREE: the new rows form a tree (positions and visibility from the state block), else a chain
 __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int hk, int qg, int gh, int s, int S, int kps, uint8_t* att,
                                             int wtid, unsigned long long* prof) {
     constexpr int HD2 = HD / 2;
@@ -627,7 +627,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
                     ssq[t] = __ldcg(sumsq + j);
                     qa[t] = ld_cg_f4_inorder(P.qkv_acc + (size_t)j * P.n_qkv + col);
                     qb[t] = ld_cg_f4_inorder(P.qkv_acc + (size_t)j * P.n_qkv + col + HD2);
-                    const int pj = P.tree ? __ldcg(P.state + ST_DEPTH + j) : j;  // tree drafts: a row's position is its depth
+                    const int pj = TREE ? __ldcg(P.state + ST_DEPTH + j) : j;  // tree drafts: a row's position is its depth
                     const float4* rp = reinterpret_cast<const float4*>(P.rope + (size_t)(L + pj) * HD2 + ii[t]);
                     c0[t] = ld_nc_f4_inorder(rp);
                     c1[t] = ld_nc_f4_inorder(rp + 1);
@@ -677,7 +677,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
                 const float4 a0 = ldcg_f4(pa), a1 = ldcg_f4(pa + 4), b0 = ldcg_f4(pa + HD2), b1 = ldcg_f4(pa + HD2 + 4);
                 const float* pv = accrow + Nq + Nkv + hk * HD + colb;
                 const float4 v0 = ldcg_f4(pv), v1 = ldcg_f4(pv + 4);
-                const int pk = P.tree ? __ldcg(P.state + ST_DEPTH + kk) : kk;
+                const int pk = TREE ? __ldcg(P.state + ST_DEPTH + kk) : kk;
                 const float4* rp = reinterpret_cast<const float4*>(P.rope + (size_t)(L + pk) * HD2 + ib);
                 const float4 r0 = __ldg(rp), r1 = __ldg(rp + 1), r2 = __ldg(rp + 2), r3 = __ldg(rp + 3);
                 float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
@@ -717,8 +717,9 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
     const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
     const int j_lo = r_lo % M, j_hi = r_hi % M;
     // new keys a row may see: rows 0..j of a chain, its own path from the root in a tree
-    const unsigned see_lo = !is_new ? 0xffffffffu : (P.tree ? (unsigned)__ldcg(P.state + ST_ANC + j_lo) : (0xffffffffu >> (31 - j_lo)));
-    const unsigned see_hi = !is_new ? 0xffffffffu : (P.tree ? (unsigned)__ldcg(P.state + ST_ANC + j_hi) : (0xffffffffu >> (31 - j_hi)));
+    const bool tree_mask = TREE && is_new;
+    const unsigned see_lo = tree_mask ? (unsigned)__ldcg(P.state + ST_ANC + j_lo) : 0u;
+    const unsigned see_hi = tree_mask ? (unsigned)__ldcg(P.state + ST_ANC + j_hi) : 0u;
     float o[NT_O][4];
 #pragma unroll
     for (int n = 0; n < NT_O; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
@@ -753,8 +754,9 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
                     for (int e = 0; e < 4; ++e) {
                         const int key = blk * KB + c * 16 + n * 8 + q2 + (e & 1);
                         const bool hi = e >= 2;
-                        const int row = hi ? r_hi : r_lo;
-                        const bool ok = key < nkeys && row < R && (!is_new || (((hi ? see_hi : see_lo) >> (key & 31)) & 1u));
+                        const int row = hi ? r_hi : r_lo, j = hi ? j_hi : j_lo;
+                        bool ok = key < nkeys && row < R && (!is_new || key <= j);
+                        if (TREE && tree_mask) ok = key < nkeys && row < R && (((hi ? see_hi : see_lo) >> (key & 31)) & 1u);
                         const float v = ok ? sc[n][e] * P.scale_log2e : -CUDART_INF_F;
                         sc[n][e] = v;
                         if (hi) mx_hi = fmaxf(mx_hi, v); else mx_lo = fmaxf(mx_lo, v);
@@ -866,8 +868,13 @@ __device__ void attention_phase(const FwdParams& P, int layer, uint8_t* att, int
     const int nunits = P.n_kv * QG * S1;
     for (int unit = blockIdx.x; unit < nunits; unit += P.G) {
         const int hk = unit / (QG * S1), rem = unit % (QG * S1), qg = rem / S1, s = rem % S1;
-        if (P.hd == 128) attention_unit<128>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof);
-        else attention_unit<64>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof);
+        if (P.tree) {
+            if (P.hd == 128) attention_unit<128, true>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof);
+            else attention_unit<64, true>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof);
+        } else {
+            if (P.hd == 128) attention_unit<128, false>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof);
+            else attention_unit<64, false>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof);
+        }
         named_bar_sync(1, kWorkerThreads);  // the unit's shared-memory tiles are free again
         if (prof && wtid == 0) { prof[6] = global_timer_ns(); prof[7] = (unsigned long long)(s == S); }
     }
