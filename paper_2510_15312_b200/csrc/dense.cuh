@@ -130,36 +130,73 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             if (ok) umma_commit(&ctl->acc_full);
         }
     } else {
-        // epilogue: warp w reads accumulator lanes 32 * (w % 4) .. + 31; lane = token row of the tile
+        // epilogue: warp w reads accumulator lanes 32 * (w % 4) .. + 31 (lane = token row of the tile), 32 columns
+        // at a time, and turns them round through shared memory (the ring is free once the accumulator is
+        // complete) so that one warp instruction touches 32 consecutive values of one output row: full 128-byte
+        // lines for the stores, the residual read-modify-write and the partial-sum reductions alike
         const int q = warp & 3;
-        const int row = m0 + q * 32 + lane;
+        const int row0 = m0 + q * 32;
         const bool got = mbar_wait_bounded(&ctl->acc_full, 0, &ctl->abort_flag, wait_limit_ns);
         const bool all_got = __all_sync(0xffffffffu, got);
         if (all_got) {
             tc_fence_after();
             const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16);
+            float* stage = reinterpret_cast<float*>(smem + q * 8192);   // [32 rows][33]: this warp's turning area
             if (EPI == EPI_SWIGLU) {
-                __nv_bfloat16* dst = out_bf16 + (size_t)row * ld_bf16 + (n0 / 2);
+                // columns 0..63 gate, 64..127 up: 16 + 16 at a time -> 16 bf16 outputs per row, staged as bf16
+                // [32 rows][64 columns (+ 8 pad)] and written as four rows of 128 bytes per instruction
+                __nv_bfloat16* st16 = reinterpret_cast<__nv_bfloat16*>(stage);
 #pragma unroll 1
                 for (int c = 0; c < kDenseBN / 2; c += 16) {
                     float g[16], u[16];
                     tmem_ld16(taddr + (uint32_t)c, g);
                     tmem_ld16(taddr + (uint32_t)(kDenseBN / 2 + c), u);
-                    if (row < M) {
-                        uint32_t pk[8];
+                    uint32_t pk[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const float a0 = __fdividef(g[2 * i], 1.f + __expf(-g[2 * i])) * u[2 * i];
-                            const float a1 = __fdividef(g[2 * i + 1], 1.f + __expf(-g[2 * i + 1])) * u[2 * i + 1];
-                            pk[i] = pack_bf16(a0, a1);
-                        }
-                        if (n0 / 2 + c + 16 <= N / 2) {
-                            *reinterpret_cast<uint4*>(dst + c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                            *reinterpret_cast<uint4*>(dst + c + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-                        }
+                    for (int i = 0; i < 8; ++i) {
+                        const float a0 = __fdividef(g[2 * i], 1.f + __expf(-g[2 * i])) * u[2 * i];
+                        const float a1 = __fdividef(g[2 * i + 1], 1.f + __expf(-g[2 * i + 1])) * u[2 * i + 1];
+                        pk[i] = pack_bf16(a0, a1);
+                    }
+                    uint4* d4 = reinterpret_cast<uint4*>(st16 + lane * 72 + c);
+                    d4[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    d4[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                }
+                __syncwarp();
+#pragma unroll 1
+                for (int r = lane >> 3; r < 32; r += 4) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(st16 + r * 72 + (lane & 7) * 8);
+                    if (row0 + r < M)
+                        *reinterpret_cast<uint4*>(out_bf16 + (size_t)(row0 + r) * ld_bf16 + n0 / 2 + (lane & 7) * 8) = v;
+                }
+            } else if (split) {
+                // partial sums of a K share: turned round through shared memory so that one warp instruction adds
+                // 32 consecutive values of one output row (full lines for the reductions in L2)
+#pragma unroll 1
+                for (int c = 0; c < kDenseBN; c += 32) {
+                    float v[32];
+                    {
+                        float lo[16], hi[16];
+                        tmem_ld16(taddr + (uint32_t)c, lo);
+                        tmem_ld16(taddr + (uint32_t)(c + 16), hi);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) { v[i] = lo[i]; v[16 + i] = hi[i]; }
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) stage[lane * 33 + i] = v[i];
+                    __syncwarp();
+                    const int col = n0 + c + lane;
+                    if (col < N) {
+                        const float b = (EPI == EPI_STORE && bias && z == 0) ? bias[col] : 0.f;
+                        float* dst = out_f32 + (size_t)row0 * ld_f32 + col;
+                        const int nr = min(32, M - row0);
+                        for (int r = 0; r < nr; ++r) red_add_f32(dst + (size_t)r * ld_f32, stage[r * 33 + lane] + b);
                     }
                 }
             } else {
+                // one block per output element: plain stores, or read-add-write of the residual, 16 bytes at a time
+                const int row = row0 + lane;
                 float* dst = out_f32 + (size_t)row * ld_f32 + n0;
 #pragma unroll 1
                 for (int c = 0; c < kDenseBN; c += 16) {
@@ -169,19 +206,14 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
                         for (int i = 0; i < 16; i += 4) {
                             float4 o = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-                            if (EPI == EPI_STORE && bias && z == 0) {
+                            if (EPI == EPI_STORE && bias) {
                                 o.x += bias[n0 + c + i]; o.y += bias[n0 + c + i + 1]; o.z += bias[n0 + c + i + 2]; o.w += bias[n0 + c + i + 3];
                             }
-                            if (split) {
-                                red_add_f32(dst + c + i, o.x); red_add_f32(dst + c + i + 1, o.y);
-                                red_add_f32(dst + c + i + 2, o.z); red_add_f32(dst + c + i + 3, o.w);
-                            } else {
-                                if (EPI == EPI_RESIDUAL) {
-                                    const float4 old = *reinterpret_cast<const float4*>(dst + c + i);
-                                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
-                                }
-                                *reinterpret_cast<float4*>(dst + c + i) = o;
+                            if (EPI == EPI_RESIDUAL) {
+                                const float4 old = *reinterpret_cast<const float4*>(dst + c + i);
+                                o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
                             }
+                            *reinterpret_cast<float4*>(dst + c + i) = o;
                         }
                     }
                 }

@@ -460,10 +460,10 @@ cudaError_t launch_dense_gemm(sdv_ctx* ctx, const CUtensorMap& a, const CUtensor
     dim3 grid((N + kDenseBN - 1) / kDenseBN, (M + kDenseBM - 1) / kDenseBM, 1);
     if (EPI != EPI_SWIGLU) {
         // few tiles and a long K (the down projection): split K so that about one block per SM runs; every share
-        // keeps at least 16 stages, below that the partial-sum reductions cost more than the idle SMs
+        // keeps at least six stages
         const int tiles = (int)(grid.x * grid.y), nkb = K / kDenseBK;
         int sp = ctx->G / tiles;
-        if (sp > nkb / 16) sp = nkb / 16;
+        if (sp > nkb / 6) sp = nkb / 6;
         if (sp < 1) sp = 1;
         grid.z = (unsigned)sp;
         if (EPI == EPI_STORE && sp > 1) {
