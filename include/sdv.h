@@ -135,6 +135,39 @@ int sdv_set_database(sdv_ctx *ctx, const int32_t *host_tokens, int n);
  * Errors: SDV_ESTATE before prefill has finished, SDV_ECAPACITY, SDV_EINVAL, SDV_ETIMEOUT. */
 int sdv_verify(sdv_ctx *ctx, const int32_t *host_draft, int draft_len, int32_t *host_y, int *accept_len);
 
+/* Batched verify: several sequences share one pass over the weights.  The paper verifies one request at
+ * a time; its utilisation argument (Sec. 2: the matrix units need a large batch or a long sequence per
+ * weight read) is what this call applies across requests, and every sequence's result is what sdv_verify
+ * on that sequence alone computes.
+ *
+ * sdv_follower_workspace_bytes / sdv_create_follower: a further sequence that reads `leader`'s weights
+ * (the leader owns its weights, has loaded them and must outlive its followers).  The follower has the
+ * leader's configuration and stream, its own KV cache, history and state in dev_workspace (256-byte
+ * aligned, at least sdv_follower_workspace_bytes(cfg) bytes, owned by the caller), and takes every call
+ * except sdv_load_weights and sdv_debug_gemm (SDV_ESTATE).  Errors: SDV_EINVAL (NULL, a leader that is
+ * itself a follower, alignment), SDV_ESTATE (leader without weights), SDV_ENOMEM, SDV_ECUDA.
+ *
+ * sdv_verify_batch: one verify step over ctxs[0..n) (1 <= n <= 8, distinct, a leader and followers of it
+ * or followers of one leader).  Each sequence contributes the rows sdv_verify(ctx, NULL, ...) would
+ * compute for it: its pending token and, after sdv_draft / sdv_extend_draft, its chain draft (k + 1 rows);
+ * the rows of all sequences together may not exceed 32.  The decoder runs once over all rows, every row
+ * attending to its own sequence's KV cache and earlier rows only, each sequence's KV rows are written
+ * speculatively into its own cache, and the accept scan runs per sequence; afterwards every context
+ * is in the state sdv_verify leaves it in (sdv_commit, sdv_extension_update, sdv_get_logits per context).
+ * The step runs on the scratch buffers of ctxs[0], whose sdv_last_verify_ms then times it.
+ * accept_len (n ints) may be NULL; if given the stream is synchronised.
+ * Errors: SDV_EINVAL (count, duplicates, unrelated contexts, more than 32 rows), SDV_ESTATE (a sequence
+ * before the end of prefill, or with a tree draft pending), SDV_ECAPACITY, SDV_ETIMEOUT. */
+/* Result of the outstanding verify step of one context (after sdv_verify, sdv_verify_tree or
+ * sdv_verify_batch, before the commit): the greedy token of each of its rows into host_y (k_max + 1 ints
+ * are always enough) and the accept length; either may be NULL.  Synchronises.  Errors: SDV_ESTATE when
+ * no verify result is outstanding, SDV_ETIMEOUT. */
+int sdv_get_verified(sdv_ctx *ctx, int32_t *host_y, int *accept_len);
+
+size_t sdv_follower_workspace_bytes(const sdv_config *cfg);
+int sdv_create_follower(sdv_ctx *leader, void *dev_workspace, size_t bytes, sdv_ctx **out);
+int sdv_verify_batch(sdv_ctx *const *ctxs, int n, int *accept_len);
+
 /* Draft extension (paper Sec. 4.4 "Reuse strategy", Eq. 3): drafts rejected by one verify step
  * are kept when they agree with the model's own predictions and are appended to later drafts.
  *

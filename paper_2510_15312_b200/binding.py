@@ -21,6 +21,7 @@ EXPORTS = [
     "sdv_gemm_noalloc", "sdv_debug_layout_check", "sdv_debug_plan",
     "sdv_set_calibration", "sdv_get_calibration", "sdv_draft_tree", "sdv_verify_tree", "sdv_debug_force_commit_tree",
     "sdv_debug_top_successors",
+    "sdv_follower_workspace_bytes", "sdv_create_follower", "sdv_verify_batch", "sdv_get_verified",
 ]
 
 
@@ -76,6 +77,11 @@ def load_library(path: Optional[str] = None):
     L.sdv_set_parity_mode.argtypes = [vp, C.c_int]
     L.sdv_get_logits.argtypes = [vp, vp, C.c_int]
     L.sdv_destroy.argtypes = [vp]
+    L.sdv_follower_workspace_bytes.argtypes = [C.POINTER(SdvConfig)]
+    L.sdv_follower_workspace_bytes.restype = C.c_size_t
+    L.sdv_create_follower.argtypes = [vp, vp, C.c_size_t, C.POINTER(vp)]
+    L.sdv_verify_batch.argtypes = [C.POINTER(vp), C.c_int, ip]
+    L.sdv_get_verified.argtypes = [vp, i32p, ip]
     L.sdv_strerror.argtypes = [C.c_int]
     L.sdv_strerror.restype = C.c_char_p
     L.sdv_last_cuda_error.argtypes = [vp]
@@ -101,7 +107,7 @@ def load_library(path: Optional[str] = None):
     L.sdv_debug_force_commit_tree.argtypes = [vp, i32p, C.c_int, C.c_int]
     L.sdv_debug_top_successors.argtypes = [vp, vp, C.c_int, C.c_int, vp]
     for name in EXPORTS:
-        if name not in ("sdv_workspace_bytes", "sdv_strerror", "sdv_launch_count"):
+        if name not in ("sdv_workspace_bytes", "sdv_follower_workspace_bytes", "sdv_strerror", "sdv_launch_count"):
             getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -130,13 +136,16 @@ def _ptr(a):
 class Sdv:
     """One sequence on the current CUDA device.  Owns the torch workspace tensor."""
 
-    def __init__(self, cconfig: SdvConfig, stream=None):
+    def __init__(self, cconfig: SdvConfig, stream=None, leader: Optional["Sdv"] = None):
+        """leader: another Sdv whose weights this sequence reads (it then needs no load_weights and can
+        join the leader in verify_batch); the leader must stay open while its followers are in use."""
         import torch
         if not torch.cuda.is_available():
             raise SdvError(ECUDA, "Sdv: no CUDA device (there is no CPU fallback)")
         L = lib()
         self.cfg = cconfig
-        nbytes = L.sdv_workspace_bytes(C.byref(cconfig))
+        self._leader = leader
+        nbytes = L.sdv_workspace_bytes(C.byref(cconfig)) if leader is None else L.sdv_follower_workspace_bytes(C.byref(cconfig))
         if nbytes == 0:
             raise SdvError(EINVAL, "sdv_workspace_bytes")
         self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
@@ -145,9 +154,16 @@ class Sdv:
         sp = None if stream is None else stream.cuda_stream
         h = C.c_void_p()
         self._h = None
-        self._check(L.sdv_create(C.byref(cconfig), base, nbytes, sp, C.byref(h)), "sdv_create", ctx=None)
+        if leader is None:
+            self._check(L.sdv_create(C.byref(cconfig), base, nbytes, sp, C.byref(h)), "sdv_create", ctx=None)
+        else:
+            self._check(L.sdv_create_follower(leader._h, base, nbytes, C.byref(h)), "sdv_create_follower", ctx=None)
         self._h = h
         self.workspace_bytes = nbytes
+
+    def follower(self) -> "Sdv":
+        """A further sequence on this one's weights (same configuration and stream)."""
+        return Sdv(self.cfg, stream=self._stream, leader=self)
 
     # -- helpers
     def _check(self, rc: int, where: str, ctx="self"):
@@ -201,6 +217,22 @@ class Sdv:
         y = np.zeros(K_MAX + 1, dtype=np.int32)
         a = C.c_int(0)
         self._check(lib().sdv_verify(self._h, dp, dl, y.ctypes.data, C.byref(a)), "sdv_verify")
+        return y, a.value
+
+    @staticmethod
+    def verify_batch(seqs: Sequence["Sdv"], fetch: bool = True) -> Optional[List[int]]:
+        """One verify step over several sequences that share weights (each after its own draft());
+        returns their accept lengths when fetch.  Commit each sequence afterwards."""
+        hs = (C.c_void_p * len(seqs))(*[q._h for q in seqs])
+        a = (C.c_int * len(seqs))()
+        seqs[0]._check(lib().sdv_verify_batch(hs, len(seqs), a if fetch else None), "sdv_verify_batch")
+        return list(a) if fetch else None
+
+    def get_verified(self) -> Tuple[np.ndarray, int]:
+        """(y, accept_len) of the outstanding verify step of this sequence."""
+        y = np.zeros(K_MAX + 1, dtype=np.int32)
+        a = C.c_int(0)
+        self._check(lib().sdv_get_verified(self._h, y.ctypes.data, C.byref(a)), "sdv_get_verified")
         return y, a.value
 
     def set_database(self, tokens):

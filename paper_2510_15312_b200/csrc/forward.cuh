@@ -546,9 +546,12 @@ __device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps)
     S = (P.L + kps - 1) / kps;
 }
 
-template <int HD, bool TREE>   // TREE: the new rows form a tree (positions and visibility from the state block), else a chain
+// MODE 0: the new rows are a chain; 1: a tree (positions and visibility from the state block); 2: the chain of
+// sequence `b` of a batched step (its rows, length and KV cache from P.seq[b]).
+template <int HD, int MODE>
 __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int hk, int qg, int gh, int s, int S, int kps, uint8_t* att,
-                                            int wtid, unsigned long long* prof) {
+                                            int wtid, unsigned long long* prof, int b) {
+    constexpr bool TREE = MODE == 1, BATCH = MODE == 2;
     constexpr int HD2 = HD / 2;
     constexpr int KSTEPS = HD / 16;
     constexpr int UNITS = HD / 8;    // 16-byte units per K/V row
@@ -561,7 +564,10 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
     // exchange area of the key-group merge: (KG - 1) * MT <= 6 tiles of (output + statistics)
     static_assert(6 * (NT_O + 1) * 32 * 16 <= NBUF * 2 * KVBYTES, "exchange area of the key-group merge");
     const int warp = wtid >> 5, lane = wtid & 31;
-    const int M = P.M, L = P.L;
+    const int M = BATCH ? P.seq[b].M : P.M, L = BATCH ? P.seq[b].L : P.L;
+    const int r0 = BATCH ? P.seq[b].r0 : 0;      // first row of this sequence in the launch's buffers
+    __nv_bfloat16* const kcache = BATCH ? P.seq[b].kcache : P.kcache;
+    __nv_bfloat16* const vcache = BATCH ? P.seq[b].vcache : P.vcache;
     const int nheads = min(gh, P.g - qg * gh);   // the last group may hold fewer heads
     const int R = nheads * M;                    // R <= 64
     const int MT = (R + 15) >> 4, RP = MT * 16;
@@ -595,8 +601,8 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
                 const bool valid = kk < nkeys;
                 const size_t off = (cache_row0 + t_begin + (valid ? kk : 0)) * HD + q16 * 8;
                 const uint32_t so = (q16 >> 3) * (KB * 128) + swz_unit(key, q16 & 7);
-                cp_async_16_zfill(Ks + so, P.kcache + off, valid);
-                cp_async_16_zfill(Vs + so, P.vcache + off, valid);
+                cp_async_16_zfill(Ks + so, kcache + off, valid);
+                cp_async_16_zfill(Vs + so, vcache + off, valid);
             }
         }
         cp_async_commit();  // possibly empty: keeps the group count uniform
@@ -624,9 +630,9 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
                 qa[t] = qb[t] = c0[t] = c1[t] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (idx < items && rr[t] < R) {
                     const int hl = rr[t] / M, j = rr[t] % M, col = (head0 + hl) * HD + ii[t];
-                    ssq[t] = __ldcg(sumsq + j);
-                    qa[t] = ld_cg_f4_inorder(P.qkv_acc + (size_t)j * P.n_qkv + col);
-                    qb[t] = ld_cg_f4_inorder(P.qkv_acc + (size_t)j * P.n_qkv + col + HD2);
+                    ssq[t] = __ldcg(sumsq + r0 + j);
+                    qa[t] = ld_cg_f4_inorder(P.qkv_acc + (size_t)(r0 + j) * P.n_qkv + col);
+                    qb[t] = ld_cg_f4_inorder(P.qkv_acc + (size_t)(r0 + j) * P.n_qkv + col + HD2);
                     const int pj = TREE ? __ldcg(P.state + ST_DEPTH + j) : j;  // tree drafts: a row's position is its depth
                     const float4* rp = reinterpret_cast<const float4*>(P.rope + (size_t)(L + pj) * HD2 + ii[t]);
                     c0[t] = ld_nc_f4_inorder(rp);
@@ -670,8 +676,8 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
             const int key = u / UNITS, q16 = u % UNITS, kk = key;
             uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
             if (kk < nkeys) {
-                const float rs = rsqrtf(__ldcg(sumsq + kk) / (float)P.d + P.eps);
-                const float* accrow = P.qkv_acc + (size_t)kk * P.n_qkv;
+                const float rs = rsqrtf(__ldcg(sumsq + r0 + kk) / (float)P.d + P.eps);
+                const float* accrow = P.qkv_acc + (size_t)(r0 + kk) * P.n_qkv;
                 const int colb = q16 * 8, ib = colb % HD2;  // 8 columns share one half of the rotary pairing
                 const float* pa = accrow + Nq + hk * HD + ib;
                 const float4 a0 = ldcg_f4(pa), a1 = ldcg_f4(pa + 4), b0 = ldcg_f4(pa + HD2), b1 = ldcg_f4(pa + HD2 + 4);
@@ -702,8 +708,8 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
                                  pack_bf16(v[6], v[7]));
                 if (qg == 0) {  // every head group computes the rows, one appends them
                     const size_t off = (cache_row0 + L + kk) * HD + q16 * 8;
-                    *reinterpret_cast<uint4*>(P.kcache + off) = kv4;
-                    *reinterpret_cast<uint4*>(P.vcache + off) = vv4;
+                    *reinterpret_cast<uint4*>(kcache + off) = kv4;
+                    *reinterpret_cast<uint4*>(vcache + off) = vv4;
                 }
             }
             const uint32_t so = (q16 >> 3) * (KB * 128) + swz_unit(key, q16 & 7);
@@ -849,7 +855,7 @@ __device__ __noinline__ void attention_unit(const FwdParams& P, int layer, int h
             const int r = half ? r_hi : r_lo;
             if (r >= R) continue;
             const int hq = head0 + r / M, j = r % M;
-            const size_t row = ((size_t)hq * (kMaxSplits + 1) + s) * kMaxRows + j;
+            const size_t row = ((size_t)hq * (kMaxSplits + 1) + s) * kMaxRows + r0 + j;
             float* po = P.part_o + row * HD + q2;
 #pragma unroll
             for (int n = 0; n < NT_O; ++n)
@@ -865,15 +871,21 @@ __device__ void attention_phase(const FwdParams& P, int layer, uint8_t* att, int
     attn_split(P, S, kps);
     const int S1 = S + 1;
     const int gh = P.att_gh, QG = (P.g + gh - 1) / gh;
-    const int nunits = P.n_kv * QG * S1;
+    const int per_seq = P.n_kv * QG * S1;
+    const int nunits = per_seq * (P.nseq > 0 ? P.nseq : 1);
     for (int unit = blockIdx.x; unit < nunits; unit += P.G) {
-        const int hk = unit / (QG * S1), rem = unit % (QG * S1), qg = rem / S1, s = rem % S1;
-        if (P.tree) {
-            if (P.hd == 128) attention_unit<128, true>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof);
-            else attention_unit<64, true>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof);
+        const int b = unit / per_seq, u = unit % per_seq;
+        const int hk = u / (QG * S1), rem = u % (QG * S1), qg = rem / S1, s = rem % S1;
+        if (P.nseq > 0) {
+            // every sequence takes the key ranges of the longest one; a range past its own length holds no key
+            if (P.hd == 128) attention_unit<128, 2>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof, b);
+            else attention_unit<64, 2>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof, b);
+        } else if (P.tree) {
+            if (P.hd == 128) attention_unit<128, 1>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof, 0);
+            else attention_unit<64, 1>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof, 0);
         } else {
-            if (P.hd == 128) attention_unit<128, false>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof);
-            else attention_unit<64, false>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof);
+            if (P.hd == 128) attention_unit<128, 0>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof, 0);
+            else attention_unit<64, 0>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof, 0);
         }
         named_bar_sync(1, kWorkerThreads);  // the unit's shared-memory tiles are free again
         if (prof && wtid == 0) { prof[6] = global_timer_ns(); prof[7] = (unsigned long long)(s == S); }

@@ -28,6 +28,7 @@ constexpr int kStepBytes = 512;                        // one row tile x one col
 constexpr int kStageBytes = 32768;                     // ring slot
 constexpr int kMaxStages = 8;                          // ring slots at most
 constexpr int kMaxRows = 32;                           // token rows a buffer is sized for
+constexpr int kMaxBatch = 8;                           // sequences one batched verify step takes at most
 constexpr int kMaxSplits = 19;                         // KV key ranges per head (+1 partial result for the new rows)
 constexpr int kSmemBudget = 232448;                    // 227 KB
 constexpr int kAttnSmemBytes = 81920;                  // Q tile (up to 16 KB) + two K|V blocks of 64 keys (64 KB)
@@ -172,6 +173,14 @@ enum StateWord {
     ST_WORDS = 320
 };
 
+// One sequence of a batched verify step: its rows [r0, r0 + M) of the launch, its committed length
+// and its own KV cache.
+struct BatchSeq {
+    __nv_bfloat16* kcache;
+    __nv_bfloat16* vcache;
+    int r0, M, L, pad;
+};
+
 struct FwdParams {
     // model
     int n_layers, d, n_q, n_kv, hd, f, V, max_seq, g, n_qkv;
@@ -220,6 +229,9 @@ struct FwdParams {
     int act_off;       // SwiGLU output operand
     int misc_off;
     unsigned long long wait_limit_ns;
+    // batched verify: nseq > 0 sequences share the launch (chains only); L is then the longest length
+    int nseq;
+    BatchSeq seq[kMaxBatch];
 };
 
 }  // namespace sdv

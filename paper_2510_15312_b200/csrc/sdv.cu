@@ -23,7 +23,7 @@ namespace {
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Regions {
-    size_t state, bar, never, hist, db, rope, norm_w, bias, wlayers, wlm, emb, kcache, vcache, h, qkv_acc, sumsq, part_o,
+    size_t state, bstate, bar, never, hist, db, rope, norm_w, bias, wlayers, wlm, emb, kcache, vcache, h, qkv_acc, sumsq, part_o,
         part_ml, cand_val, cand_idx, logits, raw_out, staging, wraw, xstage, prof, succ, occ, dw, dh, dxn, dqkv, dq, datt, dact, dtok, total;
     size_t layer_stride, staging_bytes, raw_kmax;
 };
@@ -45,7 +45,9 @@ bool config_ok(const sdv_config* c) {
     return true;
 }
 
-Regions carve(const sdv_config* c) {
+// `own_weights` false: a context that reads another context's weights carves none of the weight regions
+// (nor the staging areas only weight loading and the stand-alone GEMM use).
+Regions carve(const sdv_config* c, bool own_weights = true) {
     Regions r;
     memset(&r, 0, sizeof(r));
     const size_t d = c->d_model, f = c->d_ffn, V = c->vocab, hd = c->head_dim;
@@ -56,18 +58,20 @@ Regions carve(const sdv_config* c) {
         off = align_up(off + bytes, 256);
         return o;
     };
+    auto take_w = [&](size_t bytes) { return take(own_weights ? bytes : 0); };
     r.state = take(ST_WORDS * 4);
+    r.bstate = take(ST_WORDS * 4);  // state block a batched verify step runs on
     r.bar = take(256);
     r.never = take(256);
     r.hist = take(((size_t)c->max_seq + 64) * 4);
     r.db = take(((size_t)c->max_seq + 64) * 4);
     r.rope = take((size_t)c->max_seq * (hd / 2) * sizeof(float2));
-    r.norm_w = take(((size_t)c->n_layers * 2 + 1) * d * 4);
-    r.bias = take((size_t)c->n_layers * nqkv * 4);
+    r.norm_w = take_w(((size_t)c->n_layers * 2 + 1) * d * 4);
+    r.bias = take_w((size_t)c->n_layers * nqkv * 4);
     r.layer_stride = (nqkv * d + d * nq + 2 * f * d + d * f) * 2;
-    r.wlayers = take(r.layer_stride * c->n_layers);
-    r.wlm = take(V * d * 2);
-    r.emb = take(V * d * 2);
+    r.wlayers = take_w(r.layer_stride * c->n_layers);
+    r.wlm = take_w(V * d * 2);
+    r.emb = take_w(V * d * 2);
     const size_t kvb = (size_t)c->n_layers * c->n_kv_heads * c->max_seq * hd * 2;
     r.kcache = take(kvb);
     r.vcache = take(kvb);
@@ -88,13 +92,13 @@ Regions carve(const sdv_config* c) {
     if (d * nq * 2 > st) st = d * nq * 2;
     if (st < ((size_t)64 << 20)) st = (size_t)64 << 20;
     r.staging_bytes = st;
-    r.staging = take(st);
-    r.wraw = take(st);
-    r.raw_out = take((size_t)kMaxRows * (st / 128) * 4);  // N <= staging / (2 bytes * 64 columns)
+    r.staging = take_w(st);
+    r.wraw = take_w(st);
+    r.raw_out = take_w((size_t)kMaxRows * (st / 128) * 4);  // N <= staging / (2 bytes * 64 columns)
     r.xstage = take((size_t)kMaxRows * raw_kmax * 4);
     r.prof = take((size_t)(3 + kPhasesPerLayer * c->n_layers) * kMaxGrid * kProfWords * 8);
     // dense prefill path: row-major weight copies and the activations of one sub-chunk
-    r.dw = take(r.layer_stride * c->n_layers);
+    r.dw = take_w(r.layer_stride * c->n_layers);
     r.dh = take((size_t)kDenseMaxRows * d * 4);
     r.dxn = take((size_t)kDenseMaxRows * d * 2);
     r.dqkv = take((size_t)kDenseMaxRows * nqkv * 4);
@@ -273,6 +277,8 @@ struct sdv_ctx {
     bool calibrated;     // the calibration tables cover the whole context
     bool tree_pending;   // the device draft is a tree
     bool tree_verified;  // the outstanding verify result is a tree's
+    sdv_ctx* leader;     // the context whose weights this one reads (nullptr: its own)
+    const float* logits_src;  // where the rows of this context's last verify step lie (a batched step leaves them in the first context's buffer)
 };
 
 namespace {
@@ -337,14 +343,27 @@ void plan_attention(FwdParams& P, int rows, int L) {
 }
 
 // Runs phases [ph_begin, ph_end) over `rows` token rows at position L.
+// `batch`: the sequences of a batched step (then `rows` is their total, `L` the longest length, and the launch
+// reads its tokens from the batch state block).
+struct BatchPlan {
+    int n, max_rows;
+    BatchSeq seq[kMaxBatch];
+};
 int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph_end, bool timed, bool force_logits = false,
-                   bool tree = false) {
+                   bool tree = false, const BatchPlan* batch = nullptr) {
     FwdParams P = ctx->P;
     int smem_bytes = 0;
     const bool raw_only = (ph_begin == 2 + kPhasesPerLayer * ctx->cfg.n_layers);
     if (!apply_plan(P, rows, raw_only, &smem_bytes)) return SDV_EINVAL;
     P.L = L;
-    plan_attention(P, rows, L);
+    plan_attention(P, batch ? batch->max_rows : rows, L);
+    P.nseq = 0;
+    if (batch) {
+        P.nseq = batch->n;
+        for (int b = 0; b < batch->n; ++b) P.seq[b] = batch->seq[b];
+        P.state = (int*)(ctx->ws + ctx->r.bstate);
+    }
+    ctx->logits_src = P.logits;
     P.mode = mode;
     P.ph_begin = ph_begin;
     P.ph_end = ph_end;
@@ -492,8 +511,8 @@ int dense_prefill_rows(sdv_ctx* ctx, int rows, int L) {
     __nv_bfloat16* act = (__nv_bfloat16*)(ws + ctx->r.dact);
     const int* hist = (const int*)(ws + ctx->r.hist);
     const std::vector<CUtensorMap>& maps = *ctx->maps;
-    const float* norm_w = (const float*)(ws + ctx->r.norm_w);
-    const float* bias = c.qkv_bias ? (const float*)(ws + ctx->r.bias) : nullptr;
+    const float* norm_w = ctx->P.norm_w;
+    const float* bias = ctx->P.bias;
     const size_t att_smem = (size_t)(16 * hd * 2 + 4 * 64 * hd * 2 + 128);  // query tile + two K|V blocks
     static bool att_attr = false;
     if (!att_attr) {
@@ -554,18 +573,23 @@ int sdv_last_cuda_error(const sdv_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
 long long sdv_launch_count(const sdv_ctx* ctx) { return ctx ? ctx->launches : 0; }
 int sdv_kv_len(const sdv_ctx* ctx) { return ctx ? ctx->kv_len : SDV_EINVAL; }
 
-int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* cuda_stream, sdv_ctx** out) {
+}  // extern "C"
+
+namespace {
+// A context over `dev_workspace`; with a `leader` it reads that context's weights instead of holding its own.
+int create_context(const sdv_config* cfg, void* dev_workspace, size_t bytes, cudaStream_t stream, sdv_ctx* leader, sdv_ctx** out) {
     if (!out) return SDV_EINVAL;
     *out = nullptr;
     if (!config_ok(cfg) || !dev_workspace || ((uintptr_t)dev_workspace & 255)) return SDV_EINVAL;
-    if (bytes < sdv_workspace_bytes(cfg)) return SDV_ENOMEM;
+    if (bytes < carve(cfg, leader == nullptr).total) return SDV_ENOMEM;
     sdv_ctx* ctx = new (std::nothrow) sdv_ctx();
     if (!ctx) return SDV_ENOMEM;
     memset(ctx, 0, sizeof(*ctx));
     ctx->cfg = *cfg;
     ctx->ws = (uint8_t*)dev_workspace;
     ctx->ws_bytes = bytes;
-    ctx->stream = (cudaStream_t)cuda_stream;
+    ctx->stream = stream;
+    ctx->leader = leader;
     int sms = 0, dev = 0, coop = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -576,7 +600,7 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
     }
     if (sms > kMaxGrid) sms = kMaxGrid;
     ctx->G = sms;  // one persistent block per SM
-    ctx->r = carve(cfg);
+    ctx->r = carve(cfg, leader == nullptr);
     // every failure below leaves through this: what was created so far is released
     auto fail = [&](int code) {
         if (ctx->pinned) cudaFreeHost(ctx->pinned);
@@ -602,12 +626,21 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
     const int rows_max = cfg->k_max + 1;
     P.layer_stride = ctx->r.layer_stride;
     uint8_t* ws = ctx->ws;
-    P.wlayers = ws + ctx->r.wlayers;
-    P.wlm = ws + ctx->r.wlm;
-    P.wraw = ws + ctx->r.wraw;
-    P.emb = (const __nv_bfloat16*)(ws + ctx->r.emb);
-    P.norm_w = (const float*)(ws + ctx->r.norm_w);
-    P.bias = cfg->qkv_bias ? (const float*)(ws + ctx->r.bias) : nullptr;
+    if (leader) {
+        P.wlayers = leader->P.wlayers;
+        P.wlm = leader->P.wlm;
+        P.wraw = nullptr;  // no stand-alone GEMM on a context without weight regions
+        P.emb = leader->P.emb;
+        P.norm_w = leader->P.norm_w;
+        P.bias = leader->P.bias;
+    } else {
+        P.wlayers = ws + ctx->r.wlayers;
+        P.wlm = ws + ctx->r.wlm;
+        P.wraw = ws + ctx->r.wraw;
+        P.emb = (const __nv_bfloat16*)(ws + ctx->r.emb);
+        P.norm_w = (const float*)(ws + ctx->r.norm_w);
+        P.bias = cfg->qkv_bias ? (const float*)(ws + ctx->r.bias) : nullptr;
+    }
     P.rope = (const float2*)(ws + ctx->r.rope);
     P.kcache = (__nv_bfloat16*)(ws + ctx->r.kcache);
     P.vcache = (__nv_bfloat16*)(ws + ctx->r.vcache);
@@ -649,6 +682,7 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
         if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
     }
     if (e == cudaSuccess) e = cudaMemsetAsync(ws + ctx->r.state, 0, ST_WORDS * 4, ctx->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ws + ctx->r.bstate, 0, ST_WORDS * 4, ctx->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(ws + ctx->r.bar, 0, 256, ctx->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(ws + ctx->r.never, 0, 256, ctx->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(ws + ctx->r.hist, 0, ((size_t)cfg->max_seq + 64) * 4, ctx->stream);
@@ -669,15 +703,40 @@ int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* c
         std::vector<CUtensorMap>& m = *ctx->maps;
         ctx->dense_ok = make_map(&m[0], ws + ctx->r.dxn, kDenseMaxRows, d) && make_map(&m[1], ws + ctx->r.datt, kDenseMaxRows, nq) &&
                         make_map(&m[2], ws + ctx->r.dact, kDenseMaxRows, f);
-        for (int l = 0; l < cfg->n_layers && ctx->dense_ok; ++l) {
+        if (leader) {  // the weight copies of the dense path are the leader's as well
+            ctx->dense_ok = ctx->dense_ok && leader->dense_ok;
+            for (size_t i = 3; i < m.size() && ctx->dense_ok; ++i) m[i] = (*leader->maps)[i];
+        }
+        for (int l = 0; l < cfg->n_layers && ctx->dense_ok && !leader; ++l) {
             uint8_t* lb = ws + ctx->r.dw + (size_t)l * ctx->r.layer_stride;
             const size_t o1 = (size_t)nqkv * d * 2, o2 = o1 + (size_t)d * nq * 2, o3 = o2 + (size_t)2 * f * d * 2;
             ctx->dense_ok = make_map(&m[3 + 4 * l], lb, nqkv, d) && make_map(&m[4 + 4 * l], lb + o1, d, nq) &&
                             make_map(&m[5 + 4 * l], lb + o2, 2 * (uint64_t)f, d) && make_map(&m[6 + 4 * l], lb + o3, d, f);
         }
     }
+    ctx->logits_src = P.logits;
+    ctx->weights_loaded = leader != nullptr;
     *out = ctx;
     return SDV_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int sdv_create(const sdv_config* cfg, void* dev_workspace, size_t bytes, void* cuda_stream, sdv_ctx** out) {
+    return create_context(cfg, dev_workspace, bytes, (cudaStream_t)cuda_stream, nullptr, out);
+}
+
+size_t sdv_follower_workspace_bytes(const sdv_config* cfg) {
+    if (!config_ok(cfg)) return 0;
+    return carve(cfg, false).total;
+}
+
+int sdv_create_follower(sdv_ctx* leader, void* dev_workspace, size_t bytes, sdv_ctx** out) {
+    if (out) *out = nullptr;
+    if (!leader || leader->leader) return SDV_EINVAL;  // followers follow a context that owns its weights
+    if (!leader->weights_loaded) return SDV_ESTATE;
+    return create_context(&leader->cfg, dev_workspace, bytes, leader->stream, leader, out);
 }
 
 int sdv_destroy(sdv_ctx* ctx) {
@@ -693,6 +752,7 @@ int sdv_destroy(sdv_ctx* ctx) {
 
 int sdv_load_weights(sdv_ctx* ctx, const sdv_weights* w) {
     if (!ctx || !w || !w->emb || !w->final_norm || !w->layers) return SDV_EINVAL;
+    if (ctx->leader) return SDV_ESTATE;
     const sdv_config& c = ctx->cfg;
     if (!c.tied_lm_head && !w->lm_head) return SDV_EINVAL;
     const size_t d = c.d_model, f = c.d_ffn, hd = c.head_dim, V = c.vocab;
@@ -913,7 +973,7 @@ int sdv_verify(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, int32_t* 
     const bool tree = !host_draft && ctx->tree_pending;
     int rc = launch_forward(ctx, rows, ctx->kv_len, 0, 0, 2 + kPhasesPerLayer * c.n_layers, true, false, tree);
     if (rc) return rc;
-    accept_kernel<<<1, 32 * rows, 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0);
+    accept_kernel<<<1, 32 * rows, 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0, 0, nullptr);
     ctx->launches++;
     CK(cudaGetLastError());
     ctx->verified = true;
@@ -927,6 +987,77 @@ int sdv_verify(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, int32_t* 
         if (host_y)
             for (int i = 0; i <= dl; ++i) host_y[i] = ctx->pinned[ST_Y + i];
     }
+    return SDV_OK;
+}
+
+int sdv_verify_batch(sdv_ctx* const* ctxs, int n, int* accept_len) {
+    if (!ctxs || n < 1 || n > kMaxBatch) return SDV_EINVAL;
+    sdv_ctx* ctx = ctxs[0];  // the launch runs on the first context's scratch buffers and stream
+    if (!ctx) return SDV_EINVAL;
+    sdv_ctx* owner = ctx->leader ? ctx->leader : ctx;
+    BatchPlan bp;
+    BatchGatherArg ga;
+    memset(&bp, 0, sizeof(bp));
+    memset(&ga, 0, sizeof(ga));
+    bp.n = ga.n = n;
+    int rows = 0, Lmax = 0;
+    for (int b = 0; b < n; ++b) {
+        sdv_ctx* c = ctxs[b];
+        if (!c) return SDV_EINVAL;
+        for (int a = 0; a < b; ++a)
+            if (ctxs[a] == c) return SDV_EINVAL;
+        if ((c->leader ? c->leader : c) != owner || c->stream != ctx->stream) return SDV_EINVAL;
+        if (c->poisoned) return SDV_ETIMEOUT;
+        if (!c->prefill_done || !c->weights_loaded || c->tree_pending) return SDV_ESTATE;  // chains only
+        const int m = c->draft_pending ? c->draft_k + 1 : 1;
+        if (c->kv_len + m > c->cfg.max_seq) return SDV_ECAPACITY;
+        bp.seq[b].kcache = c->P.kcache;
+        bp.seq[b].vcache = c->P.vcache;
+        bp.seq[b].r0 = ga.r0[b] = rows;
+        bp.seq[b].M = ga.M[b] = m;
+        bp.seq[b].L = c->kv_len;
+        ga.state[b] = c->P.state;
+        if (m > bp.max_rows) bp.max_rows = m;
+        if (c->kv_len > Lmax) Lmax = c->kv_len;
+        rows += m;
+    }
+    if (rows > kMaxRows) return SDV_EINVAL;
+    int* bstate = (int*)(ctx->ws + ctx->r.bstate);
+    batch_gather_kernel<<<1, kMaxRows, 0, ctx->stream>>>(bstate, ga);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    int rc = launch_forward(ctx, rows, Lmax, 0, 0, 2 + kPhasesPerLayer * ctx->cfg.n_layers, true, false, false, &bp);
+    if (rc) return rc;
+    for (int b = 0; b < n; ++b) {
+        sdv_ctx* c = ctxs[b];
+        accept_kernel<<<1, 32 * bp.seq[b].M, 0, ctx->stream>>>(c->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0, bp.seq[b].r0,
+                                                              bstate);
+        ctx->launches++;
+        c->verified = true;
+        c->tree_verified = false;
+        c->last_rows = bp.seq[b].M;
+        c->logits_src = ctx->P.logits + (size_t)bp.seq[b].r0 * ctx->cfg.vocab;
+    }
+    CK(cudaGetLastError());
+    if (accept_len) {
+        for (int b = 0; b < n; ++b) {
+            sdv_ctx* c = ctxs[b];
+            rc = read_state(c);
+            if (rc) return rc;
+            accept_len[b] = c->pinned[ST_ACCEPT_LEN];
+        }
+    }
+    return SDV_OK;
+}
+
+int sdv_get_verified(sdv_ctx* ctx, int32_t* host_y, int* accept_len) {
+    if (!ctx) return SDV_EINVAL;
+    if (!ctx->verified) return SDV_ESTATE;
+    int rc = read_state(ctx);
+    if (rc) return rc;
+    if (accept_len) *accept_len = ctx->pinned[ST_ACCEPT_LEN];
+    if (host_y)
+        for (int i = 0; i < ctx->last_rows; ++i) host_y[i] = ctx->pinned[ST_Y + i];
     return SDV_OK;
 }
 
@@ -1066,7 +1197,7 @@ int sdv_verify_tree(sdv_ctx* ctx, const int32_t* host_tokens, const int32_t* hos
     }
     int rc = launch_forward(ctx, rows, ctx->kv_len, 0, 0, 2 + kPhasesPerLayer * c.n_layers, true, false, true);
     if (rc) return rc;
-    accept_kernel<<<1, 32 * rows, 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0);
+    accept_kernel<<<1, 32 * rows, 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0, 0, nullptr);
     ctx->launches++;
     CK(cudaGetLastError());
     ctx->verified = true;
@@ -1138,8 +1269,7 @@ int sdv_rollback(sdv_ctx* ctx, int new_kv_len) {
 int sdv_get_logits(sdv_ctx* ctx, float* host_logits, int rows) {
     if (!ctx || !host_logits || rows < 1 || rows > kMaxRows) return SDV_EINVAL;
     if (!ctx->parity) return SDV_ESTATE;
-    CK(cudaMemcpyAsync(host_logits, ctx->ws + ctx->r.logits, (size_t)rows * ctx->cfg.vocab * 4, cudaMemcpyDeviceToHost,
-                       ctx->stream));
+    CK(cudaMemcpyAsync(host_logits, ctx->logits_src, (size_t)rows * ctx->cfg.vocab * 4, cudaMemcpyDeviceToHost, ctx->stream));
     CK(cudaStreamSynchronize(ctx->stream));
     return SDV_OK;
 }
@@ -1208,7 +1338,7 @@ int sdv_debug_accept(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, con
         ctx->launches++;
     }
     set_y_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, y);
-    accept_kernel<<<1, 32 * (draft_len + 1), 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 1);
+    accept_kernel<<<1, 32 * (draft_len + 1), 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 1, 0, nullptr);
     ctx->launches += 2;
     CK(cudaGetLastError());
     ctx->verified = true;
@@ -1265,6 +1395,7 @@ int sdv_debug_gemm(sdv_ctx* ctx, const float* host_x, const uint16_t* host_w, fl
                    float* dev_ms) {
     if (!ctx || !host_x || !host_w || !host_y) return SDV_EINVAL;
     if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (ctx->leader) return SDV_ESTATE;  // no staging areas without weight regions
     if (M < 1 || M > kMaxRows || N < 16 || N % 16 || K < 64 || K % 64) return SDV_EINVAL;
     if ((size_t)K > ctx->r.raw_kmax || (size_t)N * K * 2 > ctx->r.staging_bytes || (size_t)N > ctx->r.staging_bytes / 128)
         return SDV_EINVAL;

@@ -379,10 +379,14 @@ __global__ void extension_update_kernel(int* state, int max_life) {
 // Greedy tokens and accept scan.  Row j's token is the best of the per-block candidates
 // (largest logit, lowest id among equals); a = number of leading drafts equal to the model's
 // prediction; emitted = x_1..x_a, y_{a+1}.  One block of 32 * rows threads: warp j reduces row j.
-__global__ void accept_kernel(int* state, const float* cand_val, const int* cand_idx, int G, int from_host_y) {
+// `row0`: the sequence's first row among the launch's rows (0 unless the step was batched); `launch_state`:
+// the state block the launch ran on when it is not `state` itself, whose error word is carried over.
+__global__ void accept_kernel(int* state, const float* cand_val, const int* cand_idx, int G, int from_host_y, int row0,
+                              const int* launch_state) {
     __shared__ int y_s[kMaxRows + 1];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int dl = state[ST_DRAFT_LEN];
+    if (launch_state && threadIdx.x == 0 && launch_state[ST_ERR]) state[ST_ERR] = launch_state[ST_ERR];
     if (warp <= dl) {
         int bi;
         if (from_host_y) {
@@ -391,8 +395,8 @@ __global__ void accept_kernel(int* state, const float* cand_val, const int* cand
             float bv = -CUDART_INF_F;
             bi = 0x7fffffff;
             for (int c = lane; c < G; c += 32) {
-                const float v = cand_val[(size_t)c * kMaxRows + warp];
-                const int i = cand_idx[(size_t)c * kMaxRows + warp];
+                const float v = cand_val[(size_t)c * kMaxRows + row0 + warp];
+                const int i = cand_idx[(size_t)c * kMaxRows + row0 + warp];
                 if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
             }
             for (int off = 16; off; off >>= 1) {
@@ -431,6 +435,31 @@ __global__ void accept_kernel(int* state, const float* cand_val, const int* cand
         state[ST_ACCEPT_LEN] = a;
         state[ST_N_EMITTED] = a + 1;
         state[ST_VERIFIED] = 1;
+    }
+}
+
+// Batched verify: the token rows of up to kMaxBatch sequences (each its pending token, then its draft, token 0
+// past the draft's length) are laid out one after another in the state block the shared launch reads.
+struct BatchGatherArg {
+    const int* state[kMaxBatch];
+    int r0[kMaxBatch], M[kMaxBatch];
+    int n;
+};
+__global__ void batch_gather_kernel(int* launch_state, BatchGatherArg a) {
+    const int t = threadIdx.x;
+    for (int b = 0; b < a.n; ++b) {
+        if (t < a.M[b]) {
+            const int* st = a.state[b];
+            const int tok = (t == 0) ? st[ST_PENDING] : (t <= st[ST_DRAFT_LEN] ? st[ST_DRAFT + t - 1] : 0);
+            const int row = a.r0[b] + t;
+            if (row == 0) launch_state[ST_PENDING] = tok;
+            else launch_state[ST_DRAFT + row - 1] = tok;
+        }
+    }
+    if (t == 0) {
+        launch_state[ST_DRAFT_LEN] = a.r0[a.n - 1] + a.M[a.n - 1] - 1;
+        launch_state[ST_TREE_ON] = 0;
+        launch_state[ST_ERR] = 0;
     }
 }
 

@@ -71,6 +71,14 @@ def compare_step(sdv, step: RefStep, k: int, stats: dict, predrafted: bool = Fal
     else:
         y, a = sdv.verify(step.draft)
         rows = dl + 1
+    check_verified(sdv, step, y, a, stats, before_commit)
+    return rows
+
+
+def check_verified(sdv, step: RefStep, y, a, stats: dict, before_commit=None):
+    """The part of compare_step after the verify call: logits rows, greedy tokens and accept length of the
+    context's outstanding verify result against the reference step, then the oracle's outcome is committed."""
+    dl = len(step.draft)
     logits = sdv.get_logits(dl + 1)
     assert np.all(np.isfinite(logits))
     for r in range(dl + 1):
@@ -105,7 +113,6 @@ def compare_step(sdv, step: RefStep, k: int, stats: dict, predrafted: bool = Fal
     # teacher forcing: commit what the oracle committed
     sdv.debug_force_commit(len(step.emitted) - 1, step.emitted[-1])
     assert sdv.kv_len() == step.kv_len_before + len(step.emitted)
-    return rows
 
 
 def compare_prefix_rows(sdv, step: RefStep, kp: int, stats: dict):
