@@ -426,7 +426,7 @@ def main():
                "accepted_drafts_per_step": tokens_x / args.steps - 1.0, "scope": "rank 0"}
 
     # ---- the two other labelled throughput numbers (single-GPU runs only; synthetic acceptance)
-    forced = hist_mode = prefill = None
+    forced = hist_mode = prefill = batched = None
     if extras and world == 1:
         # (C) forced acceptance.  The greedy continuation comes from this path's own plain decoding (one token
         # per step, no oracle involved), recorded before the timed region; each timed step then verifies a
@@ -500,6 +500,48 @@ def main():
                      "value": toks_h / (ms_h * 1e-3), "unit": UNIT, "ms_per_step": ms_h / args.steps,
                      "emitted_per_step": toks_h / args.steps, "verify_kernel_us": statistics.mean(kms_h) * 1e3}
 
+        # batched verify: further sequences (their own contexts, the same length) read this context's weights and
+        # share every pass over them; aggregate tokens/s over the sequences of the batch
+        n_seq = min(3, 32 // (k + 1))
+        if n_seq >= 2:
+            fols = [s.follower() for _ in range(n_seq - 1)]
+            for i, fo in enumerate(fols):
+                fctx = make_context(cfg, seed=cfg.seed + 1 + i)
+                for j in range(0, cfg.n_ctx, cfg.chunk):
+                    fo.prefill_chunk(fctx[j:j + cfg.chunk], is_last=(j + cfg.chunk >= cfg.n_ctx))
+            seqs = [s] + fols
+
+            def batch_loop(n):
+                toks, kms_b = 0, []
+                for _ in range(n):
+                    for q in seqs:
+                        q.draft(k, fetch=False)
+                    Sdv.verify_batch(seqs, fetch=False)
+                    for q in seqs:
+                        em, _ = q.commit()
+                        toks += len(em)
+                    kms_b.append(s.last_verify_ms())
+                return toks, kms_b
+            batch_loop(args.warmup)
+            torch.cuda.synchronize()
+            b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            b0.record(stream)
+            toks_b, kms_b = batch_loop(args.steps)
+            b1.record(stream)
+            torch.cuda.synchronize()
+            ms_b = b0.elapsed_time(b1)
+            wb_b, _ = s.step_bytes(k + 1, L0)
+            kv_b = sum(q.step_bytes(k + 1, q.kv_len())[1] for q in seqs)
+            gbs_b = (wb_b + kv_b) / (statistics.mean(kms_b) * 1e-3) / 1e9
+            batched = {"label": f"{n_seq} sequences per verify step (sdv_verify_batch): one pass over the weights for "
+                                f"{n_seq * (k + 1)} rows, each sequence its own context, KV cache and search_history drafter",
+                       "sequences": n_seq, "rows_per_verify": n_seq * (k + 1),
+                       "value": toks_b / (ms_b * 1e-3), "unit": UNIT, "ms_per_step": ms_b / args.steps,
+                       "emitted_per_step": toks_b / args.steps, "verify_kernel_us": statistics.mean(kms_b) * 1e3,
+                       "GB/s": gbs_b, "frac": gbs_b / load_peaks()[0]}
+            for fo in fols:
+                fo.close()
+
     (ms_total, ms_e2e), (tokens_all, tokens_e_all) = aggregate_over_ranks([ms_total, ms_e2e], [tokens, tokens_e], world,
                                                                           "cuda")
 
@@ -539,6 +581,8 @@ def main():
         if hist_mode:
             line["history"] = hist_mode
             line["prefill"] = prefill
+        if batched:
+            line["batched"] = batched
         if ext:
             line["extension"] = ext
         if sweep:

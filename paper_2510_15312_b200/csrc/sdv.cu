@@ -318,8 +318,10 @@ bool apply_plan(FwdParams& P, int rows, bool raw_only, int* smem_bytes) {
 
 // Attention split of a launch: heads per unit (a unit's rows, heads x M, fill at most four 16-row
 // tiles), number of key ranges and keys per range (a multiple of 64).  Cost of a choice = the
-// 16-key steps a warp walks one after another: blocks of 64 keys per range x steps per block.
-void plan_attention(FwdParams& P, int rows, int L) {
+// 16-key steps a warp walks one after another: blocks of 64 keys per range x steps per block; with
+// more units than blocks (several sequences, each with its own units) the blocks take them in rounds,
+// each round paying a unit's fixed cost (about three such steps) again.
+void plan_attention(FwdParams& P, int rows, int L, int nseq = 1) {
     P.att_gh = 1;
     if (P.g < 1) return;
     int best = -1;
@@ -330,11 +332,14 @@ void plan_attention(FwdParams& P, int rows, int L) {
         int cap = P.G / (P.n_kv * QG) - 1;
         if (cap > kMaxSplits) cap = kMaxSplits;
         if (cap < 1) cap = 1;
-        int cost = 1;
+        int cost = 1, S = 0;
         if (L > 0) {
             const int kps = ((L + cap - 1) / cap + 63) / 64 * 64;
+            S = (L + kps - 1) / kps;
             cost = (kps / 64) * ((4 + KG - 1) / KG);
         }
+        const int rounds = (P.n_kv * QG * (S + 1) * nseq + P.G - 1) / P.G;
+        cost = rounds * (3 + cost);
         if (best < 0 || cost <= best) {  // ties: more heads per unit (fewer reloads of the keys)
             best = cost;
             P.att_gh = gh;
@@ -342,7 +347,6 @@ void plan_attention(FwdParams& P, int rows, int L) {
     }
 }
 
-// Runs phases [ph_begin, ph_end) over `rows` token rows at position L.
 // `batch`: the sequences of a batched step (then `rows` is their total, `L` the longest length, and the launch
 // reads its tokens from the batch state block).
 struct BatchPlan {
@@ -356,7 +360,7 @@ int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph
     const bool raw_only = (ph_begin == 2 + kPhasesPerLayer * ctx->cfg.n_layers);
     if (!apply_plan(P, rows, raw_only, &smem_bytes)) return SDV_EINVAL;
     P.L = L;
-    plan_attention(P, batch ? batch->max_rows : rows, L);
+    plan_attention(P, batch ? batch->max_rows : rows, L, batch ? batch->n : 1);
     P.nseq = 0;
     if (batch) {
         P.nseq = batch->n;
