@@ -370,16 +370,21 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- device-resident loop
+    # ---- device-resident loop: the steps are enqueued as one run (sdv_decode_steps: KV length, history and drafts
+    # pass from step to step on the device; one synchronisation at the end of the run)
+    def run(n):
+        em, _ = s.decode_steps(k, n)
+        return len(em), [float(x) for x in s.run_kernel_ms(n)]
+
     sampler = ClockSampler(local)
     sampler.start()                      # before the warm-up: the first samples arrive while it runs
-    loop(args.warmup, False)
+    run(args.warmup)
     launches0 = s.launch_count()
     barrier()
     sampler.mark()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record(stream)
-    tokens, kms = loop(args.steps, False)
+    tokens, kms = run(args.steps)
     ev1.record(stream)
     barrier()
     launches = s.launch_count() - launches0
@@ -488,11 +493,11 @@ def main():
                    "tflops_linear": lin / (ms_p * 1e-3) / 1e12, "tflops_linear_plus_attention": (lin + att) / (ms_p * 1e-3) / 1e12,
                    "bf16_peak_tflops": tf[0], "peak_kind": f"of {tf[1]} (sustained)",
                    "frac": (lin + att) / (ms_p * 1e-3) / 1e12 / tf[0]}
-        loop(args.warmup, False)
+        run(args.warmup)
         torch.cuda.synchronize()
         h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         h0.record(stream)
-        toks_h, kms_h = loop(args.steps, False)
+        toks_h, kms_h = run(args.steps)
         h1.record(stream)
         torch.cuda.synchronize()
         ms_h = h0.elapsed_time(h1)

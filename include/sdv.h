@@ -135,6 +135,27 @@ int sdv_set_database(sdv_ctx *ctx, const int32_t *host_tokens, int n);
  * Errors: SDV_ESTATE before prefill has finished, SDV_ECAPACITY, SDV_EINVAL, SDV_ETIMEOUT. */
 int sdv_verify(sdv_ctx *ctx, const int32_t *host_draft, int draft_len, int32_t *host_y, int *accept_len);
 
+/* A run of decoding steps without the host in between (paper Sec. 4.1, online workflow: draft -> verify ->
+ * accept repeated until the answer ends).  Enqueues n_steps (1..4096) steps of sdv_draft(k) [+
+ * sdv_extend_draft(ext_max_total) when ext_max_total > 0] -> sdv_verify -> [sdv_extension_update(ext_max_life)]
+ * -> sdv_commit on the context's stream; every kernel takes the KV length, history and drafts from the
+ * device state the step before left, so nothing is read back until the run ends.  Each verify computes
+ * k + 1 rows (ext_max_total + 1 with the extension; k <= ext_max_total <= k_max); between two forward kernels one
+ * launch does the accept scan, the commit and the next draft.  max_tokens > 0 ends the
+ * run after that many emitted tokens: the step that reaches it is cut like sdv_commit's max_emit and the
+ * steps enqueued behind it do nothing (they cost a few microseconds each); max_tokens <= 0: no limit.
+ * The emitted tokens equal those of the same calls made one by one.  host_tokens (room for
+ * min(max_tokens, n_steps * rows) ints), n_tokens and kv_len may be NULL.  Synchronises once, at the end.
+ * Errors: SDV_EINVAL, SDV_ESTATE (before the end of prefill), SDV_ECAPACITY (n_steps * rows positions
+ * must fit behind the current KV length and history), SDV_ETIMEOUT.
+ *
+ * sdv_run_kernel_ms: device times in milliseconds of the first n forward kernels of the last run (CUDA
+ * events; a step enqueued behind the run's end shows a few microseconds).  Errors: SDV_ESTATE without a run
+ * of at least n steps. */
+int sdv_decode_steps(sdv_ctx *ctx, int k, int n_steps, int max_tokens, int ext_max_total, int ext_max_life,
+                     int32_t *host_tokens, int *n_tokens, int *kv_len);
+int sdv_run_kernel_ms(sdv_ctx *ctx, float *host_ms, int n);
+
 /* Batched verify: several sequences share one pass over the weights.  The paper verifies one request at
  * a time; its utilisation argument (Sec. 2: the matrix units need a large batch or a long sequence per
  * weight read) is what this call applies across requests, and every sequence's result is what sdv_verify

@@ -22,6 +22,7 @@ EXPORTS = [
     "sdv_set_calibration", "sdv_get_calibration", "sdv_draft_tree", "sdv_verify_tree", "sdv_debug_force_commit_tree",
     "sdv_debug_top_successors",
     "sdv_follower_workspace_bytes", "sdv_create_follower", "sdv_verify_batch", "sdv_get_verified",
+    "sdv_decode_steps", "sdv_run_kernel_ms",
 ]
 
 
@@ -82,6 +83,8 @@ def load_library(path: Optional[str] = None):
     L.sdv_create_follower.argtypes = [vp, vp, C.c_size_t, C.POINTER(vp)]
     L.sdv_verify_batch.argtypes = [C.POINTER(vp), C.c_int, ip]
     L.sdv_get_verified.argtypes = [vp, i32p, ip]
+    L.sdv_decode_steps.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, i32p, ip, ip]
+    L.sdv_run_kernel_ms.argtypes = [vp, vp, C.c_int]
     L.sdv_strerror.argtypes = [C.c_int]
     L.sdv_strerror.restype = C.c_char_p
     L.sdv_last_cuda_error.argtypes = [vp]
@@ -227,6 +230,23 @@ class Sdv:
         a = (C.c_int * len(seqs))()
         seqs[0]._check(lib().sdv_verify_batch(hs, len(seqs), a if fetch else None), "sdv_verify_batch")
         return list(a) if fetch else None
+
+    def decode_steps(self, k: int, n_steps: int, max_tokens: int = 0, ext_max_total: int = 0,
+                     ext_max_life: int = 0) -> Tuple[List[int], int]:
+        """n_steps of draft -> verify -> commit enqueued back to back (one synchronisation at the end);
+        returns (emitted tokens, KV length)."""
+        rows = (ext_max_total if ext_max_total > 0 else k) + 1
+        out = np.zeros(n_steps * rows + 1, dtype=np.int32)
+        n, kv = C.c_int(0), C.c_int(0)
+        self._check(lib().sdv_decode_steps(self._h, k, n_steps, max_tokens, ext_max_total, ext_max_life, out.ctypes.data,
+                                           C.byref(n), C.byref(kv)), "sdv_decode_steps")
+        return out[:n.value].tolist(), kv.value
+
+    def run_kernel_ms(self, n: int) -> np.ndarray:
+        """Forward-kernel times (ms) of the first n steps of the last decode_steps run."""
+        ms = np.zeros(n, dtype=np.float32)
+        self._check(lib().sdv_run_kernel_ms(self._h, ms.ctypes.data, n), "sdv_run_kernel_ms")
+        return ms
 
     def get_verified(self) -> Tuple[np.ndarray, int]:
         """(y, accept_len) of the outstanding verify step of this sequence."""

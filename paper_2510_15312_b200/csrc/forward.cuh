@@ -1012,6 +1012,11 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     Misc* misc = reinterpret_cast<Misc*>(smem + Pg.misc_off);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (Pg.l_from_state && Pg.state[ST_BUDGET] == 0) {
+        // a step enqueued behind the end of its run: nothing to do, but the barrier counter moves as the host assumed
+        if (tid == 0 && Pg.ph_end - Pg.ph_begin > 1) red_release_add_u32(Pg.bar, (unsigned)(Pg.ph_end - Pg.ph_begin - 1));
+        return;
+    }
     {
         const int* src = reinterpret_cast<const int*>(&Pg);
         int* dst = reinterpret_cast<int*>(&misc->P);
@@ -1039,6 +1044,8 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // the first reader of L (the attention phase) comes after a grid barrier, which orders this write before it
+    if (tid == 0 && Pg.l_from_state) misc->P.L = Pg.state[ST_KV_LEN];
 
     if (warp == kProducerWarp) {
         if (lane == 0) producer_loop(P, smem, misc);

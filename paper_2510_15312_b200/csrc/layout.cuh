@@ -164,6 +164,7 @@ enum StateWord {
     ST_Y = 48,        // [33]
     ST_TREE_ON = 82,  // 1: the draft is a tree (ST_PARENT .. ST_ANC hold its shape), 0: a chain
     ST_PATH_LEN = 83, // nodes on the accepted path of the last tree verify
+    ST_BUDGET = 84,   // tokens a run of enqueued steps may still emit (-1: no limit; 0: the remaining steps do nothing)
     ST_EMITTED = 96,  // [33]
     ST_SEG = 160,     // [32]
     ST_PARENT = 192,  // [32] row that row j continues (row 0 = the committed token; draft node i is row i)
@@ -229,6 +230,7 @@ struct FwdParams {
     int act_off;       // SwiGLU output operand
     int misc_off;
     unsigned long long wait_limit_ns;
+    int l_from_state;  // 1: L is read from the state block when the kernel starts (steps enqueued without the host in between)
     // batched verify: nseq > 0 sequences share the launch (chains only); L is then the longest length
     int nseq;
     BatchSeq seq[kMaxBatch];

@@ -277,6 +277,8 @@ struct sdv_ctx {
     bool calibrated;     // the calibration tables cover the whole context
     bool tree_pending;   // the device draft is a tree
     bool tree_verified;  // the outstanding verify result is a tree's
+    std::vector<cudaEvent_t>* run_ev;  // event pairs around the forward kernels of the last run of enqueued steps
+    int run_steps;       // steps of that run
     sdv_ctx* leader;     // the context whose weights this one reads (nullptr: its own)
     const float* logits_src;  // where the rows of this context's last verify step lie (a batched step leaves them in the first context's buffer)
 };
@@ -354,8 +356,9 @@ struct BatchPlan {
     BatchSeq seq[kMaxBatch];
 };
 int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph_end, bool timed, bool force_logits = false,
-                   bool tree = false, const BatchPlan* batch = nullptr) {
+                   bool tree = false, const BatchPlan* batch = nullptr, bool l_from_state = false, cudaEvent_t* run_ev = nullptr) {
     FwdParams P = ctx->P;
+    P.l_from_state = l_from_state ? 1 : 0;
     int smem_bytes = 0;
     const bool raw_only = (ph_begin == 2 + kPhasesPerLayer * ctx->cfg.n_layers);
     if (!apply_plan(P, rows, raw_only, &smem_bytes)) return SDV_EINVAL;
@@ -377,13 +380,13 @@ int launch_forward(sdv_ctx* ctx, int rows, int L, int mode, int ph_begin, int ph
     P.prof = ctx->profile ? (unsigned long long*)(ctx->ws + ctx->r.prof) : nullptr;
     const int nbar = ph_end - ph_begin - 1;
     ctx->bar_base += (unsigned)(nbar * ctx->G);
-    if (timed) CK(cudaEventRecord(ctx->ev0, ctx->stream));
+    if (timed) CK(cudaEventRecord(run_ev ? run_ev[0] : ctx->ev0, ctx->stream));
     cudaError_t e = launch_kernel(P, smem_bytes, ctx->stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches++;
     if (timed) {
-        CK(cudaEventRecord(ctx->ev1, ctx->stream));
-        ctx->have_verify_time = true;
+        CK(cudaEventRecord(run_ev ? run_ev[1] : ctx->ev1, ctx->stream));
+        if (!run_ev) ctx->have_verify_time = true;
     }
     return SDV_OK;
 }
@@ -426,7 +429,7 @@ int commit_common(sdv_ctx* ctx, int max_emit, int force_accept, int force_token,
         ctx->launches++;
         ctx->tree_verified = false;
     }
-    commit_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, hist, max_emit, force_accept, force_token);
+    commit_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, hist, max_emit, force_accept, force_token, 0);
     ctx->launches++;
     CK(cudaGetLastError());
     int rc = read_state(ctx);
@@ -750,6 +753,10 @@ int sdv_destroy(sdv_ctx* ctx) {
     cudaEventDestroy(ctx->ev0);
     cudaEventDestroy(ctx->ev1);
     delete ctx->maps;
+    if (ctx->run_ev) {
+        for (cudaEvent_t ev : *ctx->run_ev) cudaEventDestroy(ev);
+        delete ctx->run_ev;
+    }
     delete ctx;
     return SDV_OK;
 }
@@ -934,7 +941,7 @@ int sdv_draft(sdv_ctx* ctx, int k, int32_t* host_draft, int* draft_len) {
     if (!ctx->prefill_done) return SDV_ESTATE;
     int* hist = (int*)(ctx->ws + ctx->r.hist);
     ngram_draft_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->P.state, hist, (const int*)(ctx->ws + ctx->r.db), ctx->cfg.ngram_n,
-                                                    ctx->cfg.ngram_min, k, ctx->cfg.search_history);
+                                                    ctx->cfg.ngram_min, k, ctx->cfg.search_history, 0);
     ctx->launches++;
     CK(cudaGetLastError());
     ctx->draft_pending = true;
@@ -977,7 +984,7 @@ int sdv_verify(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, int32_t* 
     const bool tree = !host_draft && ctx->tree_pending;
     int rc = launch_forward(ctx, rows, ctx->kv_len, 0, 0, 2 + kPhasesPerLayer * c.n_layers, true, false, tree);
     if (rc) return rc;
-    accept_kernel<<<1, 32 * rows, 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0, 0, nullptr);
+    accept_kernel<<<1, 32 * rows, 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0, 0, nullptr, 0);
     ctx->launches++;
     CK(cudaGetLastError());
     ctx->verified = true;
@@ -1035,7 +1042,7 @@ int sdv_verify_batch(sdv_ctx* const* ctxs, int n, int* accept_len) {
     for (int b = 0; b < n; ++b) {
         sdv_ctx* c = ctxs[b];
         accept_kernel<<<1, 32 * bp.seq[b].M, 0, ctx->stream>>>(c->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0, bp.seq[b].r0,
-                                                              bstate);
+                                                              bstate, 0);
         ctx->launches++;
         c->verified = true;
         c->tree_verified = false;
@@ -1082,7 +1089,7 @@ int sdv_extend_draft(sdv_ctx* ctx, int max_total, int32_t* host_draft, int* draf
     if (!ctx || max_total < 1 || max_total > ctx->cfg.k_max) return SDV_EINVAL;
     if (ctx->poisoned) return SDV_ETIMEOUT;
     if (!ctx->prefill_done || !ctx->draft_pending) return SDV_ESTATE;
-    extend_draft_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, max_total);
+    extend_draft_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, max_total, 0);
     ctx->launches++;
     CK(cudaGetLastError());
     // rows of the next verify: the exact draft length when the caller reads it, else the bound
@@ -1103,7 +1110,7 @@ int sdv_extension_update(sdv_ctx* ctx, int max_life, int32_t* host_segment, int*
     if (!ctx || max_life < 1) return SDV_EINVAL;
     if (ctx->poisoned) return SDV_ETIMEOUT;
     if (!ctx->verified) return SDV_ESTATE;
-    extension_update_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, max_life);
+    extension_update_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, max_life, 0);
     ctx->launches++;
     CK(cudaGetLastError());
     if (host_segment || segment_len || lifetime) {
@@ -1115,6 +1122,73 @@ int sdv_extension_update(sdv_ctx* ctx, int max_life, int32_t* host_segment, int*
         if (host_segment)
             for (int i = 0; i < sl; ++i) host_segment[i] = ctx->pinned[ST_SEG + i];
     }
+    return SDV_OK;
+}
+
+int sdv_decode_steps(sdv_ctx* ctx, int k, int n_steps, int max_tokens, int ext_max_total, int ext_max_life, int32_t* host_tokens,
+                     int* n_tokens, int* kv_len) {
+    if (!ctx || k < 1 || k > ctx->cfg.k_max || n_steps < 1 || n_steps > 4096) return SDV_EINVAL;
+    if (ext_max_total < 0 || ext_max_total > ctx->cfg.k_max || (ext_max_total > 0 && (ext_max_total < k || ext_max_life < 1)))
+        return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->prefill_done || !ctx->weights_loaded) return SDV_ESTATE;
+    const sdv_config& c = ctx->cfg;
+    const int rows = (ext_max_total > 0 ? ext_max_total : k) + 1;
+    // every step may write `rows` KV rows beyond the length it starts from and emit up to `rows` tokens
+    if ((long long)ctx->kv_len + (long long)n_steps * rows > c.max_seq) return SDV_ECAPACITY;
+    if ((long long)ctx->hist_len + (long long)n_steps * rows > c.max_seq + 64) return SDV_ECAPACITY;
+    if (!ctx->run_ev) ctx->run_ev = new (std::nothrow) std::vector<cudaEvent_t>();
+    if (!ctx->run_ev) return SDV_ENOMEM;
+    while (ctx->run_ev->size() < 2 * (size_t)n_steps) {
+        cudaEvent_t ev;
+        CK(cudaEventCreate(&ev));
+        ctx->run_ev->push_back(ev);
+    }
+    int* state = ctx->P.state;
+    int* hist = (int*)(ctx->ws + ctx->r.hist);
+    const int hist_before = ctx->hist_len;
+    fill_i32_kernel<<<1, 32, 0, ctx->stream>>>(state + ST_BUDGET, max_tokens > 0 ? max_tokens : -1, 1);
+    const int* db = (const int*)(ctx->ws + ctx->r.db);
+    ngram_draft_kernel<<<1, 1024, 0, ctx->stream>>>(state, hist, db, c.ngram_n, c.ngram_min, k, c.search_history, 1);
+    if (ext_max_total > 0) extend_draft_kernel<<<1, 32, 0, ctx->stream>>>(state, ext_max_total, 1);
+    ctx->launches += ext_max_total > 0 ? 3 : 2;
+    const int all_phases = 2 + kPhasesPerLayer * c.n_layers;
+    for (int i = 0; i < n_steps; ++i) {
+        // the kernel reads the KV length from the state block; the host's value (a lower bound) only shapes the attention split
+        int rc = launch_forward(ctx, rows, ctx->kv_len, 0, 0, all_phases, true, false, false, nullptr, true,
+                                ctx->run_ev->data() + 2 * i);
+        if (rc) return rc;
+        // accept, commit and the next step's draft in one launch
+        step_tail_kernel<<<1, 1024, 0, ctx->stream>>>(state, hist, db, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, c.ngram_n,
+                                                      c.ngram_min, k, c.search_history, ext_max_total, ext_max_life,
+                                                      i + 1 < n_steps ? 1 : 0);
+        ctx->launches++;
+    }
+    CK(cudaGetLastError());
+    ctx->run_steps = n_steps;
+    ctx->verified = false;
+    ctx->draft_pending = false;
+    ctx->tree_pending = false;
+    ctx->tree_verified = false;
+    int rc = read_state(ctx);
+    if (rc) return rc;
+    ctx->kv_len = ctx->pinned[ST_KV_LEN];
+    ctx->hist_len = ctx->pinned[ST_HIST_LEN];
+    const int n = ctx->hist_len - hist_before;
+    if (n_tokens) *n_tokens = n;
+    if (kv_len) *kv_len = ctx->kv_len;
+    if (host_tokens && n > 0) {
+        CK(cudaMemcpyAsync(host_tokens, hist + hist_before, (size_t)n * 4, cudaMemcpyDeviceToHost, ctx->stream));
+        CK(cudaStreamSynchronize(ctx->stream));
+    }
+    return SDV_OK;
+}
+
+int sdv_run_kernel_ms(sdv_ctx* ctx, float* host_ms, int n) {
+    if (!ctx || !host_ms || n < 1) return SDV_EINVAL;
+    if (!ctx->run_ev || n > ctx->run_steps) return SDV_ESTATE;
+    CK(cudaStreamSynchronize(ctx->stream));
+    for (int i = 0; i < n; ++i) CK(cudaEventElapsedTime(&host_ms[i], (*ctx->run_ev)[2 * i], (*ctx->run_ev)[2 * i + 1]));
     return SDV_OK;
 }
 
@@ -1144,7 +1218,7 @@ int sdv_draft_tree(sdv_ctx* ctx, int k, int max_nodes, int32_t* host_tokens, int
     int* hist = (int*)(ctx->ws + ctx->r.hist);
     if (k > 0) {
         ngram_draft_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->P.state, hist, (const int*)(ctx->ws + ctx->r.db), ctx->cfg.ngram_n,
-                                                        ctx->cfg.ngram_min, k, ctx->cfg.search_history);
+                                                        ctx->cfg.ngram_min, k, ctx->cfg.search_history, 0);
     } else {
         DraftArg none;
         fill_draft_arg(none, nullptr, 0);
@@ -1201,7 +1275,7 @@ int sdv_verify_tree(sdv_ctx* ctx, const int32_t* host_tokens, const int32_t* hos
     }
     int rc = launch_forward(ctx, rows, ctx->kv_len, 0, 0, 2 + kPhasesPerLayer * c.n_layers, true, false, true);
     if (rc) return rc;
-    accept_kernel<<<1, 32 * rows, 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0, 0, nullptr);
+    accept_kernel<<<1, 32 * rows, 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 0, 0, nullptr, 0);
     ctx->launches++;
     CK(cudaGetLastError());
     ctx->verified = true;
@@ -1342,7 +1416,7 @@ int sdv_debug_accept(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, con
         ctx->launches++;
     }
     set_y_kernel<<<1, 32, 0, ctx->stream>>>(ctx->P.state, y);
-    accept_kernel<<<1, 32 * (draft_len + 1), 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 1, 0, nullptr);
+    accept_kernel<<<1, 32 * (draft_len + 1), 0, ctx->stream>>>(ctx->P.state, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, 1, 0, nullptr, 0);
     ctx->launches += 2;
     CK(cudaGetLastError());
     ctx->verified = true;

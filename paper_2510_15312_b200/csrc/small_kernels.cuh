@@ -74,8 +74,10 @@ __device__ __forceinline__ unsigned long long suffix_scan(const int* search, int
     return best;
 }
 
-__global__ void ngram_draft_kernel(int* state, const int* hist, const int* db, int n, int n_min, int k,
-                                   int search_history) {
+// `in_run` (all kernels of a step): the step was enqueued as part of a run with a token budget and does nothing
+// once the budget is used up.
+__device__ __forceinline__ void ngram_draft_body(int* state, const int* hist, const int* db, int n, int n_min, int k,
+                                                 int search_history) {
     __shared__ unsigned long long best_s[32];
     const int hist_len = state[ST_HIST_LEN];
     const int n_search = search_history ? hist_len : state[ST_N_CTX];
@@ -119,6 +121,11 @@ __global__ void ngram_draft_kernel(int* state, const int* hist, const int* db, i
             state[ST_TREE_ON] = 0;
         }
     }
+}
+__global__ void ngram_draft_kernel(int* state, const int* hist, const int* db, int n, int n_min, int k,
+                                   int search_history, int in_run) {
+    if (in_run && state[ST_BUDGET] == 0) return;
+    ngram_draft_body(state, hist, db, n, n_min, k, search_history);
 }
 
 __global__ void set_word_kernel(int* state, int word, int value) {
@@ -313,7 +320,7 @@ __global__ void set_y_kernel(int* state, DraftArg a) {
 //
 // extend: the retained segment is appended to the draft the drafter left, unless the draft would
 // grow beyond max_total tokens, in which case the segment is dropped.
-__global__ void extend_draft_kernel(int* state, int max_total) {
+__device__ __forceinline__ void extend_draft_body(int* state, int max_total) {  // one warp
     const int lane = threadIdx.x;
     const int m = state[ST_DRAFT_LEN], sl = state[ST_SEG_LEN];
     const bool fits = sl > 0 && m + sl <= max_total;
@@ -331,6 +338,10 @@ __global__ void extend_draft_kernel(int* state, int max_total) {
         }
     }
 }
+__global__ void extend_draft_kernel(int* state, int max_total, int in_run) {
+    if (in_run && state[ST_BUDGET] == 0) return;
+    extend_draft_body(state, max_total);
+}
 
 // update, after the accept scan of a verify step: lane i tests x_{i+1} == y_{i+1} beyond the reject
 // point; the longest run of agreeing drafts (the earliest among equals) is the candidate.  Runs of
@@ -338,7 +349,7 @@ __global__ void extend_draft_kernel(int* state, int max_total) {
 // i).  Then the retention rules: a segment that was appended ages by one step; it is dropped when
 // the accepted prefix reached into it or its age passes max_life; a strictly longer candidate
 // replaces what is retained.
-__global__ void extension_update_kernel(int* state, int max_life) {
+__device__ __forceinline__ void extension_update_body(int* state, int max_life) {  // one warp
     const int lane = threadIdx.x;
     const int dl = state[ST_DRAFT_LEN], a = state[ST_ACCEPT_LEN];
     const int x = state[ST_DRAFT + lane], y = state[ST_Y + lane];
@@ -374,6 +385,10 @@ __global__ void extension_update_kernel(int* state, int max_life) {
         state[ST_SEG_USED] = 0;
     }
 }
+__global__ void extension_update_kernel(int* state, int max_life, int in_run) {
+    if (in_run && state[ST_BUDGET] == 0) return;
+    extension_update_body(state, max_life);
+}
 
 // ------------------------------------------------------------------------------------------
 // Greedy tokens and accept scan.  Row j's token is the best of the per-block candidates
@@ -381,8 +396,8 @@ __global__ void extension_update_kernel(int* state, int max_life) {
 // prediction; emitted = x_1..x_a, y_{a+1}.  One block of 32 * rows threads: warp j reduces row j.
 // `row0`: the sequence's first row among the launch's rows (0 unless the step was batched); `launch_state`:
 // the state block the launch ran on when it is not `state` itself, whose error word is carried over.
-__global__ void accept_kernel(int* state, const float* cand_val, const int* cand_idx, int G, int from_host_y, int row0,
-                              const int* launch_state) {
+__device__ __forceinline__ void accept_body(int* state, const float* cand_val, const int* cand_idx, int G, int from_host_y,
+                                            int row0, const int* launch_state) {
     __shared__ int y_s[kMaxRows + 1];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int dl = state[ST_DRAFT_LEN];
@@ -437,6 +452,11 @@ __global__ void accept_kernel(int* state, const float* cand_val, const int* cand
         state[ST_VERIFIED] = 1;
     }
 }
+__global__ void accept_kernel(int* state, const float* cand_val, const int* cand_idx, int G, int from_host_y, int row0,
+                              const int* launch_state, int in_run) {
+    if (in_run && state[ST_BUDGET] == 0) return;
+    accept_body(state, cand_val, cand_idx, G, from_host_y, row0, launch_state);
+}
 
 // Batched verify: the token rows of up to kMaxBatch sequences (each its pending token, then its draft, token 0
 // past the draft's length) are laid out one after another in the state block the shared launch reads.
@@ -466,8 +486,17 @@ __global__ void batch_gather_kernel(int* launch_state, BatchGatherArg a) {
 // Commit: append the emitted tokens (cut to max_emit when > 0) to the history, advance the KV
 // length by their number, make the last one the pending token.  KV rows past the new length
 // are left as they are and overwritten by later steps.
-__global__ void commit_kernel(int* state, int* hist, int max_emit, int force_accept, int force_token) {
+__device__ __forceinline__ void commit_body(int* state, int* hist, int max_emit, int force_accept, int force_token, int in_run) {
     if (threadIdx.x != 0) return;
+    if (in_run) {  // the run's token budget cuts its last step and ends it
+        const int budget = state[ST_BUDGET];
+        if (budget == 0) return;
+        if (budget > 0) {
+            const int n0 = state[ST_N_EMITTED];
+            max_emit = budget;
+            state[ST_BUDGET] = budget - (n0 < budget ? n0 : budget);
+        }
+    }
     int n = state[ST_N_EMITTED];
     if (force_accept >= 0) {
         n = force_accept + 1;
@@ -485,6 +514,33 @@ __global__ void commit_kernel(int* state, int* hist, int max_emit, int force_acc
     state[ST_DRAFT_LEN] = 0;
     state[ST_VERIFIED] = 0;
     state[ST_TREE_ON] = 0;
+}
+__global__ void commit_kernel(int* state, int* hist, int max_emit, int force_accept, int force_token, int in_run) {
+    commit_body(state, hist, max_emit, force_accept, force_token, in_run);
+}
+
+// Everything between two forward kernels of a run of enqueued steps, in one launch of 1024 threads: the accept
+// scan of the step just verified, [the update of the retained segment,] its commit under the run's token
+// budget, and, unless the run ends here, the draft of the next step [and its extension].  The stages
+// meet at block barriers: what one writes to the state block and the history, the next reads.
+__global__ void __launch_bounds__(1024) step_tail_kernel(int* state, int* hist, const int* db, const float* cand_val,
+                                                         const int* cand_idx, int G, int n, int n_min, int k, int search_history,
+                                                         int ext_max_total, int ext_max_life, int draft_next) {
+    if (state[ST_BUDGET] == 0) return;   // enqueued behind the end of the run
+    accept_body(state, cand_val, cand_idx, G, 0, 0, nullptr);
+    __syncthreads();
+    if (ext_max_total > 0) {
+        if (threadIdx.x < 32) extension_update_body(state, ext_max_life);
+        __syncthreads();
+    }
+    commit_body(state, hist, 0, -1, 0, 1);
+    __syncthreads();
+    if (!draft_next || state[ST_BUDGET] == 0) return;
+    ngram_draft_body(state, hist, db, n, n_min, k, search_history);
+    if (ext_max_total > 0) {
+        __syncthreads();
+        if (threadIdx.x < 32) extend_draft_body(state, ext_max_total);
+    }
 }
 
 // After the last prefill tile: the greedy token of its last row becomes the pending token.
