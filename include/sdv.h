@@ -135,6 +135,18 @@ int sdv_set_database(sdv_ctx *ctx, const int32_t *host_tokens, int n);
  * Errors: SDV_ESTATE before prefill has finished, SDV_ECAPACITY, SDV_EINVAL, SDV_ETIMEOUT. */
 int sdv_verify(sdv_ctx *ctx, const int32_t *host_draft, int draft_len, int32_t *host_y, int *accept_len);
 
+/* One whole step in one call with one synchronisation (paper Sec. 4.1: verify, accept, then the next draft):
+ * verify host_draft (draft_len tokens, as sdv_verify; NULL: the draft on the device, left by sdv_draft or by
+ * the previous sdv_step), accept, commit, and, when k_next > 0, draft k_next tokens for the next step as
+ * sdv_draft would; accept scan, commit and draft are one launch behind the forward kernel.  The emitted tokens
+ * (host_emitted: k_max + 1 ints are always enough), their number, the new KV length and the next draft
+ * (host_next_draft: k_next ints; next_draft_len may be less than k_next, or 0) come back in one copy of the state
+ * block; any of the output pointers may be NULL.  Synchronises.  The retained segment of the draft extension is
+ * not updated by this call.  Errors: SDV_EINVAL, SDV_ESTATE (before the end of prefill; a tree draft pending),
+ * SDV_ECAPACITY, SDV_ETIMEOUT. */
+int sdv_step(sdv_ctx *ctx, const int32_t *host_draft, int draft_len, int k_next, int32_t *host_emitted,
+             int *n_emitted, int32_t *host_next_draft, int *next_draft_len, int *kv_len);
+
 /* A run of decoding steps without the host in between (paper Sec. 4.1, online workflow: draft -> verify ->
  * accept repeated until the answer ends).  Enqueues n_steps (1..4096) steps of sdv_draft(k) [+
  * sdv_extend_draft(ext_max_total) when ext_max_total > 0] -> sdv_verify -> [sdv_extension_update(ext_max_life)]

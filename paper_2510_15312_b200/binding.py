@@ -22,7 +22,7 @@ EXPORTS = [
     "sdv_set_calibration", "sdv_get_calibration", "sdv_draft_tree", "sdv_verify_tree", "sdv_debug_force_commit_tree",
     "sdv_debug_top_successors",
     "sdv_follower_workspace_bytes", "sdv_create_follower", "sdv_verify_batch", "sdv_get_verified",
-    "sdv_decode_steps", "sdv_run_kernel_ms",
+    "sdv_decode_steps", "sdv_run_kernel_ms", "sdv_step",
 ]
 
 
@@ -85,6 +85,7 @@ def load_library(path: Optional[str] = None):
     L.sdv_get_verified.argtypes = [vp, i32p, ip]
     L.sdv_decode_steps.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, i32p, ip, ip]
     L.sdv_run_kernel_ms.argtypes = [vp, vp, C.c_int]
+    L.sdv_step.argtypes = [vp, i32p, C.c_int, C.c_int, i32p, ip, i32p, ip, ip]
     L.sdv_strerror.argtypes = [C.c_int]
     L.sdv_strerror.restype = C.c_char_p
     L.sdv_last_cuda_error.argtypes = [vp]
@@ -230,6 +231,18 @@ class Sdv:
         a = (C.c_int * len(seqs))()
         seqs[0]._check(lib().sdv_verify_batch(hs, len(seqs), a if fetch else None), "sdv_verify_batch")
         return list(a) if fetch else None
+
+    def step(self, draft: Optional[Sequence[int]], k_next: int) -> Tuple[List[int], List[int], int]:
+        """Verify `draft` (None: the device draft), accept, commit and draft k_next tokens for the next step:
+        one call, one synchronisation.  Returns (emitted tokens, next draft, KV length)."""
+        d = None if draft is None else np.ascontiguousarray(draft, dtype=np.int32)
+        dp = None if d is None else (d.ctypes.data if len(d) else np.zeros(1, np.int32).ctypes.data)
+        em = np.zeros(K_MAX + 1, dtype=np.int32)
+        nd = np.zeros(K_MAX + 1, dtype=np.int32)
+        n, ndl, kv = C.c_int(0), C.c_int(0), C.c_int(0)
+        self._check(lib().sdv_step(self._h, dp, 0 if d is None else len(d), k_next, em.ctypes.data, C.byref(n),
+                                   nd.ctypes.data, C.byref(ndl), C.byref(kv)), "sdv_step")
+        return em[:n.value].tolist(), nd[:ndl.value].tolist(), kv.value
 
     def decode_steps(self, k: int, n_steps: int, max_tokens: int = 0, ext_max_total: int = 0,
                      ext_max_life: int = 0) -> Tuple[List[int], int]:

@@ -1125,6 +1125,59 @@ int sdv_extension_update(sdv_ctx* ctx, int max_life, int32_t* host_segment, int*
     return SDV_OK;
 }
 
+int sdv_step(sdv_ctx* ctx, const int32_t* host_draft, int draft_len, int k_next, int32_t* host_emitted, int* n_emitted,
+             int32_t* host_next_draft, int* next_draft_len, int* kv_len) {
+    if (!ctx || k_next < 0 || k_next > ctx->cfg.k_max) return SDV_EINVAL;
+    if (ctx->poisoned) return SDV_ETIMEOUT;
+    if (!ctx->prefill_done || !ctx->weights_loaded) return SDV_ESTATE;
+    const sdv_config& c = ctx->cfg;
+    int rows;
+    if (host_draft) {
+        if (draft_len < 0 || draft_len > c.k_max) return SDV_EINVAL;
+        for (int i = 0; i < draft_len; ++i)
+            if (host_draft[i] < 0 || host_draft[i] >= c.vocab) return SDV_EINVAL;
+        rows = draft_len + 1;
+    } else {
+        if (ctx->tree_pending) return SDV_ESTATE;  // chains only
+        rows = ctx->draft_pending ? ctx->draft_k + 1 : 1;
+    }
+    if (ctx->kv_len + rows > c.max_seq || ctx->hist_len + rows > c.max_seq + 64) return SDV_ECAPACITY;
+    int* state = ctx->P.state;
+    int* hist = (int*)(ctx->ws + ctx->r.hist);
+    if (host_draft) {
+        DraftArg a;
+        fill_draft_arg(a, host_draft, draft_len);
+        set_draft_kernel<<<1, 32, 0, ctx->stream>>>(state, a);
+        ctx->launches++;
+    }
+    int rc = launch_forward(ctx, rows, ctx->kv_len, 0, 0, 2 + kPhasesPerLayer * c.n_layers, true);
+    if (rc) return rc;
+    step_tail_kernel<<<1, 1024, 0, ctx->stream>>>(state, hist, (const int*)(ctx->ws + ctx->r.db), ctx->P.cand_val, ctx->P.cand_idx,
+                                                  ctx->G, c.ngram_n, c.ngram_min, k_next, c.search_history, 0, 0, k_next > 0 ? 1 : 0, 0);
+    ctx->launches++;
+    CK(cudaGetLastError());
+    ctx->last_rows = rows;
+    ctx->verified = false;
+    ctx->tree_pending = false;
+    ctx->tree_verified = false;
+    ctx->draft_pending = k_next > 0;
+    ctx->draft_k = k_next;
+    rc = read_state(ctx);  // one copy of the state block: emitted tokens, lengths and the next draft
+    if (rc) return rc;
+    const int n = ctx->pinned[ST_N_EMITTED];
+    ctx->kv_len = ctx->pinned[ST_KV_LEN];
+    ctx->hist_len = ctx->pinned[ST_HIST_LEN];
+    if (n_emitted) *n_emitted = n;
+    if (kv_len) *kv_len = ctx->kv_len;
+    if (host_emitted)
+        for (int i = 0; i < n; ++i) host_emitted[i] = ctx->pinned[ST_EMITTED + i];
+    const int dl = k_next > 0 ? ctx->pinned[ST_DRAFT_LEN] : 0;
+    if (next_draft_len) *next_draft_len = dl;
+    if (host_next_draft)
+        for (int i = 0; i < dl; ++i) host_next_draft[i] = ctx->pinned[ST_DRAFT + i];
+    return SDV_OK;
+}
+
 int sdv_decode_steps(sdv_ctx* ctx, int k, int n_steps, int max_tokens, int ext_max_total, int ext_max_life, int32_t* host_tokens,
                      int* n_tokens, int* kv_len) {
     if (!ctx || k < 1 || k > ctx->cfg.k_max || n_steps < 1 || n_steps > 4096) return SDV_EINVAL;
@@ -1161,7 +1214,7 @@ int sdv_decode_steps(sdv_ctx* ctx, int k, int n_steps, int max_tokens, int ext_m
         // accept, commit and the next step's draft in one launch
         step_tail_kernel<<<1, 1024, 0, ctx->stream>>>(state, hist, db, ctx->P.cand_val, ctx->P.cand_idx, ctx->G, c.ngram_n,
                                                       c.ngram_min, k, c.search_history, ext_max_total, ext_max_life,
-                                                      i + 1 < n_steps ? 1 : 0);
+                                                      i + 1 < n_steps ? 1 : 0, 1);
         ctx->launches++;
     }
     CK(cudaGetLastError());

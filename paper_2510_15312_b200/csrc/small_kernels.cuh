@@ -519,23 +519,23 @@ __global__ void commit_kernel(int* state, int* hist, int max_emit, int force_acc
     commit_body(state, hist, max_emit, force_accept, force_token, in_run);
 }
 
-// Everything between two forward kernels of a run of enqueued steps, in one launch of 1024 threads: the accept
+// Everything between two forward kernels (of a run of enqueued steps, or of sdv_step), in one launch of 1024 threads: the accept
 // scan of the step just verified, [the update of the retained segment,] its commit under the run's token
 // budget, and, unless the run ends here, the draft of the next step [and its extension].  The stages
 // meet at block barriers: what one writes to the state block and the history, the next reads.
 __global__ void __launch_bounds__(1024) step_tail_kernel(int* state, int* hist, const int* db, const float* cand_val,
                                                          const int* cand_idx, int G, int n, int n_min, int k, int search_history,
-                                                         int ext_max_total, int ext_max_life, int draft_next) {
-    if (state[ST_BUDGET] == 0) return;   // enqueued behind the end of the run
+                                                         int ext_max_total, int ext_max_life, int draft_next, int in_run) {
+    if (in_run && state[ST_BUDGET] == 0) return;   // enqueued behind the end of the run
     accept_body(state, cand_val, cand_idx, G, 0, 0, nullptr);
     __syncthreads();
     if (ext_max_total > 0) {
         if (threadIdx.x < 32) extension_update_body(state, ext_max_life);
         __syncthreads();
     }
-    commit_body(state, hist, 0, -1, 0, 1);
+    commit_body(state, hist, 0, -1, 0, in_run);
     __syncthreads();
-    if (!draft_next || state[ST_BUDGET] == 0) return;
+    if (!draft_next || (in_run && state[ST_BUDGET] == 0)) return;
     ngram_draft_body(state, hist, db, n, n_min, k, search_history);
     if (ext_max_total > 0) {
         __syncthreads();

@@ -141,3 +141,40 @@ def test_run_argument_and_capacity_errors():
     out, kv = s.decode_steps(cfg.k, 8)
     assert kv == cfg.n_ctx + len(out) and len(out) >= 8
     s.close()
+
+
+@pytest.mark.parametrize("name", ["tiny", "mini_gqa"])
+def test_one_call_step_equals_draft_verify_commit(name):
+    """sdv_step against the same step made of sdv_draft / sdv_verify / sdv_commit on a second sequence: emitted
+    tokens, KV length and the draft handed back for the next step, with host drafts and with the device's."""
+    cfg = get_config(name)
+    w, ctx = make_weights(cfg), make_context(cfg)
+    toks, _, first_tie = oracle_stream(cfg, w, ctx)
+    a = Sdv(config_from(cfg, search_history=True, max_seq=cfg.n_ctx + 2 * cfg.gen * (cfg.k + 1) + 64))
+    a.load_weights(w)
+    b = a.follower()
+    for s in (a, b):
+        gpu_prefill(s, ctx, cfg.chunk)
+    da = a.draft(cfg.k)
+    db = b.draft(cfg.k)
+    assert da == db
+    out_a, out_b = [], []
+    for i in range(min(cfg.gen - 2, 16)):
+        ya, _ = a.verify(da if i % 2 else None)          # host draft on odd steps, the device's own on even ones
+        ea, kva = a.commit()
+        da = a.draft(cfg.k)
+        eb, db, kvb = b.step(db if i % 2 else None, cfg.k)
+        out_a += ea
+        out_b += eb
+        if out_a != out_b:
+            assert matched_prefix(out_a, out_b) + 1 >= first_tie   # parted at a near-tie only
+            break
+        assert kva == kvb == b.kv_len() and da == db
+    assert len(out_b) >= 4 and matched_prefix(out_b, toks[1:]) >= max(0, min(first_tie, len(out_b) + 1) - 1)
+    eb, db, _ = b.step(None, 0)                          # no next draft asked for
+    assert db == [] and len(eb) >= 1
+    with pytest.raises(SdvError) as e:
+        b.step([cfg.vocab], cfg.k)
+    assert e.value.code == B.EINVAL
+    b.close()
+    a.close()
