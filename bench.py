@@ -376,7 +376,8 @@ def main():
         em, _ = s.decode_steps(k, n)
         return len(em), [float(x) for x in s.run_kernel_ms(n)]
 
-    sampler = ClockSampler(local)
+    # the period is only as short as 20 ms when the timed regions would otherwise end before the second sample
+    sampler = ClockSampler(local, period_ms=20 if 2 * total * 1.5 < 400 else 200)
     sampler.start()                      # before the warm-up: the first samples arrive while it runs
     run(args.warmup)
     launches0 = s.launch_count()
