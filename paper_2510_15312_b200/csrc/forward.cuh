@@ -182,25 +182,26 @@ __device__ __noinline__ void build_norm_operand(const FwdParams& P, int kind, in
     for (int row = warp; row < M; row += kBuilderWarps) {
         const float4* src = reinterpret_cast<const float4*>(xbase + (size_t)row * stride) + k4_0;
         const float4* wsrc = wn ? reinterpret_cast<const float4*>(wn) + k4_0 : nullptr;
+        const float4* wld = wsrc ? wsrc : src;  // without norm weights the loaded value is not used
         float ss = 0.f;
         for (int base = lane; base < nk4; base += 32 * UB) {
             float4 a[UB], w[UB];
+            // every unit loads (past the end: the row's last unit again, not used), so that the loads are one
+            // straight run of instructions instead of a branch per unit
 #pragma unroll
             for (int u = 0; u < UB; ++u) {
-                const int k4 = base + u * 32;
-                a[u] = w[u] = make_float4(1.f, 1.f, 1.f, 1.f);
-                if (k4 < nk4) {
-                    a[u] = ld_cg_f4_inorder(src + k4);
-                    if (wsrc) w[u] = ld_nc_f4_inorder(wsrc + k4);
-                }
+                const int k4 = min(base + u * 32, nk4 - 1);
+                a[u] = ld_cg_f4_inorder(src + k4);
+                w[u] = ld_nc_f4_inorder(wld + k4);
             }
 #pragma unroll
             for (int u = 0; u < UB; ++u) {
                 const int k4 = base + u * 32;
                 if (k4 < nk4) {
                     const float4 x = a[u];
+                    const float4 g = wsrc ? w[u] : make_float4(1.f, 1.f, 1.f, 1.f);
                     ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
-                    const uint2 out = make_uint2(pack_bf16(x.x * w[u].x, x.y * w[u].y), pack_bf16(x.z * w[u].z, x.w * w[u].w));
+                    const uint2 out = make_uint2(pack_bf16(x.x * g.x, x.y * g.y), pack_bf16(x.z * g.z, x.w * g.w));
                     *reinterpret_cast<uint2*>(U + operand_off(k4 >> 1, row, M) + (k4 & 1) * 8) = out;
                 }
             }
@@ -235,21 +236,19 @@ __device__ __noinline__ void build_merged_operand(const FwdParams& P, const Part
         const size_t base = ((size_t)hq * (kMaxSplits + 1)) * kMaxRows + j;
         float m[TPL], l[TPL];
         float4 a[TPL], b[TPL];
+        // every slot loads (beyond the last partial result: the last one again, given no weight below), so that
+        // the loads are one straight run of instructions instead of a branch per slot
 #pragma unroll
         for (int t = 0; t < TPL; ++t) {
             const int s = sub + 4 * t;
-            m[t] = -CUDART_INF_F;
-            l[t] = 0.f;
-            a[t] = b[t] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (live && s < S1) {
-                const size_t row = base + (size_t)s * kMaxRows;
-                const float2 ml = ld_cg_f2_inorder(P.part_ml + row * 2);
-                m[t] = ml.x;
-                l[t] = ml.y;
-                const float* op = P.part_o + row * hd + c;
-                a[t] = ld_cg_f4_inorder(op);
-                b[t] = ld_cg_f4_inorder(op + 4);
-            }
+            const size_t row = base + (size_t)min(s, S) * kMaxRows;
+            const float2 ml = ld_cg_f2_inorder(P.part_ml + row * 2);
+            const float* op = P.part_o + row * hd + c;
+            a[t] = ld_cg_f4_inorder(op);
+            b[t] = ld_cg_f4_inorder(op + 4);
+            const bool use = live && s < S1;
+            m[t] = use ? ml.x : -CUDART_INF_F;
+            l[t] = use ? ml.y : 0.f;
         }
         float mmax = m[0];
 #pragma unroll
