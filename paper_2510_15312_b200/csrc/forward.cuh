@@ -104,7 +104,7 @@ __device__ __forceinline__ bool grid_barrier(const FwdParams& P, unsigned target
 
 // ------------------------------------------------------------------------------------------
 // Weight streamer (one thread).
-__device__ __noinline__ void producer_loop(const FwdParams& P, uint8_t* smem, Misc* misc) {
+__device__ __forceinline__ void producer_loop(const FwdParams& P, uint8_t* smem, Misc* misc) {
     const uint64_t policy = l2_policy_evict_first();
     const uint32_t nstage = (uint32_t)P.nstage;
     uint32_t slot = 0, par = 0, issued = 0;  // ring position; parity of the current trip round the ring
@@ -168,7 +168,7 @@ __device__ __forceinline__ uint32_t operand_off(int k8, int row, int M) {
 // batch are issued before the first use.  Leaves the rows' sums of squares over this block's
 // columns in misc->sumsq; QKV blocks of row partition 0 also add them to the global sums the
 // attention step reads.
-__device__ __noinline__ void build_norm_operand(const FwdParams& P, int kind, int layer, const Part& pt, uint8_t* U,
+__device__ __forceinline__ void build_norm_operand(const FwdParams& P, int kind, int layer, const Part& pt, uint8_t* U,
                                                 Misc* misc, int wtid) {
     constexpr int UB = 12;  // 4-column units per lane and batch; a warp instruction reads 512 contiguous bytes
     const int warp = wtid >> 5, lane = wtid & 31;
@@ -220,7 +220,7 @@ __device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps)
 // Operand of the output projection = attention output of this block's columns: the split-KV
 // partial results (un-normalised sums with their running maximum and sum) are merged on the way.
 // Four lanes share one (row, 8 columns) item, each taking every fourth partial result.
-__device__ __noinline__ void build_merged_operand(const FwdParams& P, const Part& pt, uint8_t* U, int wtid) {
+__device__ __forceinline__ void build_merged_operand(const FwdParams& P, const Part& pt, uint8_t* U, int wtid) {
     constexpr int TPL = (kMaxSplits + 1 + 3) / 4;  // partial results per lane at most
     int S, kps;
     attn_split(P, S, kps);
@@ -501,7 +501,7 @@ __device__ __forceinline__ void argmax_finish(const FwdParams& P, Misc* misc, in
 }
 
 template <int NBT>
-__device__ __noinline__ void epilogue_phase(const FwdParams& P, int kind, int layer, uint8_t* act, Misc* misc, PipePos& pos,
+__device__ __forceinline__ void epilogue_phase(const FwdParams& P, int kind, int layer, uint8_t* act, Misc* misc, PipePos& pos,
                                             bool& dead, int warp, int lane) {
     float bv[NBT];
     int bi[NBT];
@@ -933,7 +933,7 @@ __device__ __forceinline__ void advance_pos(PipePos& pos, const Part& pt, uint32
     pos.q += (uint32_t)pt.npass;
 }
 
-__device__ __noinline__ void gemm_phase(const FwdParams& P, int kind, int layer, uint8_t* smem, Misc* misc, PipePos& pos, int wtid,
+__device__ __forceinline__ void gemm_phase(const FwdParams& P, int kind, int layer, uint8_t* smem, Misc* misc, PipePos& pos, int wtid,
                                         unsigned long long* prof) {
     const int warp = wtid >> 5, lane = wtid & 31;
     uint8_t* U = smem + P.u_off;
