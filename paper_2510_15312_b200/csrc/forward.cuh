@@ -364,6 +364,37 @@ __device__ __forceinline__ void mma_op(const FwdParams& P, const Part& pt, uint8
 // ------------------------------------------------------------------------------------------
 // Epilogues (warps 0..7).  Thread t = 32 * (warp & 3) + lane owns row t of its 128-row accumulator,
 // i.e. one weight row (output feature), for the token columns its warp group takes.
+// SwiGLU on one accumulator row per thread.  Rows 0..7 of a 16-row tile are gate rows, rows 8..15 the
+// matching up rows, so the two values of an output sit 8 lanes apart.  Token columns are taken in
+// pairs: the gate lane evaluates the even column of a pair, the up lane the odd one; one shuffle per
+// pair hands each lane the partner's value it needs.  All pairs are independent and written without
+// branches, so that their shuffles, exponentials and divisions overlap.  SEL >= 0: only pairs j with
+// (j & 1) == SEL (the other group of epilogue warps takes the rest).
+template <int NBT, int SEL>
+__device__ __forceinline__ void swiglu_pairs(const float (&v)[NBT], const float (&rstd)[NBT], int t, bool valid, int M,
+                                             uint8_t* dst) {
+    constexpr int STEP = SEL < 0 ? 1 : 2, J0 = SEL < 0 ? 0 : SEL, NP = (NBT / 2 - J0 + STEP - 1) / STEP;
+    const bool is_up = (t & 8) != 0;
+    float got[NP], out[NP];
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+        const int j = J0 + i * STEP;
+        got[i] = __shfl_xor_sync(0xffffffffu, is_up ? v[2 * j] : v[2 * j + 1], 8);
+    }
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+        const int j = J0 + i * STEP;
+        const float mine = is_up ? v[2 * j + 1] : v[2 * j], r = is_up ? rstd[2 * j + 1] : rstd[2 * j];
+        const float x = (is_up ? got[i] : mine) * r, y = (is_up ? mine : got[i]) * r;
+        out[i] = __fdividef(x, 1.f + __expf(-x)) * y;
+    }
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+        const int n = 2 * (J0 + i * STEP) + (is_up ? 1 : 0);
+        if (valid && n < M) *reinterpret_cast<__nv_bfloat16*>(dst + n * 16) = __float2bfloat16(out[i]);
+    }
+}
+
 template <int NBT>  // token columns read: 16 or 32
 __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op, int layer, const Part& pt, uint8_t* act, Misc* misc,
                                             PipePos& pos, bool& dead, int warp, int lane, float (&bv)[NBT], int (&bi)[NBT]) {
@@ -422,18 +453,11 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
             if (op == OP_GU) {
                 // rows 0..7 of a tile are gate rows, 8..15 the matching up rows, 8 lanes apart: the gate
                 // lane evaluates the even token columns, the up lane the odd ones
-                const bool is_up = (t & 8) != 0;
                 const int col = (pstart + (tt >> 4)) * 8 + (tt & 7);  // SwiGLU column within this block's slice
                 uint8_t* dst = act + operand_off(col >> 3, 0, M) + (col & 7) * 2;
-#pragma unroll
-                for (int n = 0; n < NBT; ++n) {
-                    const float other = __shfl_xor_sync(0xffffffffu, v[n], 8);
-                    if (valid && n < M && ((n & 1) != 0) == is_up && (nsel < 0 || ((n >> 1) & 1) == nsel)) {
-                        const float x = (is_up ? other : v[n]) * rstd[n], y = (is_up ? v[n] : other) * rstd[n];
-                        const float a = __fdividef(x, 1.f + __expf(-x)) * y;
-                        *reinterpret_cast<__nv_bfloat16*>(dst + n * 16) = __float2bfloat16(a);
-                    }
-                }
+                if (nsel < 0) swiglu_pairs<NBT, -1>(v, rstd, t, valid, M, dst);
+                else if (nsel == 0) swiglu_pairs<NBT, 0>(v, rstd, t, valid, M, dst);
+                else swiglu_pairs<NBT, 1>(v, rstd, t, valid, M, dst);
             } else if (op == OP_LM) {
 #pragma unroll
                 for (int n = 0; n < NBT; ++n) {
@@ -536,6 +560,10 @@ __device__ __forceinline__ void epilogue_phase(const FwdParams& P, int kind, int
 // The heads per group are chosen on the host per launch; the key ranges follow from it: as many
 // as there are blocks to take a (KV head, head group, range) unit each, at most kMaxSplits.
 __device__ __forceinline__ void attn_split(const FwdParams& P, int& S, int& kps) {
+    S = P.att_S;      // worked out once per launch (attn_split_compute): the divisions are not repeated per phase
+    kps = P.att_kps;
+}
+__device__ __forceinline__ void attn_split_compute(const FwdParams& P, int& S, int& kps) {
     if (P.L <= 0) { S = 0; kps = 0; return; }
     const int QG = (P.g + P.att_gh - 1) / P.att_gh;
     int cap = P.G / (P.n_kv * QG) - 1;
@@ -1043,8 +1071,12 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    // the first reader of L (the attention phase) comes after a grid barrier, which orders this write before it
-    if (tid == 0 && Pg.l_from_state) misc->P.L = Pg.state[ST_KV_LEN];
+    // the first reader of L and of the key ranges (the attention phase) comes after a grid barrier, which orders
+    // these writes before it
+    if (tid == 0) {
+        if (Pg.l_from_state) misc->P.L = Pg.state[ST_KV_LEN];
+        attn_split_compute(misc->P, misc->P.att_S, misc->P.att_kps);
+    }
 
     if (warp == kProducerWarp) {
         if (lane == 0) producer_loop(P, smem, misc);

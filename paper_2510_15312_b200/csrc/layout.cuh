@@ -219,6 +219,7 @@ struct FwdParams {
     int M;             // rows computed (1..kMaxRows)
     int NB;            // N of the tensor-core instruction: 16, or 32 when M > 16
     int att_gh;        // attention split: query heads per unit (the key ranges follow from it)
+    int att_S, att_kps;  // key ranges and keys per range: derived from L and att_gh by the kernel when it starts
     int mode;          // 0: rows are [pending, draft...]; 1: rows are hist[L..L+M)
     int ph_begin, ph_end;
     unsigned bar_base; // barrier counter value before this launch
