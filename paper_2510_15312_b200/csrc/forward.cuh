@@ -897,12 +897,18 @@ __device__ void attention_phase(const FwdParams& P, int layer, uint8_t* att, int
     int S, kps;
     attn_split(P, S, kps);
     const int S1 = S + 1;
-    const int gh = P.att_gh, QG = (P.g + gh - 1) / gh;
-    const int per_seq = P.n_kv * QG * S1;
+    const int gh = P.att_gh, QG = P.att_QG;
+    const int per_seq = P.att_per_seq;
     const int nunits = per_seq * (P.nseq > 0 ? P.nseq : 1);
     for (int unit = blockIdx.x; unit < nunits; unit += P.G) {
-        const int b = unit / per_seq, u = unit % per_seq;
-        const int hk = u / (QG * S1), rem = u % (QG * S1), qg = rem / S1, s = rem % S1;
+        int b = P.att_b0, hk = P.att_hk0, qg = P.att_qg0, s = P.att_s0;
+        if (unit != (int)blockIdx.x) {  // further units of this block (more units than blocks: batched steps)
+            const int u = unit % per_seq, rem = u % (QG * S1);
+            b = unit / per_seq;
+            hk = u / (QG * S1);
+            qg = rem / S1;
+            s = rem % S1;
+        }
         if (P.nseq > 0) {
             // every sequence takes the key ranges of the longest one; a range past its own length holds no key
             if (P.hd == 128) attention_unit<128, 2>(P, layer, hk, qg, gh, s, S, kps, att, wtid, prof, b);
@@ -1076,6 +1082,16 @@ __global__ void __launch_bounds__(kThreads, 1) sdv_forward_kernel(const __grid_c
     if (tid == 0) {
         if (Pg.l_from_state) misc->P.L = Pg.state[ST_KV_LEN];
         attn_split_compute(misc->P, misc->P.att_S, misc->P.att_kps);
+        // the block's first attention unit: the same for every layer, so its index arithmetic is done here
+        FwdParams& Q = misc->P;
+        const int S1 = Q.att_S + 1;
+        Q.att_QG = (Q.g + Q.att_gh - 1) / Q.att_gh;
+        Q.att_per_seq = Q.n_kv * Q.att_QG * S1;
+        const int unit = blockIdx.x, u = unit % Q.att_per_seq, rem = u % (Q.att_QG * S1);
+        Q.att_b0 = unit / Q.att_per_seq;
+        Q.att_hk0 = u / (Q.att_QG * S1);
+        Q.att_qg0 = rem / S1;
+        Q.att_s0 = rem % S1;
     }
 
     if (warp == kProducerWarp) {

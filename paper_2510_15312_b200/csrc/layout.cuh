@@ -220,6 +220,8 @@ struct FwdParams {
     int NB;            // N of the tensor-core instruction: 16, or 32 when M > 16
     int att_gh;        // attention split: query heads per unit (the key ranges follow from it)
     int att_S, att_kps;  // key ranges and keys per range: derived from L and att_gh by the kernel when it starts
+    int att_QG, att_per_seq;            // head groups per KV head; attention units per sequence
+    int att_b0, att_hk0, att_qg0, att_s0;  // the block's first attention unit, decoded (each block works this out for itself)
     int mode;          // 0: rows are [pending, draft...]; 1: rows are hist[L..L+M)
     int ph_begin, ph_end;
     unsigned bar_base; // barrier counter value before this launch
