@@ -395,9 +395,12 @@ __device__ __forceinline__ void swiglu_pairs(const float (&v)[NBT], const float 
     }
 }
 
-template <int NBT>  // token columns read: 16 or 32
+// LM: the operation is the LM head (bv / bi carry the running best logit per token row); the other operations
+// are compiled without that state, which would otherwise occupy 2 x NBT registers through every phase.
+template <int NBT, bool LM>  // NBT: token columns read, 16 or 32
 __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op, int layer, const Part& pt, uint8_t* act, Misc* misc,
-                                            PipePos& pos, bool& dead, int warp, int lane, float (&bv)[NBT], int (&bi)[NBT]) {
+                                            PipePos& pos, bool& dead, int warp, int lane, float (&bv)[LM ? NBT : 1],
+                                            int (&bi)[LM ? NBT : 1]) {
     const int M = P.M;
     const int quarter = warp & 3, myhalf = warp >> 2;  // this warp's 32 accumulator lanes; which of the two accumulators
     const int t = quarter * 32 + lane;
@@ -405,7 +408,7 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
     const uint32_t tmem_lane = misc->tmem_base + ((uint32_t)(quarter * 32) << 16);
     const int npass = pt.npass, tile0 = pt.tile0;
     float rstd[NBT];
-    if (op == OP_GU || op == OP_LM) {
+    if (op == OP_GU || LM) {
         const float inv_d = 1.f / (float)P.d, eps = P.eps;
 #pragma unroll
         for (int n = 0; n < NBT; ++n) rstd[n] = (n < M) ? rsqrtf(misc->sumsq[n] * inv_d + eps) : 0.f;
@@ -450,7 +453,7 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
             const int tt = half * 128 + t;         // row within the pass
             const bool valid = tt < 16 * pcount;
             const int row = (tile0 + pstart) * 16 + tt;  // weight row = output feature
-            if (op == OP_GU) {
+            if (!LM && op == OP_GU) {
                 // rows 0..7 of a tile are gate rows, 8..15 the matching up rows, 8 lanes apart: the gate
                 // lane evaluates the even token columns, the up lane the odd ones
                 const int col = (pstart + (tt >> 4)) * 8 + (tt & 7);  // SwiGLU column within this block's slice
@@ -458,14 +461,14 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
                 if (nsel < 0) swiglu_pairs<NBT, -1>(v, rstd, t, valid, M, dst);
                 else if (nsel == 0) swiglu_pairs<NBT, 0>(v, rstd, t, valid, M, dst);
                 else swiglu_pairs<NBT, 1>(v, rstd, t, valid, M, dst);
-            } else if (op == OP_LM) {
+            } else if (LM) {
 #pragma unroll
                 for (int n = 0; n < NBT; ++n) {
                     if (valid && n < M && (nsel < 0 || ((n >> 1) & 1) == nsel)) {
                         const float x = v[n] * rstd[n];
                         if (store_logits) __stcg(P.logits + (size_t)n * P.V + row, x);
                         // rows come in ascending order per thread, so ">" keeps the lowest id among equals
-                        if (x > bv[n]) { bv[n] = x; bi[n] = row; }
+                        if (x > bv[LM ? n : 0]) { bv[LM ? n : 0] = x; bi[LM ? n : 0] = row; }
                     }
                 }
             } else if (valid) {
@@ -482,7 +485,7 @@ __device__ __forceinline__ void epilogue_op(const FwdParams& P, int kind, int op
             }
         }
     }
-    if (op == OP_GU) {
+    if (!LM && op == OP_GU) {
         // this warp's SwiGLU columns are written: hand them to the tensor-core thread
         fence_proxy_async_smem();
         __syncwarp();
@@ -527,18 +530,25 @@ __device__ __forceinline__ void argmax_finish(const FwdParams& P, Misc* misc, in
 template <int NBT>
 __device__ __forceinline__ void epilogue_phase(const FwdParams& P, int kind, int layer, uint8_t* act, Misc* misc, PipePos& pos,
                                             bool& dead, int warp, int lane) {
-    float bv[NBT];
-    int bi[NBT];
+    if (kind == PH_LM) {
+        float bv[NBT];
+        int bi[NBT];
 #pragma unroll
-    for (int n = 0; n < NBT; ++n) { bv[n] = -CUDART_INF_F; bi[n] = 0x7fffffff; }
+        for (int n = 0; n < NBT; ++n) { bv[n] = -CUDART_INF_F; bi[n] = 0x7fffffff; }
+        const Part& pt = misc->part[OP_LM];
+        if (pt.ntiles > 0 && pt.nk > 0) epilogue_op<NBT, true>(P, kind, OP_LM, layer, pt, act, misc, pos, dead, warp, lane, bv, bi);
+        argmax_finish<NBT>(P, misc, warp, lane, bv, bi, dead);
+        return;
+    }
+    float none_v[1];
+    int none_i[1];
     int ops[2];
     const int nops = phase_ops(kind, ops);
     for (int oi = 0; oi < nops; ++oi) {
         const Part& pt = misc->part[ops[oi]];
         if (pt.ntiles == 0 || pt.nk == 0) continue;
-        epilogue_op<NBT>(P, kind, ops[oi], layer, pt, act, misc, pos, dead, warp, lane, bv, bi);
+        epilogue_op<NBT, false>(P, kind, ops[oi], layer, pt, act, misc, pos, dead, warp, lane, none_v, none_i);
     }
-    if (kind == PH_LM) argmax_finish<NBT>(P, misc, warp, lane, bv, bi, dead);
 }
 
 // ------------------------------------------------------------------------------------------
