@@ -1,7 +1,7 @@
 """GPU-vs-oracle parity of the whole path (prefill, draft, verify, accept, commit) through the
 C-ABI.  Tolerances: drafts, accept lengths and KV lengths bit-exact; logits max |d| <= 0.05 and
 cosine >= 0.999 per row; greedy tokens identical except where the oracle's own top-2 margin is
-below 0.05 (then the other token must be the oracle's runner-up)."""
+below 0.05 (then the other token's oracle logit must lie within 0.05 of the oracle's best)."""
 import os
 
 import numpy as np
