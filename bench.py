@@ -34,7 +34,7 @@ UNIT = "tokens/s"
 # algorithmic bytes: from an ncu capture on the 0.5B-shaped workload, scaled to the timed workload by its
 # algorithmic bytes (traffic grows with the bytes streamed).  None once the kernel has changed since the
 # capture.
-NCU_TRAFFIC_RATIO = 1.0041
+NCU_TRAFFIC_RATIO = 1.0039
 
 
 NOMINAL_HBM_GBS = 8000.0   # the "about 8 TB/s" the target is worded against
